@@ -1,0 +1,125 @@
+"""Bit-exact FP8-E4M3 codec and block quantisation (oracle; test infrastructure only).
+
+Section 2.1 of the paper gives symmetric quantisation as
+``Q(X) = clamp(round(X / s)) * s`` with ``s = max|X| / q_max`` and names FP8-E4M3
+(4 exponent bits, 3 mantissa bits) as the grid.  The paper says nothing more
+about the format, so the published OCP 8-bit floating point definition is used:
+
+* 1 sign bit, 4 exponent bits (bias 7), 3 mantissa bits;
+* no infinities; the only NaN pattern is S.1111.111;
+* largest finite magnitude 448 (code 0x7E), smallest normal 2^-6,
+  subnormals k * 2^-9 for k = 1..7.
+
+``round`` is round-to-nearest, ties to the code whose mantissa LSB is even;
+``clamp`` saturates at +-448.  The encoder works on the IEEE-754 binary32 bit
+pattern with integer arithmetic only; it does not use any float8 data type.
+"""
+
+from __future__ import annotations
+
+import numpy as np
+
+E4M3_MAX = 448.0
+_BIAS = 7
+
+
+def _build_decode_table() -> np.ndarray:
+    table = np.zeros(256, dtype=np.float64)
+    for code in range(256):
+        sign = -1.0 if code & 0x80 else 1.0
+        e = (code >> 3) & 0xF
+        m = code & 0x7
+        if e == 0xF and m == 0x7:
+            val = float("nan")
+        elif e == 0:
+            val = sign * m * 2.0 ** (1 - _BIAS - 3)          # subnormal: m * 2^-9
+        else:
+            val = sign * (1.0 + m / 8.0) * 2.0 ** (e - _BIAS)
+        table[code] = val
+    return table
+
+
+DECODE_TABLE = _build_decode_table()
+
+
+def decode(codes) -> np.ndarray:
+    """E4M3 code (uint8) -> value, exactly, as float64."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    return DECODE_TABLE[codes]
+
+
+def encode(x) -> np.ndarray:
+    """binary32 value -> E4M3 code with round-to-nearest-even and saturation.
+
+    ``x`` is converted to float32 first (inputs are expected to be float32
+    already).  Non-finite inputs are an error.  The sign bit is always copied,
+    so -0.0 and negative values that round to zero give 0x80.
+    """
+    xf = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
+    if not np.all(np.isfinite(xf)):
+        raise ValueError("e4m3.encode: non-finite input")
+    bits = xf.view(np.uint32).astype(np.int64)
+    sign = (bits >> 31) & 1
+    efield = (bits >> 23) & 0xFF
+    m23 = bits & 0x7FFFFF
+    E = efield - 127                                   # unbiased binary32 exponent
+
+    # --- normal E4M3 range: |x| >= 2^-6 -----------------------------------
+    keep = m23 >> 20
+    rem = m23 & 0xFFFFF
+    half = 1 << 19
+    up = (rem > half) | ((rem == half) & ((keep & 1) == 1))
+    code_norm = (((E + _BIAS) << 3) | keep) + up.astype(np.int64)   # carry may bump the exponent
+    code_norm = np.minimum(code_norm, 0x7E)
+
+    # --- subnormal E4M3 range: |x| < 2^-6, grid step 2^-9 -----------------
+    # |x| = M * 2^(E-23) with M = 2^23 + m23;  k = round(|x| / 2^-9) = round(M / 2^shift)
+    M = m23 | (1 << 23)
+    shift = np.clip(14 - E, 0, 40)
+    keep_s = M >> shift
+    rem_s = M & ((np.int64(1) << shift) - 1)
+    half_s = np.int64(1) << np.maximum(shift - 1, 0)
+    up_s = (rem_s > half_s) | ((rem_s == half_s) & ((keep_s & 1) == 1))
+    code_sub = keep_s + up_s.astype(np.int64)          # k = 8 is the smallest normal, code 0x08
+    code_sub = np.where(efield == 0, 0, code_sub)      # binary32 zero / subnormal -> 0
+
+    mag = np.where(E >= -6, code_norm, code_sub)
+    mag = np.where(E > 8, 0x7E, mag)                   # >= 512: saturate (also guards the shift above)
+    return ((sign << 7) | mag).astype(np.uint8)
+
+
+def quantize_blocks(x, block: int):
+    """Per-block FP8 quantisation along the last axis.
+
+    x      [R, K] array holding bf16-representable values (any float dtype)
+    block  number of consecutive elements along K sharing one scale
+
+    For each block: amax = max|x|; s = fl32(amax / 448) (one binary32 division),
+    s = 1 when amax == 0; q = encode(fl32(fl32(x) / s)) (one binary32 division,
+    then round-to-nearest-even onto the E4M3 grid, saturating).
+
+    Returns (codes uint8 [R, K], scales float32 [R, K // block]).
+    """
+    x32 = np.asarray(x, dtype=np.float32)
+    R, K = x32.shape
+    if K % block:
+        raise ValueError("block must divide the last dimension")
+    xb = x32.reshape(R, K // block, block)
+    amax = np.max(np.abs(xb), axis=2).astype(np.float32)
+    scales = (amax / np.float32(E4M3_MAX)).astype(np.float32)
+    scales = np.where(amax == 0, np.float32(1.0), scales).astype(np.float32)
+    with np.errstate(over="ignore"):
+        quot = (xb / scales[:, :, None]).astype(np.float32)
+    # a quotient can only overflow binary32 when the scale is subnormal; it saturates anyway
+    quot = np.clip(quot, -3.0e38, 3.0e38).astype(np.float32)
+    codes = encode(quot).reshape(R, K)
+    return codes, scales
+
+
+def dequantize_blocks(codes, scales, block: int) -> np.ndarray:
+    """codes [R, K], scales [R, K // block] -> float64 [R, K] = decode(q) * s (exact product)."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    R, K = codes.shape
+    vals = decode(codes).reshape(R, K // block, block)
+    out = vals * np.asarray(scales, dtype=np.float64)[:, :, None]
+    return out.reshape(R, K)

@@ -1,0 +1,190 @@
+"""Pins for the oracle's E4M3 codec and block quantiser (CPU only).
+
+The pins are independent of the oracle's own arithmetic: the format's landmark values
+(tests/golden/e4m3_landmarks.txt), exhaustive round-trips, midpoint behaviour worked out from
+the grid itself, a third-party float8 implementation used as a black box, and error bounds.
+"""
+
+import os
+
+import numpy as np
+import pytest
+
+from oracle import e4m3
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _finite_codes():
+    return np.array([c for c in range(256) if (c & 0x7F) != 0x7F], dtype=np.uint8)
+
+
+def test_landmark_values():
+    for line in open(os.path.join(GOLDEN, "e4m3_landmarks.txt")):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        code, val = line.split()
+        code = int(code, 16)
+        got = e4m3.decode(np.array([code], dtype=np.uint8))[0]
+        assert got == float(val), (hex(code), got, val)
+        assert np.signbit(got) == bool(code & 0x80)
+        assert e4m3.encode(np.array([float(val)], dtype=np.float32))[0] == code
+
+
+def test_nan_codes_and_grid_shape():
+    assert np.isnan(e4m3.decode(np.array([0x7F, 0xFF], dtype=np.uint8))).all()
+    pos = e4m3.decode(np.arange(0, 0x7F, dtype=np.uint8))
+    assert np.all(np.diff(pos) > 0)                       # strictly increasing in the code
+    assert pos[-1] == 448.0 and pos[1] == 2.0 ** -9 and pos[8] == 2.0 ** -6
+    # mantissa spacing: within one binade 8 equal steps
+    for e in range(1, 15):
+        seg = pos[e * 8:(e + 1) * 8]
+        assert np.allclose(np.diff(seg), seg[0] / 8.0, rtol=0, atol=0)
+
+
+def test_round_trip_all_codes():
+    codes = _finite_codes()
+    vals = e4m3.decode(codes).astype(np.float32)
+    assert np.array_equal(e4m3.encode(vals), codes)
+
+
+def test_midpoints_tie_to_even_and_neighbours():
+    pos = e4m3.decode(np.arange(0, 0x7F, dtype=np.uint8))          # 0 .. 448
+    for c in range(0, 0x7E):
+        lo, hi = pos[c], pos[c + 1]
+        mid = np.float32((lo + hi) / 2.0)                          # exactly representable in binary32
+        assert float(mid) == (lo + hi) / 2.0
+        even = c if (c & 1) == 0 else c + 1
+        assert e4m3.encode(np.array([mid]))[0] == even, (c, mid)
+        below = np.nextafter(mid, np.float32(0))
+        above = np.nextafter(mid, np.float32(1e9))
+        assert e4m3.encode(np.array([below]))[0] == c
+        assert e4m3.encode(np.array([above]))[0] == c + 1
+        # negative side mirrors
+        assert e4m3.encode(np.array([-mid]))[0] == (0x80 | even)
+
+
+def test_saturation():
+    xs = np.array([448.0, 449.0, 463.9, 464.0, 465.0, 480.0, 512.0, 1e4, 3e38], dtype=np.float32)
+    assert np.all(e4m3.encode(xs) == 0x7E)
+    assert np.all(e4m3.encode(-xs) == 0xFE)
+
+
+def test_subnormal_range():
+    tiny = 2.0 ** -9
+    assert e4m3.encode(np.array([tiny / 2], dtype=np.float32))[0] == 0x00          # tie -> even (zero)
+    assert e4m3.encode(np.array([np.nextafter(np.float32(tiny / 2), np.float32(1))]))[0] == 0x01
+    assert e4m3.encode(np.array([tiny * 0.49], dtype=np.float32))[0] == 0x00
+    assert e4m3.encode(np.array([tiny * 7.5], dtype=np.float32))[0] == 0x08        # tie -> even (8 = min normal)
+    assert e4m3.encode(np.array([tiny * 6.5], dtype=np.float32))[0] == 0x06
+    assert e4m3.encode(np.array([-1e-30], dtype=np.float32))[0] == 0x80            # sign kept
+    assert e4m3.encode(np.array([-0.0], dtype=np.float32))[0] == 0x80
+    assert e4m3.encode(np.array([1e-45], dtype=np.float32))[0] == 0x00             # binary32 subnormal
+
+
+def test_non_finite_rejected():
+    with pytest.raises(ValueError):
+        e4m3.encode(np.array([np.inf], dtype=np.float32))
+    with pytest.raises(ValueError):
+        e4m3.encode(np.array([np.nan], dtype=np.float32))
+
+
+def test_nearest_by_brute_force():
+    """Every encoded value is a nearest grid point (brute-force search over the 127 magnitudes)."""
+    rng = np.random.default_rng(7)
+    x = np.concatenate([rng.normal(0, 1, 20000), rng.uniform(-448, 448, 20000),
+                        rng.normal(0, 0.01, 20000)]).astype(np.float32)
+    grid = e4m3.decode(np.arange(0, 0x7F, dtype=np.uint8))
+    got = np.abs(e4m3.decode(e4m3.encode(x)))
+    dist = np.abs(np.abs(x.astype(np.float64))[:, None] - grid[None, :]).min(axis=1)
+    assert np.array_equal(np.abs(np.abs(x.astype(np.float64)) - got), dist)
+
+
+def test_against_ml_dtypes_black_box():
+    ml_dtypes = pytest.importorskip("ml_dtypes")
+    rng = np.random.default_rng(11)
+    x = np.concatenate([rng.uniform(-448, 448, 500000), rng.normal(0, 1, 300000),
+                        rng.normal(0, 2.0 ** -7, 200000)]).astype(np.float32)
+    ref = x.astype(ml_dtypes.float8_e4m3fn).view(np.uint8)
+    assert np.array_equal(e4m3.encode(x), ref)
+    # all bf16 values with |x| <= 448
+    bits = np.arange(0, 1 << 16, dtype=np.uint32) << 16
+    v = bits.view(np.float32)
+    v = v[np.isfinite(v) & (np.abs(v) <= 448)]
+    assert np.array_equal(e4m3.encode(v), v.astype(ml_dtypes.float8_e4m3fn).view(np.uint8))
+
+
+# ------------------------------------------------------------------ block quantisation
+def _bf16_round(x):
+    import torch
+    return torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).float().numpy()
+
+
+def test_block_scale_rule_and_zero_block():
+    x = np.zeros((2, 256), dtype=np.float32)
+    x[0, :128] = _bf16_round(np.linspace(-3, 3, 128))
+    x[1, 128:] = 0.0
+    x[1, :128] = _bf16_round(np.random.default_rng(0).normal(size=128))
+    codes, scales = e4m3.quantize_blocks(x, 128)
+    assert scales.dtype == np.float32 and codes.dtype == np.uint8
+    assert scales[0, 1] == 1.0 and scales[1, 1] == 1.0                # zero block -> scale 1
+    assert np.all(codes[0, 128:] == 0)
+    for r in range(2):
+        amax = np.abs(x[r, :128]).max()
+        assert scales[r, 0] == np.float32(amax) / np.float32(448.0)
+        # the largest element of a non-zero block lands on +-448
+        j = np.abs(x[r, :128]).argmax()
+        assert codes[r, j] & 0x7F == 0x7E
+
+
+def test_power_of_two_scale_block_is_exact():
+    """amax = 3.5 = 448 * 2^-7: the scale is exactly 2^-7, so grid values round-trip exactly and
+    halfway values go to the even code."""
+    s = 2.0 ** -7
+    grid = e4m3.decode(np.arange(0, 0x7F, dtype=np.uint8))
+    vals = grid[8:0x7F:3] * s                                          # all bf16-exact (4 significant bits)
+    x = np.zeros((1, 128), dtype=np.float32)
+    x[0, :len(vals)] = vals
+    x[0, 127] = 3.5
+    # halfway between codes 0x38 (1.0) and 0x39 (1.125), times s: 1.0625 * 2^-7 -> even code 0x38
+    x[0, 126] = 1.0625 * s
+    # halfway between 0x39 (1.125) and 0x3A (1.25): 1.1875 -> even code 0x3A
+    x[0, 125] = 1.1875 * s
+    codes, scales = e4m3.quantize_blocks(x, 128)
+    assert scales[0, 0] == np.float32(s)
+    assert np.array_equal(codes[0, :len(vals)], np.arange(8, 0x7F, 3, dtype=np.uint8))
+    assert codes[0, 127] == 0x7E and codes[0, 126] == 0x38 and codes[0, 125] == 0x3A
+    deq = e4m3.dequantize_blocks(codes, scales, 128)
+    assert np.array_equal(deq[0, :len(vals)], vals)
+
+
+@pytest.mark.parametrize("block", [32, 128])
+def test_block_error_bound(block):
+    rng = np.random.default_rng(3)
+    x = _bf16_round(rng.normal(0, 1, size=(64, 512)) * rng.lognormal(0, 2, size=(64, 1)))
+    codes, scales = e4m3.quantize_blocks(x, block)
+    deq = e4m3.dequantize_blocks(codes, scales, block)
+    s = np.repeat(scales.astype(np.float64), block, axis=1)
+    q = np.abs(x.astype(np.float64)) / s
+    # half the local grid spacing: normal codes 2^(floor(log2 q) - 4); subnormal region 2^-10
+    half_step = np.where(q >= 2.0 ** -6, 2.0 ** (np.floor(np.log2(np.maximum(q, 1e-300))) - 4), 2.0 ** -10)
+    err = np.abs(deq - x.astype(np.float64))
+    assert np.all(err <= s * half_step * (1 + 1e-6) + s * q * 2.0 ** -23)
+    # relative error at most 2^-4 for everything that maps to a normal code
+    norm = q >= 2.0 ** -6
+    assert np.all(err[norm] <= 2.0 ** -4 * np.abs(x.astype(np.float64))[norm] * (1 + 1e-6))
+    assert np.all(np.sign(deq) * np.sign(x) >= 0)
+
+
+def test_block_axis_is_last_axis_only():
+    """Changing an element changes only its own block's scale."""
+    rng = np.random.default_rng(5)
+    x = _bf16_round(rng.normal(size=(4, 256)))
+    c0, s0 = e4m3.quantize_blocks(x, 128)
+    y = x.copy()
+    y[2, 130] = 64.0
+    c1, s1 = e4m3.quantize_blocks(y, 128)
+    diff = (s0 != s1)
+    assert diff.sum() == 1 and diff[2, 1]
+    assert np.array_equal(c0[:, :128], c1[:, :128]) and np.array_equal(c0[[0, 1, 3]], c1[[0, 1, 3]])
