@@ -1,0 +1,196 @@
+/*
+ * ais.h - C ABI of the B200 (sm_100a) library for the LM-head step of an AIS-GRPO update.
+ *
+ * The path: hidden states H [T,d] meet the LM head W twice - once with bf16 operands (the trainer's
+ * policy pi_train) and once with block-scaled FP8-E4M3 operands (the rollout policy pi_rollout) - each
+ * pass fused with a streaming log-sum-exp over the vocabulary and a pick of the sampled token's logit,
+ * so the [T,V] logits never reach global memory.  The two log-probability vectors feed the three AIS
+ * diagnostics and the per-batch mixing coefficient alpha (Section 3.1, Algorithm 1); the last call gives
+ * the AIS-GRPO surrogate loss (Section 3.2, Eq. ais-grpo, without the KL term) and its gradient with
+ * respect to H.
+ *
+ * Conventions
+ * -----------
+ *  - Every data pointer is a DEVICE pointer owned by the caller unless it says "host".  The library
+ *    never allocates or frees device memory; scratch comes from the caller's `workspace`
+ *    (256-byte aligned, at least ais_workspace_bytes() bytes).
+ *  - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it; they never
+ *    synchronise the device.  Calls on one stream are ordered; calls that share a workspace must not
+ *    overlap on the GPU.
+ *  - Return value: AIS_OK or a negative AIS_ERR_* code.  On a host-detected error nothing has been
+ *    enqueued.  Conditions only the device can see (token id outside [0,V), a bounded wait that ran
+ *    out, no valid token) are OR-ed into the caller's `dev_status` word / ais_diag.status_flags and the
+ *    affected outputs take their documented neutral values; the kernels never trap.
+ *  - Layouts: H is row-major [T, ldh] bf16 (ldh >= d).  W is row-major [V, ldw] bf16, one row per
+ *    vocabulary entry (the layout of a torch lm_head.weight), so logits are z = H W^T.
+ *    FP8 codes keep the layout of their source matrix ([rows, cols] uint8).  Scales are "block-major":
+ *    scales[kb * ld_scales + row] is the scale of block kb (elements kb*B .. kb*B+B-1 along d) of `row`.
+ *  - Rows with mask[t] == 0 yield lp = 0, lse = 0, rho = 1, w_tilde = 1 and a zero row of dH.
+ *  - Alignment: H, W, codes, scales and dH 16 bytes, the workspace 256 bytes; ldh and ldw multiples
+ *    of 16; d a multiple of 128 (one shared-memory stage is 128 bytes of FP8 along d) and of
+ *    fp8_block; V a multiple of 8; ld of scale arrays a multiple of 4.
+ */
+#ifndef AIS_H_
+#define AIS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AIS_VERSION 100
+
+/* status codes */
+#define AIS_OK                 0
+#define AIS_ERR_NULL          -1   /* a required pointer is NULL                            */
+#define AIS_ERR_SHAPE         -2   /* a size is out of range or inconsistent (S != P*G ...) */
+#define AIS_ERR_ALIGN         -3   /* pointer or leading dimension not aligned as required  */
+#define AIS_ERR_WORKSPACE     -4   /* workspace missing, misaligned or too small            */
+#define AIS_ERR_DEVICE        -5   /* current device is not sm_100, or a CUDA call failed   */
+#define AIS_ERR_PARAM         -6   /* a hyper-parameter is out of range                     */
+#define AIS_ERR_LIMIT         -7   /* size beyond a fixed limit of an entry point           */
+
+/* bits of a device status word / ais_diag.status_flags */
+#define AIS_FLAG_EMPTY        1u   /* no valid token in the batch: alpha = 0, loss = 0      */
+#define AIS_FLAG_TOKEN_RANGE  2u   /* a valid row has a token id outside [0, V): lp = 0     */
+#define AIS_FLAG_NONFINITE    4u   /* a log-prob of a valid row is not finite               */
+#define AIS_FLAG_TIMEOUT      8u   /* a bounded device-side wait ran out; outputs undefined */
+
+typedef struct ais_shape {
+    int64_t T;            /* token rows                                                      */
+    int32_t d;            /* hidden size                                                     */
+    int32_t V;            /* vocabulary size                                                 */
+    int32_t P;            /* prompts in the batch                                            */
+    int32_t G;            /* responses per prompt; sequence s belongs to prompt s / G        */
+    int32_t fp8_block;    /* elements along d sharing one FP8 scale: 32, 64 or 128           */
+    int32_t reserved;
+    int64_t ldh;          /* row stride of H (and of its codes) in elements                  */
+    int64_t ldw;          /* row stride of W (and of its codes) in elements                  */
+} ais_shape;
+
+/* Hyper-parameters (Algorithm 1 'Require' line; Appendix 'AIS hyperparameters'; PPO clipping of the
+ * hyper-parameter table).  The paper prints no value for beta_var; 1 is this library's default. */
+typedef struct ais_params {
+    float C;              /* truncation of the importance ratio, >= 1          (5)           */
+    float delta;          /* saturation threshold of the divergence gate, > 0  (0.02)        */
+    float gamma;          /* tolerance of the variance-amplification ratio, >0 (1.2)         */
+    float eps;            /* stabiliser in that ratio                          (1e-6)        */
+    float beta_var;       /* weight of the variance penalty                    (1.0)         */
+    float clip_eps;       /* PPO clip range of rho_on                          (0.2)         */
+    float alpha_override; /* NaN: adaptive alpha.  Otherwise alpha is forced to this value in
+                             [0,1] (0 = plain GRPO, 1 = truncated importance sampling); the
+                             diagnostics are still reported.                                 */
+    int32_t adv_std_norm; /* 0: A = r - mean(group) (the paper's form).  1: also divide by
+                             (population std of the group + eps).                            */
+    int32_t vocab_chunk;  /* 0: library default.  Otherwise the vocabulary is streamed in
+                             independent chunks of about this many columns whose partial
+                             (max, sum-exp, target logit) triples are merged afterwards.     */
+    int32_t reserved;
+} ais_params;
+
+/* Everything the reductions produce; lives in DEVICE memory, the caller copies it back. */
+typedef struct ais_diag {
+    double n_valid;       /* N = number of rows with mask 1                                  */
+    double mean_w;        /* mean of w_bar = min(rho, C)                                     */
+    double cv2;           /* squared coefficient of variation of w_bar (population moments)  */
+    double ess;           /* (sum w_bar)^2 / sum w_bar^2                                     */
+    double ess_ratio;     /* ess / N                                                         */
+    double alpha_ess;     /* (1 + cv2)^(-1/2)                         Eq. alpha-ess          */
+    double d_bar;         /* mean |lp_train - lp_roll|                Eq. discrepancy        */
+    double alpha_mis;     /* min(1, d_bar / delta)                    Eq. alpha-mis          */
+    double std_A;         /* population std of the token-level advantage                     */
+    double std_Aw;        /* population std of A * w_bar                                     */
+    double delta_sigma;   /* std_Aw / (std_A + eps)                                          */
+    double alpha_var;     /* max(0, (delta_sigma - gamma) / gamma)    Eq. alpha-var          */
+    double alpha_adaptive;/* clip(alpha_ess - beta_var alpha_var, 0, 1) * alpha_mis          */
+    double alpha;         /* the coefficient in force (alpha_adaptive or the override)       */
+    double loss;          /* written by ais_loss_bwd                                         */
+    double kl_k1;         /* monitor: mean(lp_roll - lp_train)                               */
+    double mean_abs_dp;   /* monitor: mean |exp(lp_train) - exp(lp_roll)|                    */
+    uint32_t status_flags;
+    uint32_t reserved;
+} ais_diag;
+
+int ais_version(void);
+const char* ais_strerror(int status);
+
+/* Fills *p with the defaults listed above (alpha_override = NaN). `p` is a host pointer. */
+void ais_default_params(ais_params* p);
+
+/* Recommended workspace size in bytes for all entry points on this shape (host pointers in).
+ * Any 256-byte aligned workspace of at least ais_workspace_min_bytes() is accepted; a larger one
+ * lets ais_loss_bwd process more rows per pass.  Returns 0 for an invalid shape. */
+size_t ais_workspace_bytes(const ais_shape* shape, const ais_params* params);
+size_t ais_workspace_min_bytes(const ais_shape* shape, const ais_params* params);
+
+/*
+ * FP8-E4M3 block quantisation (Section 2.1, quantisation equation, with the E4M3 grid in place of the
+ * integer grid): for every run of `block` consecutive elements of a row,
+ *     s = fl32(max|x| / 448)   (s = 1 for an all-zero block)
+ *     q = E4M3_rne_saturating( fl32(fl32(x) / s) )
+ * x       [rows, ld]  bf16, row-major
+ * codes   [rows, ldq] uint8                       (written)
+ * scales  [cols/block, lds] float, block-major    (written; lds >= rows)
+ * cols must be a multiple of `block`; block is 32, 64 or 128.  Used for H (rows = T) and W (rows = V).
+ */
+int ais_quantize_fp8(const void* x, int64_t rows, int64_t cols, int64_t ld, int block,
+                     uint8_t* codes, int64_t ldq, float* scales, int64_t lds, void* stream);
+
+/*
+ * Trainer and rollout log-probabilities (Algorithm 1: "full-precision log-probs" and the sampler's
+ * log-probs entering rho_rt; Eq. logit-mismatch).  For every row t with mask[t] = 1:
+ *     lse_train[t] = log sum_v exp(z[t,v]),  z = H W^T  (bf16 operands, fp32 accumulation)
+ *     lp_train[t]  = z[t, tokens[t]] - lse_train[t]
+ *     lp_roll[t], lse_roll[t]: the same with z^[t,v] = sum_kb sH[kb,t] sW[kb,v] sum_{k in kb} qH[t,k] qW[v,k]
+ * The train pass is skipped when lp_train is NULL; the rollout pass when lp_roll is NULL.
+ * lse_train / lse_roll may be NULL when not wanted (lse_train is needed later by ais_loss_bwd).
+ * sH is [d/B, ldsH] and sW is [d/B, ldsW] (block-major, as ais_quantize_fp8 writes them).
+ * tokens [T] int32, mask [T] uint8, dev_status: one uint32 on the device (OR-ed into; may be NULL).
+ */
+int ais_logprob_fwd(const ais_shape* shape, const ais_params* params,
+                    const void* H, const void* W,
+                    const uint8_t* qH, const float* sH, int64_t ldsH,
+                    const uint8_t* qW, const float* sW, int64_t ldsW,
+                    const int32_t* tokens, const uint8_t* mask,
+                    float* lp_train, float* lse_train, float* lp_roll, float* lse_roll,
+                    uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Ratios, advantages, diagnostics, alpha and the rectification weight (Algorithm 1, "Adaptive
+ * Coefficient Estimation" and "Advantage Rectification"; Eqs. grpo_adv, alpha-ess, discrepancy,
+ * alpha-mis, alpha-var, alpha-final, adjusted-advantage).
+ * seq_offsets [S+1] int32 row offsets of the S = P*G sequences (seq_offsets[S] == T), rewards [S].
+ * Outputs: adv [S] (A_s), n_valid_seq [S] int32 (valid rows per sequence; may be NULL),
+ * rho [T] = exp(lp_train - lp_roll) (may be NULL), w_tilde [T] = 1 + alpha (min(rho, C) - 1),
+ * diag (one ais_diag on the device).  All moments are population moments over the valid rows.
+ */
+int ais_diagnostics(const ais_shape* shape, const ais_params* params,
+                    const float* lp_train, const float* lp_roll, const uint8_t* mask,
+                    const int32_t* seq_offsets, const float* rewards,
+                    float* adv, int32_t* n_valid_seq, float* rho, float* w_tilde, ais_diag* diag,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * AIS-GRPO surrogate loss and its gradient with respect to H (Eq. ais-grpo without the KL term;
+ * the objective is maximised, so loss = -J).  With rho_on = exp(lp_train - lp_old)
+ * (lp_old == NULL means rho_on = 1) and n_s the valid rows of sequence s:
+ *     loss  = - sum_s 1/(P G n_s) sum_{t in s, mask} w_tilde[t] min(rho_on A_s, clip(rho_on, 1 +- clip_eps) A_s)
+ *     c_t   = mask[t] w_tilde[t] A_s rho_on [unclipped branch active] / (P G n_s)
+ *     dH[t,:] = c_t (softmax(z[t,:]) - onehot(tokens[t])) W
+ * The softmax is recomputed from H, W and lse_train; w_tilde, A and lp_old are constants.
+ * dH [T, ldh] bf16 (written, zero rows where mask = 0), loss: one float on the device (may be NULL),
+ * diag: if not NULL its `loss` field is written too.
+ */
+int ais_loss_bwd(const ais_shape* shape, const ais_params* params,
+                 const void* H, const void* W, const int32_t* tokens, const uint8_t* mask,
+                 const int32_t* seq_offsets, const float* lse_train, const float* lp_train,
+                 const float* lp_old, const float* adv, const float* w_tilde,
+                 void* dH, float* loss, ais_diag* diag,
+                 uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AIS_H_ */

@@ -1,0 +1,233 @@
+"""ctypes binding of the C ABI declared in include/ais.h (argument marshalling only)."""
+
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libais_b200.so")
+_lib = None
+
+FLAG_EMPTY, FLAG_TOKEN_RANGE, FLAG_NONFINITE, FLAG_TIMEOUT = 1, 2, 4, 8
+
+
+class AisError(RuntimeError):
+    pass
+
+
+class Shape(C.Structure):
+    _fields_ = [("T", C.c_int64), ("d", C.c_int32), ("V", C.c_int32), ("P", C.c_int32), ("G", C.c_int32),
+                ("fp8_block", C.c_int32), ("reserved", C.c_int32), ("ldh", C.c_int64), ("ldw", C.c_int64)]
+
+
+class Params(C.Structure):
+    _fields_ = [("C", C.c_float), ("delta", C.c_float), ("gamma", C.c_float), ("eps", C.c_float),
+                ("beta_var", C.c_float), ("clip_eps", C.c_float), ("alpha_override", C.c_float),
+                ("adv_std_norm", C.c_int32), ("vocab_chunk", C.c_int32), ("reserved", C.c_int32)]
+
+
+class Diag(C.Structure):
+    _fields_ = [(n, C.c_double) for n in
+                ("n_valid", "mean_w", "cv2", "ess", "ess_ratio", "alpha_ess", "d_bar", "alpha_mis", "std_A", "std_Aw",
+                 "delta_sigma", "alpha_var", "alpha_adaptive", "alpha", "loss", "kl_k1", "mean_abs_dp")] + \
+               [("status_flags", C.c_uint32), ("reserved", C.c_uint32)]
+
+    def as_dict(self) -> dict:
+        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> C.CDLL:
+    """Loads the CUDA library; raises if it has not been built (python -m paper_2605_13907_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise AisError(f"{_LIB_PATH} is missing: build it with `python paper_2605_13907_b200/build.py`; "
+                           "there is no CPU fallback")
+        L = C.CDLL(_LIB_PATH)
+        vp, i64, sz = C.c_void_p, C.c_int64, C.c_size_t
+        L.ais_version.restype = C.c_int
+        L.ais_strerror.restype = C.c_char_p
+        L.ais_strerror.argtypes = [C.c_int]
+        L.ais_default_params.restype = None
+        L.ais_default_params.argtypes = [C.POINTER(Params)]
+        for f in (L.ais_workspace_bytes, L.ais_workspace_min_bytes):
+            f.restype = sz
+            f.argtypes = [C.POINTER(Shape), C.POINTER(Params)]
+        L.ais_quantize_fp8.restype = C.c_int
+        L.ais_quantize_fp8.argtypes = [vp, i64, i64, i64, C.c_int, vp, i64, vp, i64, vp]
+        L.ais_logprob_fwd.restype = C.c_int
+        L.ais_logprob_fwd.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, i64, vp, vp, i64, vp, vp,
+                                      vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ais_diagnostics.restype = C.c_int
+        L.ais_diagnostics.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ais_loss_bwd.restype = C.c_int
+        L.ais_loss_bwd.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 14 + [vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def _check(status: int, what: str) -> None:
+    if status != 0:
+        raise AisError(f"{what}: {lib().ais_strerror(status).decode()} ({status})")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(t: torch.Tensor):
+    return C.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+def default_params(**overrides) -> Params:
+    p = Params()
+    lib().ais_default_params(C.byref(p))
+    for k, v in overrides.items():
+        if k == "alpha_override" and v is None:
+            v = math.nan
+        setattr(p, k, v)
+    return p
+
+
+def make_shape(T: int, d: int, V: int, P: int, G: int, fp8_block: int, ldh: int | None = None, ldw: int | None = None) -> Shape:
+    return Shape(T=T, d=d, V=V, P=P, G=G, fp8_block=fp8_block, reserved=0, ldh=ldh or d, ldw=ldw or d)
+
+
+def workspace_bytes(shape: Shape, params: Params) -> int:
+    return int(lib().ais_workspace_bytes(C.byref(shape), C.byref(params)))
+
+
+def workspace_min_bytes(shape: Shape, params: Params) -> int:
+    return int(lib().ais_workspace_min_bytes(C.byref(shape), C.byref(params)))
+
+
+def _require_cuda(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise AisError("all tensors must live on a CUDA device; this library has no CPU path")
+
+
+def quantize_fp8(x: torch.Tensor, block: int, codes: torch.Tensor | None = None, scales: torch.Tensor | None = None):
+    """x [rows, cols] bf16 -> (codes [rows, cols] uint8, scales [cols/block, lds] float32, block-major)."""
+    _require_cuda(x, codes, scales)
+    rows, cols = x.shape
+    if codes is None:
+        codes = torch.empty(rows, cols, dtype=torch.uint8, device=x.device)
+    if scales is None:
+        lds = (rows + 3) // 4 * 4
+        scales = torch.empty(cols // block, max(lds, 4), dtype=torch.float32, device=x.device)
+    _check(lib().ais_quantize_fp8(_ptr(x), rows, cols, x.stride(0), block, _ptr(codes), codes.stride(0), _ptr(scales),
+                                  scales.stride(0), _stream(x)), "ais_quantize_fp8")
+    return codes, scales
+
+
+def logprob_fwd(shape: Shape, params: Params, H, W, qH, sH, qW, sW, tokens, mask, lp_train, lse_train, lp_roll, lse_roll,
+                dev_status, workspace):
+    _require_cuda(H, W, qH, sH, qW, sW, tokens, mask, lp_train, lse_train, lp_roll, lse_roll, dev_status, workspace)
+    _check(lib().ais_logprob_fwd(C.byref(shape), C.byref(params), _ptr(H), _ptr(W), _ptr(qH), _ptr(sH),
+                                 sH.stride(0) if sH is not None else 0, _ptr(qW), _ptr(sW),
+                                 sW.stride(0) if sW is not None else 0, _ptr(tokens), _ptr(mask), _ptr(lp_train),
+                                 _ptr(lse_train), _ptr(lp_roll), _ptr(lse_roll), _ptr(dev_status), _ptr(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream(workspace)), "ais_logprob_fwd")
+
+
+def diagnostics(shape: Shape, params: Params, lp_train, lp_roll, mask, seq_offsets, rewards, adv, n_valid_seq, rho, w_tilde,
+                diag, workspace):
+    _require_cuda(lp_train, lp_roll, mask, seq_offsets, rewards, adv, n_valid_seq, rho, w_tilde, diag, workspace)
+    _check(lib().ais_diagnostics(C.byref(shape), C.byref(params), _ptr(lp_train), _ptr(lp_roll), _ptr(mask), _ptr(seq_offsets),
+                                 _ptr(rewards), _ptr(adv), _ptr(n_valid_seq), _ptr(rho), _ptr(w_tilde), _ptr(diag),
+                                 _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(workspace)),
+           "ais_diagnostics")
+
+
+def loss_bwd(shape: Shape, params: Params, H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, adv, w_tilde, dH, loss,
+             diag, dev_status, workspace):
+    _require_cuda(H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, adv, w_tilde, dH, loss, diag, dev_status, workspace)
+    _check(lib().ais_loss_bwd(C.byref(shape), C.byref(params), _ptr(H), _ptr(W), _ptr(tokens), _ptr(mask), _ptr(seq_offsets),
+                              _ptr(lse_train), _ptr(lp_train), _ptr(lp_old), _ptr(adv), _ptr(w_tilde), _ptr(dH), _ptr(loss),
+                              _ptr(diag), _ptr(dev_status), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                              _stream(workspace)), "ais_loss_bwd")
+
+
+def read_diag(diag_buf: torch.Tensor) -> dict:
+    """Copies the device-side ais_diag back (synchronises the current stream)."""
+    host = diag_buf.cpu().numpy().tobytes()
+    return Diag.from_buffer_copy(host[:C.sizeof(Diag)]).as_dict()
+
+
+class AisStep:
+    """Buffers and call order of one pass of the whole path for a fixed shape.
+
+    step() enqueues: quantise H (and W unless its codes are cached) -> trainer and rollout log-probs ->
+    ratios / diagnostics / alpha / w_tilde -> loss and dH.  Nothing synchronises; results stay on the device.
+    """
+
+    def __init__(self, T: int, d: int, V: int, P: int, G: int, fp8_block: int, device="cuda", params: Params | None = None,
+                 workspace_bytes_cap: int | None = None, want_grad: bool = True):
+        self.device = torch.device(device)
+        self.shape = make_shape(T, d, V, P, G, fp8_block)
+        self.params = params or default_params()
+        S = P * G
+        dev = self.device
+        nkb = d // fp8_block
+        ws = workspace_bytes(self.shape, self.params)
+        if workspace_bytes_cap is not None:
+            ws = max(workspace_min_bytes(self.shape, self.params), min(ws, workspace_bytes_cap))
+        if ws == 0:
+            raise AisError("invalid shape or parameters")
+        self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
+        self.qH = torch.empty(max(T, 1), d, dtype=torch.uint8, device=dev)
+        self.sH = torch.empty(nkb, max((T + 3) // 4 * 4, 4), dtype=torch.float32, device=dev)
+        self.qW = torch.empty(V, d, dtype=torch.uint8, device=dev)
+        self.sW = torch.empty(nkb, (V + 3) // 4 * 4, dtype=torch.float32, device=dev)
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.lp_train = torch.empty(max(T, 1), **f32)
+        self.lse_train = torch.empty(max(T, 1), **f32)
+        self.lp_roll = torch.empty(max(T, 1), **f32)
+        self.lse_roll = torch.empty(max(T, 1), **f32)
+        self.rho = torch.empty(max(T, 1), **f32)
+        self.w_tilde = torch.empty(max(T, 1), **f32)
+        self.adv = torch.empty(S, **f32)
+        self.n_valid_seq = torch.empty(S, dtype=torch.int32, device=dev)
+        self.loss = torch.zeros(1, **f32)
+        self.diag = torch.zeros((C.sizeof(Diag) + 7) // 8, dtype=torch.float64, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.dH = torch.empty(max(T, 1), d, dtype=torch.bfloat16, device=dev) if want_grad else None
+        self.w_quantized = False
+
+    def quantize_weights(self, W: torch.Tensor) -> None:
+        quantize_fp8(W, self.shape.fp8_block, self.qW, self.sW)
+        self.w_quantized = True
+
+    def forward(self, H, W, tokens, mask, requantize_w: bool = True) -> None:
+        if self.shape.T > 0:
+            quantize_fp8(H, self.shape.fp8_block, self.qH, self.sH)
+        if requantize_w or not self.w_quantized:
+            self.quantize_weights(W)
+        logprob_fwd(self.shape, self.params, H, W, self.qH, self.sH, self.qW, self.sW, tokens, mask, self.lp_train,
+                    self.lse_train, self.lp_roll, self.lse_roll, self.status, self.workspace)
+
+    def diagnose(self, mask, seq_offsets, rewards) -> None:
+        diagnostics(self.shape, self.params, self.lp_train, self.lp_roll, mask, seq_offsets, rewards, self.adv,
+                    self.n_valid_seq, self.rho, self.w_tilde, self.diag, self.workspace)
+
+    def backward(self, H, W, tokens, mask, seq_offsets, lp_old=None) -> None:
+        loss_bwd(self.shape, self.params, H, W, tokens, mask, seq_offsets, self.lse_train, self.lp_train, lp_old, self.adv,
+                 self.w_tilde, self.dH, self.loss, self.diag, self.status, self.workspace)
+
+    def step(self, H, W, tokens, mask, seq_offsets, rewards, lp_old=None, requantize_w: bool = True) -> None:
+        self.forward(H, W, tokens, mask, requantize_w)
+        self.diagnose(mask, seq_offsets, rewards)
+        if self.dH is not None:
+            self.backward(H, W, tokens, mask, seq_offsets, lp_old)
+
+    def read_diag(self) -> dict:
+        return read_diag(self.diag)

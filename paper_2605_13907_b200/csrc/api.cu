@@ -1,0 +1,387 @@
+// C ABI of the library: argument validation, workspace carving, tensor-map construction and the order
+// in which the kernels of each entry point are enqueued.  Declarations and contracts live in include/ais.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "../../include/ais.h"
+#include "lmhead.cuh"
+#include "stream_kernels.cuh"
+
+namespace {
+
+using namespace ais;
+
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+    bool ready = false;
+    int status = AIS_OK;
+    int num_sms = 0;
+};
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_mutex;
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+
+// Per-device set-up, done once: checks the architecture, raises the kernels' dynamic shared-memory limit
+// and resolves the driver's tensor-map encoder.
+int device_setup(int* num_sms) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AIS_ERR_DEVICE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceInfo& info = g_dev[dev];
+    if (!info.ready) {
+        info.ready = true;
+        info.status = AIS_ERR_DEVICE;
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return info.status;
+        if (prop.major != 10) return info.status;
+        if (!g_encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+                qres != cudaDriverEntryPointSuccess || !fn)
+                return info.status;
+            g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+        }
+        if (lmhead_prepare() != cudaSuccess) return info.status;
+        info.num_sms = prop.multiProcessorCount;
+        info.status = AIS_OK;
+    }
+    if (num_sms) *num_sms = info.num_sms;
+    return info.status;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// 2-D row-major tensor map: dim0 is the contiguous axis.
+bool make_tmap(CUtensorMap* map, CUtensorMapDataType dtype, int elem_bytes, const void* base, uint64_t dim0, uint64_t dim1,
+               uint64_t stride1_bytes, uint32_t box0, uint32_t box1, CUtensorMapSwizzle swz) {
+    cuuint64_t dims[2] = {dim0, dim1};
+    cuuint64_t strides[1] = {stride1_bytes};
+    cuuint32_t box[2] = {box0, box1};
+    cuuint32_t estr[2] = {1, 1};
+    (void)elem_bytes;
+    CUresult r = g_encode(map, dtype, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int check_shape(const ais_shape* s) {
+    if (!s) return AIS_ERR_NULL;
+    if (s->T < 0 || s->T > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
+    if (s->d <= 0 || s->V <= 0 || s->P <= 0 || s->G <= 0) return AIS_ERR_SHAPE;
+    if (s->d % 128 != 0 || s->V % 8 != 0) return AIS_ERR_SHAPE;
+    if (s->fp8_block != 32 && s->fp8_block != 64 && s->fp8_block != 128) return AIS_ERR_SHAPE;
+    if (s->d % s->fp8_block != 0) return AIS_ERR_SHAPE;
+    if (s->ldh < s->d || s->ldw < s->d) return AIS_ERR_SHAPE;
+    if (s->ldh % 16 != 0 || s->ldw % 16 != 0) return AIS_ERR_ALIGN;
+    if (static_cast<int64_t>(s->P) * s->G > (1 << 24)) return AIS_ERR_SHAPE;
+    return AIS_OK;
+}
+
+int check_params(const ais_params* p) {
+    if (!p) return AIS_ERR_NULL;
+    if (!(p->C >= 1.0f) || !(p->delta > 0.f) || !(p->gamma > 0.f) || !(p->eps >= 0.f) || !(p->clip_eps >= 0.f) ||
+        !(p->beta_var >= 0.f))
+        return AIS_ERR_PARAM;
+    if (!isnan(p->alpha_override) && !(p->alpha_override >= 0.f && p->alpha_override <= 1.f)) return AIS_ERR_PARAM;
+    if (p->vocab_chunk < 0) return AIS_ERR_PARAM;
+    return AIS_OK;
+}
+
+int pick_nsplit(const ais_shape* s, const ais_params* p) {
+    const int n_col_tiles = (s->V + kBN - 1) / kBN;
+    int nsplit = 4;
+    if (p->vocab_chunk > 0) nsplit = (s->V + p->vocab_chunk - 1) / p->vocab_chunk;
+    if (nsplit > 64) nsplit = 64;
+    if (nsplit > n_col_tiles) nsplit = n_col_tiles;
+    if (nsplit < 1) nsplit = 1;
+    return nsplit;
+}
+
+struct Layout {
+    int64_t t_ld;          // padded length of per-row vectors
+    int nsplit, nparts;
+    size_t off_part_m, off_part_s, off_part_z;   // forward partials
+    size_t off_diag;                              // reduction partials (doubles)
+    size_t off_coef, off_nseq;                    // backward: c_t, valid rows per sequence
+    size_t off_u;                                 // backward scratch
+    int64_t ldU;
+    size_t fixed_bytes;                           // everything but the scratch rows
+    size_t u_row_bytes;
+};
+
+Layout make_layout(const ais_shape* s, const ais_params* p) {
+    Layout L;
+    L.t_ld = static_cast<int64_t>(align_up(static_cast<size_t>(s->T > 0 ? s->T : 1), 64));
+    L.nsplit = pick_nsplit(s, p);
+    L.nparts = L.nsplit * 2;
+    size_t off = 0;
+    const size_t part_bytes = align_up(static_cast<size_t>(L.nparts) * L.t_ld * sizeof(float), 256);
+    L.off_part_m = off; off += part_bytes;
+    L.off_part_s = off; off += part_bytes;
+    L.off_part_z = off; off += part_bytes;
+    L.off_diag = off;   off += align_up(static_cast<size_t>(kDiagBlocks) * kNumMoments * sizeof(double), 256);
+    L.off_coef = off;   off += align_up(static_cast<size_t>(L.t_ld) * sizeof(float), 256);
+    L.off_nseq = off;   off += align_up(static_cast<size_t>(s->P) * s->G * sizeof(int32_t), 256);
+    L.off_u = off;
+    L.ldU = static_cast<int64_t>(align_up(static_cast<size_t>(s->V), 64));
+    L.fixed_bytes = off;
+    L.u_row_bytes = static_cast<size_t>(L.ldU) * sizeof(__nv_bfloat16);
+    return L;
+}
+
+constexpr int64_t kBwdRowsRecommended = 2 * 148 * kBM;
+
+}  // namespace
+
+extern "C" {
+
+int ais_version(void) { return AIS_VERSION; }
+
+const char* ais_strerror(int status) {
+    switch (status) {
+        case AIS_OK: return "ok";
+        case AIS_ERR_NULL: return "a required pointer is NULL";
+        case AIS_ERR_SHAPE: return "invalid or inconsistent shape";
+        case AIS_ERR_ALIGN: return "pointer or leading dimension not aligned as required";
+        case AIS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case AIS_ERR_DEVICE: return "no sm_100 device, or a CUDA call failed";
+        case AIS_ERR_PARAM: return "hyper-parameter out of range";
+        case AIS_ERR_LIMIT: return "size beyond a fixed limit of this entry point";
+        default: return "unknown status";
+    }
+}
+
+void ais_default_params(ais_params* p) {
+    if (!p) return;
+    p->C = 5.0f;
+    p->delta = 0.02f;
+    p->gamma = 1.2f;
+    p->eps = 1e-6f;
+    p->beta_var = 1.0f;
+    p->clip_eps = 0.2f;
+    p->alpha_override = NAN;
+    p->adv_std_norm = 0;
+    p->vocab_chunk = 0;
+    p->reserved = 0;
+}
+
+size_t ais_workspace_min_bytes(const ais_shape* shape, const ais_params* params) {
+    if (check_shape(shape) != AIS_OK || check_params(params) != AIS_OK) return 0;
+    const Layout L = make_layout(shape, params);
+    return L.fixed_bytes + static_cast<size_t>(kBM) * L.u_row_bytes;
+}
+
+size_t ais_workspace_bytes(const ais_shape* shape, const ais_params* params) {
+    if (check_shape(shape) != AIS_OK || check_params(params) != AIS_OK) return 0;
+    const Layout L = make_layout(shape, params);
+    int64_t rows = static_cast<int64_t>(align_up(static_cast<size_t>(shape->T > 0 ? shape->T : 1), kBM));
+    if (rows > kBwdRowsRecommended) rows = kBwdRowsRecommended;
+    return L.fixed_bytes + static_cast<size_t>(rows) * L.u_row_bytes;
+}
+
+int ais_quantize_fp8(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes, int64_t ldq,
+                     float* scales, int64_t lds, void* stream) {
+    if (!x || !codes || !scales) return AIS_ERR_NULL;
+    if (rows < 0 || cols < 0 || (block != 32 && block != 64 && block != 128)) return AIS_ERR_SHAPE;
+    if (cols % block != 0 || ld < cols || ldq < cols || lds < rows) return AIS_ERR_SHAPE;
+    if (ld % 8 != 0 || ldq % 8 != 0 || !aligned(x, 16) || !aligned(codes, 8) || !aligned(scales, 4)) return AIS_ERR_ALIGN;
+    if (rows > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
+    int st = device_setup(nullptr);
+    if (st != AIS_OK) return st;
+    return launch_quantize(x, rows, cols, ld, block, codes, ldq, scales, lds, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? AIS_OK
+               : AIS_ERR_DEVICE;
+}
+
+int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void* H, const void* W, const uint8_t* qH,
+                    const float* sH, int64_t ldsH, const uint8_t* qW, const float* sW, int64_t ldsW, const int32_t* tokens,
+                    const uint8_t* mask, float* lp_train, float* lse_train, float* lp_roll, float* lse_roll,
+                    uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream) {
+    int st = check_shape(shape);
+    if (st != AIS_OK) return st;
+    st = check_params(params);
+    if (st != AIS_OK) return st;
+    if (!tokens || !mask) return AIS_ERR_NULL;
+    const bool do_train = lp_train != nullptr, do_roll = lp_roll != nullptr;
+    if (do_train && (!H || !W)) return AIS_ERR_NULL;
+    if (do_roll && (!qH || !sH || !qW || !sW)) return AIS_ERR_NULL;
+    if (do_train && (!aligned(H, 16) || !aligned(W, 16))) return AIS_ERR_ALIGN;
+    if (do_roll) {
+        if (!aligned(qH, 16) || !aligned(qW, 16) || !aligned(sH, 16) || !aligned(sW, 16)) return AIS_ERR_ALIGN;
+        if (ldsH < shape->T || ldsW < shape->V) return AIS_ERR_SHAPE;
+        if (ldsH % 4 != 0 || ldsW % 4 != 0) return AIS_ERR_ALIGN;
+    }
+    const Layout L = make_layout(shape, params);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.off_diag) return AIS_ERR_WORKSPACE;
+    int num_sms = 0;
+    st = device_setup(&num_sms);
+    if (st != AIS_OK) return st;
+    if (shape->T == 0 || (!do_train && !do_roll)) return AIS_OK;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    LmheadArgs a;
+    memset(&a, 0, sizeof(a));
+    a.rows = shape->T;
+    a.row0 = 0;
+    a.n_row_tiles = static_cast<int32_t>((shape->T + kBM - 1) / kBM);
+    a.ncols = shape->V;
+    a.n_col_tiles = (shape->V + kBN - 1) / kBN;
+    a.nsplit = L.nsplit;
+    a.sgroups = 128 / shape->fp8_block;
+    a.tokens = tokens;
+    a.mask = mask;
+    a.part_m = reinterpret_cast<float*>(ws + L.off_part_m);
+    a.part_s = reinterpret_cast<float*>(ws + L.off_part_s);
+    a.part_z = reinterpret_cast<float*>(ws + L.off_part_z);
+    a.part_ld = L.t_ld;
+    a.status = dev_status;
+    const int units = a.n_row_tiles * a.nsplit;
+    const int ctas = units < num_sms ? units : num_sms;
+    const uint64_t T = static_cast<uint64_t>(shape->T), V = static_cast<uint64_t>(shape->V), d = static_cast<uint64_t>(shape->d);
+
+    CUtensorMap tmA, tmB, tmSA, tmSB;
+    if (do_train) {
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, H, d, T, shape->ldh * 2, 64, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
+            return AIS_ERR_DEVICE;
+        a.ksteps = shape->d / 64;
+        if (launch_lmhead(kFwdBf16, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
+        if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_train, lse_train, dev_status, s) !=
+            cudaSuccess)
+            return AIS_ERR_DEVICE;
+    }
+    if (do_roll) {
+        const uint64_t nkb = d / shape->fp8_block;
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmSA, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, sH, T, nkb, ldsH * 4, kBM, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+            !make_tmap(&tmSB, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, sW, V, nkb, ldsW * 4, kBN, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE))
+            return AIS_ERR_DEVICE;
+        a.ksteps = shape->d / 128;
+        if (launch_lmhead(kFwdFp8, tmA, tmB, tmSA, tmSB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
+        if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_roll, lse_roll, dev_status, s) !=
+            cudaSuccess)
+            return AIS_ERR_DEVICE;
+    }
+    return AIS_OK;
+}
+
+int ais_diagnostics(const ais_shape* shape, const ais_params* params, const float* lp_train, const float* lp_roll,
+                    const uint8_t* mask, const int32_t* seq_offsets, const float* rewards, float* adv, int32_t* n_valid_seq,
+                    float* rho, float* w_tilde, ais_diag* diag, void* workspace, size_t workspace_bytes, void* stream) {
+    int st = check_shape(shape);
+    if (st != AIS_OK) return st;
+    st = check_params(params);
+    if (st != AIS_OK) return st;
+    if (!lp_train || !lp_roll || !mask || !seq_offsets || !rewards || !adv || !w_tilde || !diag) return AIS_ERR_NULL;
+    if (!aligned(diag, 8)) return AIS_ERR_ALIGN;
+    const Layout L = make_layout(shape, params);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.off_coef) return AIS_ERR_WORKSPACE;
+    st = device_setup(nullptr);
+    if (st != AIS_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const int S = shape->P * shape->G;
+    if (launch_seq_stats(mask, seq_offsets, rewards, S, shape->G, params->adv_std_norm, params->eps, adv, n_valid_seq, s) !=
+        cudaSuccess)
+        return AIS_ERR_DEVICE;
+    if (launch_diag(lp_train, lp_roll, mask, seq_offsets, adv, shape->T, S, *params, reinterpret_cast<double*>(ws + L.off_diag),
+                    rho, w_tilde, diag, s) != cudaSuccess)
+        return AIS_ERR_DEVICE;
+    return AIS_OK;
+}
+
+int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H, const void* W, const int32_t* tokens,
+                 const uint8_t* mask, const int32_t* seq_offsets, const float* lse_train, const float* lp_train,
+                 const float* lp_old, const float* adv, const float* w_tilde, void* dH, float* loss, ais_diag* diag,
+                 uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream) {
+    int st = check_shape(shape);
+    if (st != AIS_OK) return st;
+    st = check_params(params);
+    if (st != AIS_OK) return st;
+    if (!H || !W || !tokens || !mask || !seq_offsets || !lse_train || !lp_train || !adv || !w_tilde || !dH) return AIS_ERR_NULL;
+    if (!aligned(H, 16) || !aligned(W, 16) || !aligned(dH, 16)) return AIS_ERR_ALIGN;
+    const Layout L = make_layout(shape, params);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.fixed_bytes + static_cast<size_t>(kBM) * L.u_row_bytes)
+        return AIS_ERR_WORKSPACE;
+    int num_sms = 0;
+    st = device_setup(&num_sms);
+    if (st != AIS_OK) return st;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const int S = shape->P * shape->G;
+    float* coef = reinterpret_cast<float*>(ws + L.off_coef);
+    int32_t* nseq = reinterpret_cast<int32_t*>(ws + L.off_nseq);
+    if (launch_seq_stats(mask, seq_offsets, nullptr, S, shape->G, 0, 0.f, nullptr, nseq, s) != cudaSuccess) return AIS_ERR_DEVICE;
+    if (launch_loss_coef(lp_train, lp_old, mask, seq_offsets, adv, w_tilde, nseq, shape->T, S, params->clip_eps,
+                         reinterpret_cast<double*>(ws + L.off_diag), coef, loss, diag, s) != cudaSuccess)
+        return AIS_ERR_DEVICE;
+    if (shape->T == 0) return AIS_OK;
+
+    // rows of scratch the workspace can hold (whole row tiles)
+    int64_t blk_rows = static_cast<int64_t>((workspace_bytes - L.fixed_bytes) / L.u_row_bytes) / kBM * kBM;
+    const int64_t t_pad = static_cast<int64_t>(align_up(static_cast<size_t>(shape->T), kBM));
+    if (blk_rows > t_pad) blk_rows = t_pad;
+    __nv_bfloat16* U = reinterpret_cast<__nv_bfloat16*>(ws + L.off_u);
+    const uint64_t V = static_cast<uint64_t>(shape->V), d = static_cast<uint64_t>(shape->d);
+
+    CUtensorMap tmW_k, tmW_n, tmU;
+    if (!make_tmap(&tmW_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap(&tmW_n, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, d, V, shape->ldw * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap(&tmU, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, U, V, static_cast<uint64_t>(blk_rows), L.ldU * 2, 64, kBM,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+        return AIS_ERR_DEVICE;
+
+    for (int64_t r0 = 0; r0 < shape->T; r0 += blk_rows) {
+        const int64_t rows = (shape->T - r0) < blk_rows ? (shape->T - r0) : blk_rows;
+        CUtensorMap tmH;
+        const __nv_bfloat16* Hc = static_cast<const __nv_bfloat16*>(H) + r0 * shape->ldh;
+        if (!make_tmap(&tmH, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Hc, d, static_cast<uint64_t>(rows), shape->ldh * 2, 64, kBM,
+                       CU_TENSOR_MAP_SWIZZLE_128B))
+            return AIS_ERR_DEVICE;
+        LmheadArgs a;
+        memset(&a, 0, sizeof(a));
+        a.rows = rows;
+        a.row0 = r0;
+        a.n_row_tiles = static_cast<int32_t>((rows + kBM - 1) / kBM);
+        a.tokens = tokens;
+        a.mask = mask;
+        a.lse = lse_train;
+        a.U = U;
+        a.ldU = L.ldU;
+        a.coef = coef;
+        a.dH = static_cast<__nv_bfloat16*>(dH);
+        a.lddh = shape->ldh;
+        a.status = dev_status;
+        a.sgroups = 1;
+        // recompute softmax - onehot into the scratch
+        a.ncols = shape->V;
+        a.n_col_tiles = (shape->V + kBN - 1) / kBN;
+        a.nsplit = L.nsplit;
+        a.ksteps = shape->d / 64;
+        int units = a.n_row_tiles * a.nsplit;
+        if (launch_lmhead(kBwdP, tmH, tmW_k, tmH, tmW_k, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
+            return AIS_ERR_DEVICE;
+        // dH = c (.) (U W)
+        a.ncols = shape->d;
+        a.n_col_tiles = (shape->d + kBN - 1) / kBN;
+        a.nsplit = 1;
+        a.ksteps = (shape->V + 63) / 64;
+        units = a.n_row_tiles * a.n_col_tiles;
+        if (launch_lmhead(kBwdDh, tmU, tmW_n, tmU, tmW_n, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
+            return AIS_ERR_DEVICE;
+    }
+    return AIS_OK;
+}
+
+}  // extern "C"

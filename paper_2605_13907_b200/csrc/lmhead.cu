@@ -1,0 +1,413 @@
+// LM-head tensor-core passes for sm_100a: TMA-fed tcgen05.mma with accumulators in tensor memory and
+// fused epilogues (streaming log-sum-exp + target pick, softmax-minus-onehot scratch, dH scaling).
+//
+// One persistent CTA per SM.  Warp 0 issues TMA tile loads, warp 1 issues the MMAs, warps 2..9 are the
+// epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (one row per thread) and column half (w-2)/4 of the
+// 256-column accumulator.  Two 256-column accumulators alternate so that the epilogue of one tile (or,
+// in the FP8 pass, the promotion of one scale block) overlaps the MMAs of the next.
+#include "lmhead.cuh"
+#include "ptx.cuh"
+#include "../../include/ais.h"
+
+namespace ais {
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kNegBig = -1.0e30f;
+
+struct Pipe {
+    uint32_t idx = 0, phase = 0;
+    int n;
+    __device__ explicit Pipe(int n_) : n(n_) {}
+    __device__ __forceinline__ void advance() {
+        if (++idx == static_cast<uint32_t>(n)) { idx = 0; phase ^= 1u; }
+    }
+};
+
+// Warp-wide wait: every lane polls (so every lane observes the completed phase itself) and the outcome is
+// made uniform, because the tcgen05.ld / __syncwarp that follow need the whole warp.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    const bool r = mbar_wait(bar, parity, abort_flag);
+    return __all_sync(0xffffffffu, r);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Which row tile and which column tiles a work unit covers.
+struct Unit {
+    int rt, t0, t1, part;
+};
+template <int MODE>
+__device__ __forceinline__ Unit decode_unit(const LmheadArgs& a, int u) {
+    Unit w;
+    if (MODE == kBwdDh) {
+        w.rt = u / a.n_col_tiles;
+        w.t0 = u % a.n_col_tiles;
+        w.t1 = w.t0 + 1;
+        w.part = 0;
+    } else {
+        w.rt = u / a.nsplit;
+        const int c = u % a.nsplit;
+        w.t0 = static_cast<int>((static_cast<int64_t>(c) * a.n_col_tiles) / a.nsplit);
+        w.t1 = static_cast<int>((static_cast<int64_t>(c + 1) * a.n_col_tiles) / a.nsplit);
+        w.part = c;
+    }
+    return w;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1)
+lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+              const __grid_constant__ CUtensorMap tmSA, const __grid_constant__ CUtensorMap tmSB,
+              const LmheadArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* stage_base = smem;
+    uint8_t* scale_base = smem + kStages * kStageBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(scale_base + kScaleSlots * kScaleSlotBytes);
+    uint64_t* full = bars;                       // [kStages]   TMA -> MMA
+    uint64_t* empty = full + kStages;            // [kStages]   MMA -> TMA
+    uint64_t* tfull = empty + kStages;           // [2]         MMA -> epilogue
+    uint64_t* tempty = tfull + 2;                // [2]         epilogue -> MMA
+    uint64_t* sfull = tempty + 2;                // [kScaleSlots] TMA -> epilogue (FP8 scales)
+    uint64_t* sempty = sfull + kScaleSlots;      // [kScaleSlots] epilogue -> TMA
+    uint64_t* done = sempty + kScaleSlots;       // [1]         all MMAs of this CTA have completed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBarriers);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_units = (MODE == kBwdDh) ? a.n_row_tiles * a.n_col_tiles : a.n_row_tiles * a.nsplit;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
+        for (int i = 0; i < kScaleSlots; ++i) { mbar_init(&sfull[i], 1); mbar_init(&sempty[i], kEpiWarps); }
+        mbar_init(done, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            Pipe st(kStages), sc(kScaleSlots);
+            uint32_t issued = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+                const Unit w = decode_unit<MODE>(a, u);
+                for (int t = w.t0; t < w.t1 && ok; ++t) {
+                    for (int ks = 0; ks < a.ksteps; ++ks) {
+                        if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag)) { ok = false; break; }
+                        uint8_t* sA = stage_base + st.idx * kStageBytes;
+                        uint8_t* sB = sA + kAStageBytes;
+                        mbar_expect_tx(&full[st.idx], kStageBytes);
+                        const int kelem = (MODE == kFwdFp8) ? ks * 128 : ks * 64;
+                        tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kBM);
+                        if (MODE == kBwdDh) {
+                            // B is W[v, n]: n (the output column) is the contiguous axis -> four 64-column boxes
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                tma_load_2d(sB + j * (kBStageBytes / 4), &tmB, &full[st.idx], t * kBN + j * 64, kelem);
+                        } else {
+                            tma_load_2d(sB, &tmB, &full[st.idx], kelem, t * kBN);
+                        }
+                        ++issued;
+                        st.advance();
+                        if (MODE == kFwdFp8) {
+                            if (!mbar_wait(&sempty[sc.idx], sc.phase ^ 1u, abort_flag)) { ok = false; break; }
+                            uint8_t* sS = scale_base + sc.idx * kScaleSlotBytes;
+                            mbar_expect_tx(&sfull[sc.idx], static_cast<uint32_t>(a.sgroups) * (kBM + kBN) * 4u);
+                            tma_load_2d(sS, &tmSA, &sfull[sc.idx], w.rt * kBM, ks * a.sgroups);
+                            tma_load_2d(sS + kScaleBOffset, &tmSB, &sfull[sc.idx], t * kBN, ks * a.sgroups);
+                            sc.advance();
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                // another role gave up: let the copies already in flight land before the CTA exits
+                const uint32_t pending = issued < static_cast<uint32_t>(kStages) ? issued : kStages;
+                for (uint32_t i = 0; i < pending; ++i) {
+                    const uint32_t n = issued - 1 - i;                 // n-th load overall
+                    mbar_wait_drain(&full[n % kStages], (n / kStages) & 1u);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc =
+                (MODE == kFwdFp8) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
+                                  : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, 0, MODE == kBwdDh ? 1 : 0);
+            Pipe st(kStages), tb(2);
+            bool ok = true;
+            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+                const Unit w = decode_unit<MODE>(a, u);
+                for (int t = w.t0; t < w.t1 && ok; ++t) {
+                    if (MODE != kFwdFp8) {
+                        if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                    }
+                    for (int ks = 0; ks < a.ksteps; ++ks) {
+                        if (!mbar_wait(&full[st.idx], st.phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sA = smem_u32(stage_base + st.idx * kStageBytes);
+                        const uint32_t sB = sA + kAStageBytes;
+                        if (MODE == kFwdFp8) {
+                            const int per = 4 / a.sgroups;             // MMAs per scale block
+                            for (int g = 0; g < a.sgroups && ok; ++g) {
+                                if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag)) { ok = false; break; }
+                                tc_fence_after();
+                                const uint32_t dcol = tmem_base + tb.idx * kBN;
+                                for (int j = 0; j < per; ++j) {
+                                    const uint32_t off = (g * per + j) * 32;
+                                    mma_f8(dcol, smem_desc_sw128(sA + off, 16, 1024), smem_desc_sw128(sB + off, 16, 1024),
+                                           idesc, j > 0 ? 1u : 0u);
+                                }
+                                tc_commit(&tfull[tb.idx]);
+                                tb.advance();
+                            }
+                            if (!ok) break;
+                        } else {
+                            const uint32_t dcol = tmem_base + tb.idx * kBN;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const uint64_t adesc = smem_desc_sw128(sA + j * 32, 16, 1024);
+                                const uint64_t bdesc = (MODE == kBwdDh)
+                                                           ? smem_desc_sw128(sB + j * 2048, kBStageBytes / 4, 1024)
+                                                           : smem_desc_sw128(sB + j * 32, 16, 1024);
+                                mma_f16(dcol, adesc, bdesc, idesc, (ks > 0 || j > 0) ? 1u : 0u);
+                            }
+                        }
+                        tc_commit(&empty[st.idx]);
+                        st.advance();
+                    }
+                    if (MODE != kFwdFp8 && ok) {
+                        tc_commit(&tfull[tb.idx]);
+                        tb.advance();
+                    }
+                }
+            }
+            // everything issued has to finish before the tensor memory is given back
+            tc_commit(done);
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;             // column half of the accumulator
+        const int r_in_tile = q * 32 + lane;
+        const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+        Pipe tb(2), sc(kScaleSlots);
+        bool ok = true;
+        uint32_t flags = 0;
+        for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+            const Unit w = decode_unit<MODE>(a, u);
+            const int64_t lrow = static_cast<int64_t>(w.rt) * kBM + r_in_tile;   // row inside this launch
+            const bool row_ok = lrow < a.rows;
+            const int64_t grow = a.row0 + lrow;
+            int y = -1;
+            bool valid = false;
+            if (row_ok && MODE != kBwdDh) {
+                y = a.tokens[grow];
+                valid = a.mask[grow] != 0;
+                if (valid && (y < 0 || y >= a.ncols)) { flags |= AIS_FLAG_TOKEN_RANGE; y = -1; }
+            }
+            float m2 = kNegBig, s = 0.f, zy = -INFINITY;       // log2-domain running max, sum, target logit
+            float lse2 = 0.f, coef = 0.f;
+            if (MODE == kBwdP && row_ok) lse2 = a.lse[grow] * kLog2e;
+            if (MODE == kBwdDh && row_ok) coef = a.coef[grow];
+
+            for (int t = w.t0; t < w.t1 && ok; ++t) {
+                const int col_base = t * kBN + half * 128;    // first output column of this thread's half
+                float acc[128];
+                if (MODE == kFwdFp8) {
+#pragma unroll
+                    for (int i = 0; i < 128; ++i) acc[i] = 0.f;
+                    for (int ks = 0; ks < a.ksteps && ok; ++ks) {
+                        if (!mbar_wait_warp(&sfull[sc.idx], sc.phase, abort_flag)) { ok = false; break; }
+                        const float* sS = reinterpret_cast<const float*>(scale_base + sc.idx * kScaleSlotBytes);
+                        for (int g = 0; g < a.sgroups; ++g) {
+                            if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                            const float sh = sS[g * kBM + r_in_tile];
+                            const float4* sw4 = reinterpret_cast<const float4*>(sS + (kScaleBOffset / 4) + g * kBN + half * 128);
+                            const uint32_t taddr = tmem_base + lane_addr + tb.idx * kBN + half * 128;
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t v[32];
+                                tmem_ld32(taddr + c * 32, v);
+                                tmem_ld_wait();
+#pragma unroll
+                                for (int i = 0; i < 32; i += 4) {
+                                    const float4 sw = sw4[(c * 32 + i) >> 2];
+                                    acc[c * 32 + i + 0] = fmaf(sh * sw.x, __uint_as_float(v[i + 0]), acc[c * 32 + i + 0]);
+                                    acc[c * 32 + i + 1] = fmaf(sh * sw.y, __uint_as_float(v[i + 1]), acc[c * 32 + i + 1]);
+                                    acc[c * 32 + i + 2] = fmaf(sh * sw.z, __uint_as_float(v[i + 2]), acc[c * 32 + i + 2]);
+                                    acc[c * 32 + i + 3] = fmaf(sh * sw.w, __uint_as_float(v[i + 3]), acc[c * 32 + i + 3]);
+                                }
+                            }
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&tempty[tb.idx]);
+                            tb.advance();
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sempty[sc.idx]);
+                        sc.advance();
+                    }
+                    if (!ok) break;
+                } else {
+                    if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                }
+
+                const uint32_t taddr = tmem_base + lane_addr + tb.idx * kBN + half * 128;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int col0 = col_base + c * 32;
+                    float x[32];
+                    if (MODE == kFwdFp8) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) x[i] = acc[c * 32 + i];
+                    } else {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + c * 32, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(v[i]);
+                    }
+                    if (MODE == kFwdBf16 || MODE == kFwdFp8) {
+                        if (y >= col0 && y < col0 + 32) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (col0 + i == y) zy = x[i];
+                        }
+                        if (col0 + 32 > a.ncols) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (col0 + i >= a.ncols) x[i] = -INFINITY;
+                        }
+                        float cm = x[0];
+#pragma unroll
+                        for (int i = 1; i < 32; ++i) cm = fmaxf(cm, x[i]);
+                        const float m_new = fmaxf(m2, cm * kLog2e);
+                        float add = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) add += ex2(fmaf(x[i], kLog2e, -m_new));
+                        s = fmaf(s, ex2(m2 - m_new), add);
+                        m2 = m_new;
+                    } else if (MODE == kBwdP) {
+                        if (row_ok && col0 < a.ncols) {
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int i = 0; i < 32; i += 2) {
+                                float p0 = valid ? ex2(fmaf(x[i], kLog2e, -lse2)) : 0.f;
+                                float p1 = valid ? ex2(fmaf(x[i + 1], kLog2e, -lse2)) : 0.f;
+                                if (col0 + i == y) p0 -= 1.f;
+                                if (col0 + i + 1 == y) p1 -= 1.f;
+                                pk[i >> 1] = pack_bf16(p0, p1);
+                            }
+                            uint4* dst = reinterpret_cast<uint4*>(a.U + lrow * a.ldU + col0);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (col0 + j * 8 < a.ncols) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                        }
+                    } else {   // kBwdDh
+                        if (row_ok && col0 < a.ncols) {
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int i = 0; i < 32; i += 2) {
+                                const float v0 = (coef == 0.f) ? 0.f : coef * x[i];
+                                const float v1 = (coef == 0.f) ? 0.f : coef * x[i + 1];
+                                pk[i >> 1] = pack_bf16(v0, v1);
+                            }
+                            uint4* dst = reinterpret_cast<uint4*>(a.dH + grow * a.lddh + col0);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (col0 + j * 8 < a.ncols) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                        }
+                    }
+                }
+                if (MODE != kFwdFp8) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tempty[tb.idx]);
+                    tb.advance();
+                }
+            }
+            if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8)) {
+                const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow;
+                a.part_m[o] = m2 * kLn2;
+                a.part_s[o] = s;
+                a.part_z[o] = zy;
+            }
+        }
+        if (flags && a.status) atomicOr(a.status, flags);
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        if (lane == 0) mbar_wait_drain(done, 0);   // immediate unless the CTA is giving up early
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && *abort_flag && a.status) atomicOr(a.status, AIS_FLAG_TIMEOUT);
+}
+
+}  // namespace
+
+template <int MODE>
+static cudaError_t launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA, const CUtensorMap& tmSB,
+                               const LmheadArgs& args, int num_ctas, cudaStream_t stream) {
+    lmhead_kernel<MODE><<<num_ctas, kThreads, kSmemBytes, stream>>>(tmA, tmB, tmSA, tmSB, args);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
+                          const CUtensorMap& tmSB, const LmheadArgs& args, int num_ctas, cudaStream_t stream) {
+    switch (mode) {
+        case kFwdBf16: return launch_mode<kFwdBf16>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
+        case kFwdFp8:  return launch_mode<kFwdFp8>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
+        case kBwdP:    return launch_mode<kBwdP>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
+        case kBwdDh:   return launch_mode<kBwdDh>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t lmhead_prepare() {
+    cudaError_t e;
+    e = cudaFuncSetAttribute(lmhead_kernel<kFwdBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(lmhead_kernel<kFwdFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(lmhead_kernel<kBwdP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(lmhead_kernel<kBwdDh>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+}  // namespace ais

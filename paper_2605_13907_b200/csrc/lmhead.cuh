@@ -1,0 +1,61 @@
+// Arguments shared by the host launcher and the LM-head tensor-core kernels.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace ais {
+
+enum LmheadMode : int {
+    kFwdBf16 = 0,   // z = H W^T (bf16), streaming log-sum-exp + target pick -> partial triples
+    kFwdFp8  = 1,   // z^ from E4M3 codes with per-block scale promotion, same epilogue
+    kBwdP    = 2,   // recompute z (bf16), write u = softmax - onehot as bf16 scratch
+    kBwdDh   = 3    // dH = c (.) (U W), contraction over the vocabulary
+};
+
+constexpr int kBM = 128;                 // rows per tile (TMEM lanes)
+constexpr int kBN = 256;                 // columns per tile (TMEM columns of one accumulator)
+constexpr int kStageKBytes = 128;        // bytes of K per shared-memory stage row (one swizzle span)
+constexpr int kAStageBytes = kBM * kStageKBytes;
+constexpr int kBStageBytes = kBN * kStageKBytes;
+constexpr int kStageBytes = kAStageBytes + kBStageBytes;
+constexpr int kStages = 4;
+constexpr int kScaleSlots = 4;
+constexpr int kScaleSlotBytes = 4 * (kBM + kBN) * 4;   // up to 4 scale blocks per stage
+constexpr int kScaleBOffset = 4 * kBM * 4;
+constexpr int kNumBarriers = 2 * kStages + 4 + 2 * kScaleSlots + 1;
+constexpr int kThreads = 320;            // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int kEpiWarps = 8;
+constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kScaleSlots * kScaleSlotBytes + kNumBarriers * 8 + 64;
+
+struct LmheadArgs {
+    int64_t rows;          // valid rows handled by this launch
+    int64_t row0;          // global index of local row 0 (per-row vectors are indexed globally)
+    int32_t n_row_tiles;
+    int32_t ncols;         // output columns: V (forward, recompute) or d (dH)
+    int32_t n_col_tiles;
+    int32_t ksteps;        // shared-memory stages per accumulator tile
+    int32_t nsplit;        // forward / recompute: independent column ranges per row tile
+    int32_t sgroups;       // FP8: scale blocks per stage (128 / fp8_block)
+    const int32_t* tokens;
+    const uint8_t* mask;
+    float* part_m;         // [nsplit*2][part_ld] running maxima (natural log units)
+    float* part_s;         // sums of exp(z - m)
+    float* part_z;         // target logit or -inf
+    int64_t part_ld;
+    const float* lse;      // recompute: log-sum-exp of the trainer pass
+    __nv_bfloat16* U;      // recompute output / dH input scratch [rows_pad, ldU]
+    int64_t ldU;
+    const float* coef;     // dH: per-row factor c_t
+    __nv_bfloat16* dH;
+    int64_t lddh;
+    uint32_t* status;
+};
+
+// Launches one pass.  tmSA / tmSB are only read in kFwdFp8 mode.
+cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
+                          const CUtensorMap& tmSB, const LmheadArgs& args, int num_ctas, cudaStream_t stream);
+cudaError_t lmhead_prepare();   // sets the dynamic shared-memory attribute of every instantiation
+
+}  // namespace ais

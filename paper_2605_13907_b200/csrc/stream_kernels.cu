@@ -1,0 +1,375 @@
+// Streaming kernels of the AIS path (everything that is not a dense contraction).
+#include "stream_kernels.cuh"
+
+#include <cuda_bf16.h>
+#include <math.h>
+
+namespace ais {
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------
+// FP8-E4M3 block quantisation.  A CTA covers 32 rows x 2048 columns; each warp walks 4 rows, a lane
+// holds 8 consecutive bf16 values (16-byte load), the lanes of one block share the block's amax by
+// shuffles, and the block-major scales are staged in shared memory so that they leave coalesced.
+// ------------------------------------------------------------------------------------------------
+constexpr int kQRows = 32;
+constexpr int kQCols = 2048;
+constexpr int kQThreads = 256;
+
+__device__ __forceinline__ uint16_t cvt_e4m3x2(float hi, float lo) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+template <int BLOCK>
+__global__ void __launch_bounds__(kQThreads) quantize_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols,
+                                                             int64_t ld, uint8_t* __restrict__ codes, int64_t ldq,
+                                                             float* __restrict__ scales, int64_t lds) {
+    constexpr int kLanesPerBlock = BLOCK / 8;
+    constexpr int kBlocksPerTile = kQCols / BLOCK;
+    __shared__ float sc[kBlocksPerTile][kQRows + 1];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kQRows;
+    const int64_t col0 = static_cast<int64_t>(blockIdx.x) * kQCols;
+
+#pragma unroll
+    for (int rr = 0; rr < 4; ++rr) {
+        const int r_local = warp * 4 + rr;
+        const int64_t row = row0 + r_local;
+        if (row >= rows) break;
+        const __nv_bfloat16* xr = x + row * ld;
+        uint4 raw[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int64_t col = col0 + it * 256 + lane * 8;
+            raw[it] = (col < cols) ? __ldg(reinterpret_cast<const uint4*>(xr + col)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int64_t col = col0 + it * 256 + lane * 8;
+            float v[8];
+            const uint32_t w[4] = {raw[it].x, raw[it].y, raw[it].z, raw[it].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                v[2 * i] = __uint_as_float(w[i] << 16);
+                v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+            }
+            float amax = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
+#pragma unroll
+            for (int off = 1; off < kLanesPerBlock; off <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+            const float s = (amax == 0.f) ? 1.0f : __fdiv_rn(amax, 448.0f);
+            if (col < cols) {
+                float qv[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) qv[i] = __fdiv_rn(v[i], s);
+                uint2 out;
+                out.x = static_cast<uint32_t>(cvt_e4m3x2(qv[1], qv[0])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[3], qv[2])) << 16);
+                out.y = static_cast<uint32_t>(cvt_e4m3x2(qv[5], qv[4])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[7], qv[6])) << 16);
+                *reinterpret_cast<uint2*>(codes + row * ldq + col) = out;
+                if ((lane % kLanesPerBlock) == 0) sc[(it * 256 + lane * 8) / BLOCK][r_local] = s;
+            }
+        }
+    }
+    __syncthreads();
+    const int64_t kb0 = col0 / BLOCK;
+    const int64_t nkb = cols / BLOCK;
+    for (int idx = threadIdx.x; idx < kBlocksPerTile * kQRows; idx += kQThreads) {
+        const int kb_l = idx / kQRows, r_l = idx % kQRows;
+        if (kb0 + kb_l < nkb && row0 + r_l < rows) scales[(kb0 + kb_l) * lds + row0 + r_l] = sc[kb_l][r_l];
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Merge of the per-split (max, sum-exp, target-logit) triples into lp and lse.
+// ------------------------------------------------------------------------------------------------
+__global__ void combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_s,
+                               const float* __restrict__ part_z, int nparts, int64_t part_ld,
+                               const uint8_t* __restrict__ mask, int64_t T, float* __restrict__ lp,
+                               float* __restrict__ lse, uint32_t* status) {
+    uint32_t flags = 0;
+    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T;
+         t += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        float out_lp = 0.f, out_lse = 0.f;
+        if (mask[t]) {
+            float M = -INFINITY, zy = -INFINITY;
+            for (int j = 0; j < nparts; ++j) {
+                M = fmaxf(M, part_m[j * part_ld + t]);
+                zy = fmaxf(zy, part_z[j * part_ld + t]);
+            }
+            float S = 0.f;
+            for (int j = 0; j < nparts; ++j) S += part_s[j * part_ld + t] * expf(part_m[j * part_ld + t] - M);
+            out_lse = M + logf(S);
+            if (zy == -INFINITY) {
+                out_lp = 0.f;                       // token id out of range: flagged by the producer kernel
+            } else {
+                out_lp = zy - out_lse;
+            }
+            if (!isfinite(out_lse) || !isfinite(out_lp)) flags |= AIS_FLAG_NONFINITE;
+        }
+        lp[t] = out_lp;
+        if (lse) lse[t] = out_lse;
+    }
+    if (flags && status) atomicOr(status, flags);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Segmented reductions: valid rows per sequence and group-relative advantages (Eq. grpo_adv).
+// One CTA per sequence.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+
+// Block-wide sum in a fixed order (lanes by butterfly, then warps 0..n-1 serially); result valid in thread 0.
+__device__ double block_sum(double v, double* scratch /*[32]*/) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    double tot = 0.0;
+    if (threadIdx.x == 0) {
+        const int nw = (blockDim.x + 31) >> 5;
+        for (int i = 0; i < nw; ++i) tot += scratch[i];
+    }
+    return tot;
+}
+
+__global__ void seq_stats_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ seq_offsets,
+                                 const float* __restrict__ rewards, int G, int adv_std_norm, float eps,
+                                 float* __restrict__ adv, int32_t* __restrict__ n_valid_seq) {
+    __shared__ double scratch[32];
+    const int s = blockIdx.x;
+    const int b = seq_offsets[s], e = seq_offsets[s + 1];
+    double cnt = 0.0;
+    for (int t = b + threadIdx.x; t < e; t += blockDim.x) cnt += mask[t] ? 1.0 : 0.0;
+    const double tot = block_sum(cnt, scratch);
+    if (threadIdx.x == 0) {
+        if (n_valid_seq) n_valid_seq[s] = static_cast<int32_t>(tot);
+        if (rewards && adv) {
+            const int g0 = (s / G) * G;
+            double mean = 0.0;
+            for (int j = 0; j < G; ++j) mean += static_cast<double>(rewards[g0 + j]);
+            mean /= G;
+            double a = static_cast<double>(rewards[s]) - mean;
+            if (adv_std_norm) {
+                double var = 0.0;
+                for (int j = 0; j < G; ++j) {
+                    const double dlt = static_cast<double>(rewards[g0 + j]) - mean;
+                    var += dlt * dlt;
+                }
+                a /= (sqrt(var / G) + static_cast<double>(eps));
+            }
+            adv[s] = static_cast<float>(a);
+        }
+    }
+}
+
+__device__ __forceinline__ int seq_of_row(const int32_t* __restrict__ seq_offsets, int S, int64_t t) {
+    int lo = 0, hi = S;                 // largest s with seq_offsets[s] <= t
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (static_cast<int64_t>(seq_offsets[mid]) <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Whole-batch masked moments in double precision, fixed grid and fixed summation order.
+//   0 N   1 sum w   2 sum w^2   3 sum |D|   4 sum A   5 sum A^2   6 sum Aw   7 sum (Aw)^2
+//   8 sum (lp_roll - lp_train)   9 sum |exp(lp_train) - exp(lp_roll)|
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
+                                                                const uint8_t* __restrict__ mask,
+                                                                const int32_t* __restrict__ seq_offsets,
+                                                                const float* __restrict__ adv, int64_t T, int S, double logC,
+                                                                double* __restrict__ partials) {
+    __shared__ double scratch[32];
+    double acc[kNumMoments];
+#pragma unroll
+    for (int i = 0; i < kNumMoments; ++i) acc[i] = 0.0;
+    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T;
+         t += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        if (!mask[t]) continue;
+        const double lt = lp_train[t], lr = lp_roll[t];
+        const double dl = lt - lr;
+        const double w = exp(fmin(dl, logC));
+        const double A = adv[seq_of_row(seq_offsets, S, t)];
+        const double Aw = A * w;
+        acc[0] += 1.0;
+        acc[1] += w;
+        acc[2] += w * w;
+        acc[3] += fabs(dl);
+        acc[4] += A;
+        acc[5] += A * A;
+        acc[6] += Aw;
+        acc[7] += Aw * Aw;
+        acc[8] += -dl;
+        acc[9] += fabs(exp(lt) - exp(lr));
+    }
+    for (int i = 0; i < kNumMoments; ++i) {
+        const double tot = block_sum(acc[i], scratch);
+        if (threadIdx.x == 0) partials[blockIdx.x * kNumMoments + i] = tot;
+    }
+}
+
+__global__ void diag_finalize_kernel(const double* __restrict__ partials, int nblocks, ais_params p, ais_diag* __restrict__ diag) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    double m[kNumMoments];
+    for (int i = 0; i < kNumMoments; ++i) m[i] = 0.0;
+    for (int b = 0; b < nblocks; ++b)
+        for (int i = 0; i < kNumMoments; ++i) m[i] += partials[b * kNumMoments + i];
+    ais_diag d;
+    d.status_flags = 0;
+    d.reserved = 0;
+    d.loss = 0.0;
+    const double N = m[0];
+    d.n_valid = N;
+    if (N <= 0.0) {
+        d.mean_w = 1.0; d.cv2 = 0.0; d.ess = 0.0; d.ess_ratio = 1.0; d.alpha_ess = 1.0; d.d_bar = 0.0;
+        d.alpha_mis = 0.0; d.std_A = 0.0; d.std_Aw = 0.0; d.delta_sigma = 0.0; d.alpha_var = 0.0;
+        d.alpha_adaptive = 0.0; d.kl_k1 = 0.0; d.mean_abs_dp = 0.0;
+        d.status_flags |= AIS_FLAG_EMPTY;
+    } else {
+        const double mu = m[1] / N;
+        const double var = fmax(m[2] / N - mu * mu, 0.0);
+        d.mean_w = mu;
+        d.cv2 = var / (mu * mu);
+        d.ess = m[1] * m[1] / m[2];
+        d.ess_ratio = d.ess / N;
+        d.alpha_ess = 1.0 / sqrt(1.0 + d.cv2);
+        d.d_bar = m[3] / N;
+        d.alpha_mis = fmin(1.0, d.d_bar / static_cast<double>(p.delta));
+        const double mA = m[4] / N, mAw = m[6] / N;
+        d.std_A = sqrt(fmax(m[5] / N - mA * mA, 0.0));
+        d.std_Aw = sqrt(fmax(m[7] / N - mAw * mAw, 0.0));
+        d.delta_sigma = d.std_Aw / (d.std_A + static_cast<double>(p.eps));
+        d.alpha_var = fmax(0.0, (d.delta_sigma - static_cast<double>(p.gamma)) / static_cast<double>(p.gamma));
+        d.alpha_adaptive = fmin(1.0, fmax(0.0, d.alpha_ess - static_cast<double>(p.beta_var) * d.alpha_var)) * d.alpha_mis;
+        d.kl_k1 = m[8] / N;
+        d.mean_abs_dp = m[9] / N;
+    }
+    d.alpha = isnan(p.alpha_override) ? d.alpha_adaptive : static_cast<double>(p.alpha_override);
+    *diag = d;
+}
+
+__global__ void rectify_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
+                               const uint8_t* __restrict__ mask, int64_t T, double logC, const ais_diag* __restrict__ diag,
+                               float* __restrict__ rho, float* __restrict__ w_tilde) {
+    const double alpha = diag->alpha;
+    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T;
+         t += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        double r = 1.0, wt = 1.0;
+        if (mask[t]) {
+            const double dl = static_cast<double>(lp_train[t]) - static_cast<double>(lp_roll[t]);
+            r = exp(dl);
+            wt = 1.0 + alpha * (exp(fmin(dl, logC)) - 1.0);
+        }
+        if (rho) rho[t] = static_cast<float>(r);
+        w_tilde[t] = static_cast<float>(wt);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Per-token gradient factor c_t and the surrogate loss (Eq. ais-grpo without the KL term).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_old,
+                                                                  const uint8_t* __restrict__ mask,
+                                                                  const int32_t* __restrict__ seq_offsets,
+                                                                  const float* __restrict__ adv, const float* __restrict__ w_tilde,
+                                                                  const int32_t* __restrict__ n_valid_seq, int64_t T, int S,
+                                                                  double clip_eps, double* __restrict__ partials,
+                                                                  float* __restrict__ coef) {
+    __shared__ double scratch[32];
+    double J = 0.0;
+    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T;
+         t += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        double c = 0.0;
+        if (mask[t]) {
+            const int s = seq_of_row(seq_offsets, S, t);
+            const double A = adv[s];
+            const int n = n_valid_seq[s] > 0 ? n_valid_seq[s] : 1;
+            const double norm = 1.0 / (static_cast<double>(S) * static_cast<double>(n));
+            const double rho_on = lp_old ? exp(static_cast<double>(lp_train[t]) - static_cast<double>(lp_old[t])) : 1.0;
+            const double un = rho_on * A;
+            const double cl = fmin(fmax(rho_on, 1.0 - clip_eps), 1.0 + clip_eps) * A;
+            const double wt = w_tilde[t];
+            J += wt * fmin(un, cl) * norm;
+            if (un <= cl) c = wt * A * rho_on * norm;
+        }
+        coef[t] = static_cast<float>(c);
+    }
+    const double tot = block_sum(J, scratch);
+    if (threadIdx.x == 0) partials[blockIdx.x] = tot;
+}
+
+__global__ void loss_finalize_kernel(const double* __restrict__ partials, int nblocks, float* loss, ais_diag* diag) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    double J = 0.0;
+    for (int b = 0; b < nblocks; ++b) J += partials[b];
+    if (loss) *loss = static_cast<float>(-J);
+    if (diag) diag->loss = -J;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------ launchers
+cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes,
+                            int64_t ldq, float* scales, int64_t lds, cudaStream_t stream) {
+    if (rows == 0 || cols == 0) return cudaSuccess;
+    dim3 grid(static_cast<unsigned>((cols + kQCols - 1) / kQCols), static_cast<unsigned>((rows + kQRows - 1) / kQRows));
+    const __nv_bfloat16* xp = static_cast<const __nv_bfloat16*>(x);
+    switch (block) {
+        case 32:  quantize_kernel<32><<<grid, kQThreads, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scales, lds); break;
+        case 64:  quantize_kernel<64><<<grid, kQThreads, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scales, lds); break;
+        case 128: quantize_kernel<128><<<grid, kQThreads, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scales, lds); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const float* part_m, const float* part_s, const float* part_z, int nparts, int64_t part_ld,
+                           const uint8_t* mask, int64_t T, float* lp, float* lse, uint32_t* status, cudaStream_t stream) {
+    if (T == 0) return cudaSuccess;
+    const int blocks = static_cast<int>(((T + 255) / 256) < 1184 ? ((T + 255) / 256) : 1184);
+    combine_kernel<<<blocks, 256, 0, stream>>>(part_m, part_s, part_z, nparts, part_ld, mask, T, lp, lse, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_seq_stats(const uint8_t* mask, const int32_t* seq_offsets, const float* rewards, int S, int G,
+                             int adv_std_norm, float eps, float* adv, int32_t* n_valid_seq, cudaStream_t stream) {
+    if (S == 0) return cudaSuccess;
+    seq_stats_kernel<<<S, 256, 0, stream>>>(mask, seq_offsets, rewards, G, adv_std_norm, eps, adv, n_valid_seq);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
+                        const float* adv, int64_t T, int S, const ais_params& p, double* partials, float* rho,
+                        float* w_tilde, ais_diag* diag, cudaStream_t stream) {
+    const double logC = log(static_cast<double>(p.C));
+    moments_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, logC, partials);
+    diag_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, p, diag);
+    if (T > 0) {
+        const int blocks = static_cast<int>(((T + 255) / 256) < 1184 ? ((T + 255) / 256) : 1184);
+        rectify_kernel<<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, logC, diag, rho, w_tilde);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const uint8_t* mask, const int32_t* seq_offsets,
+                             const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S,
+                             float clip_eps, double* partials, float* coef, float* loss, ais_diag* diag, cudaStream_t stream) {
+    loss_coef_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, mask, seq_offsets, adv, w_tilde, n_valid_seq,
+                                                                 T, S, static_cast<double>(clip_eps), partials, coef);
+    loss_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, loss, diag);
+    return cudaGetLastError();
+}
+
+}  // namespace ais

@@ -1,0 +1,37 @@
+// Host-callable launchers of the streaming (HBM / latency bound) kernels: FP8 block quantisation, merge of
+// the per-split log-sum-exp partials, segmented and whole-batch reductions, per-token loss coefficients.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ais.h"
+
+namespace ais {
+
+constexpr int kDiagBlocks = 296;      // fixed grid of the batch reductions (keeps the summation order fixed)
+constexpr int kDiagThreads = 256;
+constexpr int kNumMoments = 12;
+
+cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes,
+                            int64_t ldq, float* scales, int64_t lds, cudaStream_t stream);
+
+// lp[t] = z_y - lse, lse[t] from nparts partial triples laid out [nparts][part_ld].
+cudaError_t launch_combine(const float* part_m, const float* part_s, const float* part_z, int nparts, int64_t part_ld,
+                           const uint8_t* mask, int64_t T, float* lp, float* lse, uint32_t* status, cudaStream_t stream);
+
+// n_valid_seq[s] and (when rewards != nullptr) adv[s].
+cudaError_t launch_seq_stats(const uint8_t* mask, const int32_t* seq_offsets, const float* rewards, int S, int G,
+                             int adv_std_norm, float eps, float* adv, int32_t* n_valid_seq, cudaStream_t stream);
+
+cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
+                        const float* adv, int64_t T, int S, const ais_params& p, double* partials /*[kDiagBlocks][kNumMoments]*/,
+                        float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
+
+// coef[t] and the loss; n_valid_seq must already hold the valid counts.
+cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const uint8_t* mask, const int32_t* seq_offsets,
+                             const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S,
+                             float clip_eps, double* partials /*[kDiagBlocks]*/, float* coef, float* loss, ais_diag* diag,
+                             cudaStream_t stream);
+
+}  // namespace ais

@@ -1,0 +1,245 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 oracle on the same seeded inputs.
+
+Tolerances (stated with the workloads): FP8 codes and scales bit-exact; log-probs 1e-2 absolute; ratios 2e-2
+relative; mixing coefficient 1e-3 absolute; hidden-state gradient 1e-2 relative Frobenius error.
+"""
+
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle import ais as oais
+from oracle import e4m3
+
+pytestmark = pytest.mark.gpu
+
+LP_ATOL = 1e-2
+RHO_RTOL = 2e-2
+ALPHA_ATOL = 1e-3
+DH_REL = 1e-2
+
+
+def _lib():
+    import paper_2605_13907_b200 as ais
+    return ais
+
+
+def _rel_fro(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
+
+
+def _run_gpu(batch, params=None, lp_old=None, ws_cap=None):
+    ais = _lib()
+    w = batch.workload
+    dev = batch.H.device
+    step = ais.AisStep(batch.T, w.d, w.V, w.P, w.G, w.block, device=dev, params=params, workspace_bytes_cap=ws_cap)
+    offs = batch.seq_offsets.to(dev)
+    rew = batch.rewards.to(dev)
+    step.step(batch.H, batch.W, batch.tokens, batch.mask, offs, rew, lp_old=lp_old)
+    torch.cuda.synchronize()
+    return step
+
+
+def _oracle(batch, params=None, lp_old=None, rows=None):
+    a = workloads.to_numpy(batch)
+    w = batch.workload
+    return a, oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, w.block,
+                             params=params, lp_old=lp_old)
+
+
+def _compare_all(batch, step, ref, a, check_grad=True):
+    T = batch.T
+    valid = a["mask"].astype(bool)
+    # FP8 codes and scales: bit-exact
+    assert np.array_equal(step.qH.cpu().numpy()[:T], ref["qH"])
+    assert np.array_equal(step.qW.cpu().numpy(), ref["qW"])
+    assert np.array_equal(step.sH.cpu().numpy()[:, :T].T.view(np.uint32), ref["sH"].view(np.uint32))
+    assert np.array_equal(step.sW.cpu().numpy()[:, :batch.W.shape[0]].T.view(np.uint32), ref["sW"].view(np.uint32))
+    lp_t = step.lp_train.cpu().numpy()[:T].astype(np.float64)
+    lp_r = step.lp_roll.cpu().numpy()[:T].astype(np.float64)
+    assert np.max(np.abs(lp_t - ref["lp_train"])) <= LP_ATOL
+    assert np.max(np.abs(lp_r - ref["lp_roll"])) <= LP_ATOL
+    assert np.max(np.abs(step.lse_train.cpu().numpy()[:T] - ref["lse_train"])) <= LP_ATOL
+    assert np.all(lp_t[~valid] == 0) and np.all(lp_r[~valid] == 0)
+    rho = step.rho.cpu().numpy()[:T].astype(np.float64)
+    assert np.max(np.abs(rho - ref["rho"]) / ref["rho"]) <= RHO_RTOL
+    assert np.all(rho[~valid] == 1)
+    d = step.read_diag()
+    assert abs(d["alpha"] - ref["diag"]["alpha"]) <= ALPHA_ATOL
+    assert d["n_valid"] == ref["diag"]["n_valid"]
+    assert np.allclose(step.adv.cpu().numpy(), ref["adv"], atol=1e-6)
+    assert int(step.status.item()) == 0 and d["status_flags"] == 0
+    if check_grad:
+        dH = step.dH.float().cpu().numpy()[:T].astype(np.float64)
+        assert _rel_fro(dH, ref["dH"]) <= DH_REL
+        assert np.all(dH[~valid] == 0)
+        assert abs(float(step.loss.item()) - ref["loss"]) <= 1e-3 * max(1.0, abs(ref["loss"]))
+    return d
+
+
+# ------------------------------------------------------------------ quantiser
+@pytest.mark.parametrize("block", [32, 64, 128])
+def test_quantize_bit_exact_adversarial(block):
+    ais = _lib()
+    g = torch.Generator().manual_seed(5)
+    rows, cols = 77, 640                                    # ragged row count, several blocks per row
+    x = torch.randn(rows, cols, generator=g) * torch.exp(torch.randn(rows, 1, generator=g) * 3)
+    x[3] = 0.0                                              # all-zero row -> scale 1, codes 0
+    x[4, :block] = 0.0
+    x[5, 7] = 3.0e38                                        # huge amax
+    x[6] = x[6] * 1e-38                                     # bf16 subnormals
+    x[7, :block] = 3.5 * torch.linspace(-1, 1, block)       # near power-of-two scale
+    x[8, 0] = -0.0
+    xb = x.to(torch.bfloat16).cuda()
+    codes, scales = ais.quantize_fp8(xb, block)
+    torch.cuda.synchronize()
+    rc, rs = e4m3.quantize_blocks(xb.float().cpu().numpy(), block)
+    assert np.array_equal(scales.cpu().numpy()[:, :rows].T.view(np.uint32), rs.view(np.uint32))
+    assert np.array_equal(codes.cpu().numpy(), rc)
+
+
+def test_quantize_every_bf16_value():
+    """All finite bf16 bit patterns, several scales: the hardware conversion agrees with the oracle's codec."""
+    ais = _lib()
+    bits = torch.arange(0, 1 << 16, dtype=torch.int32)
+    vals = (bits << 16).view(torch.float32)
+    vals = vals[torch.isfinite(vals)]
+    n = (vals.numel() // 128) * 128
+    for amax in (448.0, 1.0, 3.0e-3, 1.7e5):
+        x = vals[:n].clone().reshape(-1, 128)
+        x = torch.where(x.abs() > amax, torch.zeros_like(x), x)
+        x[:, 0] = amax                                      # fixes every block's scale
+        xb = x.to(torch.bfloat16).cuda()
+        codes, scales = ais.quantize_fp8(xb, 128)
+        torch.cuda.synchronize()
+        rc, rs = e4m3.quantize_blocks(xb.float().cpu().numpy(), 128)
+        assert np.array_equal(codes.cpu().numpy(), rc)
+        assert np.array_equal(scales.cpu().numpy()[:, :x.shape[0]].T.view(np.uint32), rs.view(np.uint32))
+
+
+# ------------------------------------------------------------------ whole path
+def test_tiny_config_full_parity():
+    batch = workloads.make_batch(workloads.WORKLOADS["tiny"], device="cpu")
+    batch = _to_cuda(batch)
+    step = _run_gpu(batch)
+    a, ref = _oracle(batch)
+    d = _compare_all(batch, step, ref, a)
+    assert 0.0 <= d["alpha"] <= 1.0
+
+
+def _to_cuda(b):
+    return workloads.Batch(b.workload, b.H.cuda(), b.W.cuda(), b.tokens.cuda(), b.mask.cuda(), b.seq_offsets, b.rewards)
+
+
+@pytest.mark.parametrize("case", ["ragged", "block32", "masked", "chunked"])
+def test_small_shapes_full_parity(case):
+    base = workloads.WORKLOADS["tiny"]
+    if case == "ragged":      # T not a multiple of 128, V not a multiple of 256, several row tiles
+        w = workloads.scaled(base, d=384, V=1336, P=3, G=4, lengths="uniform:5:90", seed=21)
+    elif case == "block32":
+        w = workloads.scaled(base, d=256, V=2048, P=2, G=4, block=32, lengths="uniform:40:120", seed=22)
+    elif case == "masked":    # LLaDA-style scattered validity, one sequence with no valid row at all
+        w = workloads.scaled(base, d=256, V=1024, P=2, G=4, lengths="const:96", mask_mode="llada", seed=23)
+    else:                     # explicit vocabulary chunks with a ragged last chunk
+        w = workloads.scaled(base, d=512, V=5000 // 8 * 8, P=2, G=2, lengths="uniform:100:300", vocab_chunk=1024, seed=24)
+    batch = workloads.make_batch(w, device="cpu")
+    if case == "masked":
+        lo, hi = int(batch.seq_offsets[2]), int(batch.seq_offsets[3])
+        batch.mask[lo:hi] = 0
+    batch = _to_cuda(batch)
+    ais = _lib()
+    params = ais.default_params(vocab_chunk=w.vocab_chunk)
+    step = _run_gpu(batch, params=params)
+    a, ref = _oracle(batch)
+    _compare_all(batch, step, ref, a)
+
+
+def test_alpha_endpoints_and_clip_on_gpu():
+    """alpha_override 0 / 1 reproduce the plain GRPO and truncated-IS gradients; lp_old != lp_train exercises the clip."""
+    ais = _lib()
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], V=768, lengths="uniform:30:70", seed=31)
+    batch = _to_cuda(workloads.make_batch(w, device="cpu"))
+    a = workloads.to_numpy(batch)
+    grads = {}
+    for alpha in (0.0, 1.0, 0.4):
+        step = _run_gpu(batch, params=ais.default_params(alpha_override=alpha))
+        _, ref = _oracle(batch, params=oais.Params(alpha_override=alpha))
+        _compare_all(batch, step, ref, a)
+        grads[alpha] = step.dH.float().cpu().numpy().astype(np.float64)
+    mix = 0.6 * grads[0.0] + 0.4 * grads[1.0]
+    assert _rel_fro(grads[0.4], mix) <= 2e-2                    # bf16 outputs: linear up to output rounding
+    # clip: shift lp_old so that rho_on leaves [0.8, 1.2] on many tokens
+    _, ref0 = _oracle(batch)
+    rng = np.random.default_rng(3)
+    lp_old = ref0["lp_train"] + 0.3 * rng.choice([-1.0, 1.0], batch.T)
+    lp_old_gpu = torch.tensor(lp_old, dtype=torch.float32, device="cuda")
+    step = _run_gpu(batch, lp_old=lp_old_gpu)
+    _, ref = _oracle(batch, lp_old=lp_old_gpu.cpu().numpy().astype(np.float64))
+    assert np.any((ref["c"] == 0) & (a["mask"] == 1))
+    _compare_all(batch, step, ref, a)
+
+
+def test_on_policy_recovery_on_gpu():
+    """Feeding the trainer's log-probs as the rollout's: rho == 1 exactly, alpha == 0 (Proposition 'on-policy recovery')."""
+    ais = _lib()
+    batch = _to_cuda(workloads.make_batch(workloads.WORKLOADS["tiny"], device="cpu"))
+    step = _run_gpu(batch)
+    offs, rew = batch.seq_offsets.cuda(), batch.rewards.cuda()
+    ais.diagnostics(step.shape, step.params, step.lp_train, step.lp_train, batch.mask, offs, rew, step.adv, step.n_valid_seq,
+                    step.rho, step.w_tilde, step.diag, step.workspace)
+    torch.cuda.synchronize()
+    d = step.read_diag()
+    assert torch.all(step.rho == 1.0) and torch.all(step.w_tilde == 1.0)
+    assert d["alpha"] == 0.0 and d["d_bar"] == 0.0 and d["alpha_ess"] == 1.0
+
+
+def test_small_workspace_chunks_rows_and_is_deterministic():
+    """The minimum workspace forces the backward pass through one 128-row chunk at a time; results do not change."""
+    ais = _lib()
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], V=1024, lengths="uniform:60:120", seed=41)
+    batch = _to_cuda(workloads.make_batch(w, device="cpu"))
+    big = _run_gpu(batch)
+    small = _run_gpu(batch, ws_cap=1)
+    again = _run_gpu(batch)
+    assert torch.equal(big.dH, small.dH)
+    assert torch.equal(big.dH, again.dH) and torch.equal(big.lp_roll, again.lp_roll)
+    assert big.read_diag() == again.read_diag()
+
+
+def test_empty_batch_and_bad_tokens_flags():
+    ais = _lib()
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], V=512, lengths="const:32", seed=51)
+    batch = _to_cuda(workloads.make_batch(w, device="cpu"))
+    batch.mask.zero_()
+    step = _run_gpu(batch)
+    d = step.read_diag()
+    assert d["status_flags"] & ais.FLAG_EMPTY and d["alpha"] == 0.0 and float(step.loss.item()) == 0.0
+    assert torch.all(step.dH == 0) and torch.all(step.lp_train == 0)
+    batch.mask.fill_(1)
+    batch.tokens[5] = w.V + 3
+    batch.tokens[9] = -1
+    step = _run_gpu(batch)
+    assert int(step.status.item()) & ais.FLAG_TOKEN_RANGE
+    assert float(step.lp_train[5]) == 0.0 and float(step.lp_roll[9]) == 0.0
+
+
+def test_host_side_argument_errors():
+    ais = _lib()
+    batch = _to_cuda(workloads.make_batch(workloads.scaled(workloads.WORKLOADS["tiny"], V=512, lengths="const:32"), device="cpu"))
+    step = ais.AisStep(batch.T, 256, 512, 2, 4, 128)
+    with pytest.raises(ais.AisError):
+        ais.logprob_fwd(step.shape, step.params, batch.H, batch.W, step.qH, step.sH, step.qW, step.sW, None, batch.mask,
+                        step.lp_train, step.lse_train, step.lp_roll, step.lse_roll, step.status, step.workspace)
+    with pytest.raises(ais.AisError):                        # workspace too small
+        ais.loss_bwd(step.shape, step.params, batch.H, batch.W, batch.tokens, batch.mask, batch.seq_offsets.cuda(),
+                     step.lse_train, step.lp_train, None, step.adv, step.w_tilde, step.dH, step.loss, step.diag, step.status,
+                     step.workspace[:256])
+    bad = ais.binding.make_shape(batch.T, 200, 512, 2, 4, 128)   # d not a multiple of 128
+    with pytest.raises(ais.AisError):
+        ais.diagnostics(bad, step.params, step.lp_train, step.lp_roll, batch.mask, batch.seq_offsets.cuda(),
+                        batch.rewards.cuda(), step.adv, step.n_valid_seq, step.rho, step.w_tilde, step.diag, step.workspace)
+    with pytest.raises(ais.AisError):
+        ais.quantize_fp8(batch.H.cpu(), 128)
