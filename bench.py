@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the AIS-GRPO LM-head path on B200.
+
+One step = one pass of the whole path over one synthetic batch: FP8 quantisation of H and W, trainer (bf16)
+and rollout (FP8) log-probabilities, diagnostics / alpha / rectification weights, loss and dH.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload qwen3_8b] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is valid tokens per second over all ranks with inputs resident in HBM;
+`e2e` is the same through host buffers (pinned host -> device copies of the step's inputs and a device -> host
+read of loss, diagnostics and dH inside the timed region).  `--impl reference` times the float64 CPU oracle
+on a bounded sample instead.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "AIS-corrected fwd+bwd tokens/sec"
+UNIT = "tokens/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"], bf16_tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle sample
+def oracle_sample(w: workloads.Workload, tokens_n: int = 192, vocab_n: int = 8192):
+    """Times the oracle, as it stands, on `tokens_n` rows against `vocab_n` vocabulary rows of the workload's
+    shape and scales the rate to the full vocabulary (every stage of the path costs O(V) per token)."""
+    from oracle import ais as oais
+    vocab_n = min(vocab_n, w.V)
+    rng = np.random.default_rng(w.seed)
+    G, P = w.G, 1
+    S = P * G
+    per = max(1, tokens_n // S)
+    T = per * S
+    H = torch.randn(T, w.d, generator=torch.Generator().manual_seed(w.seed))
+    if w.rmsnorm:
+        H = H * torch.rsqrt(H.pow(2).mean(dim=1, keepdim=True) + 1e-6)
+    H = H.to(torch.bfloat16).float().numpy().astype(np.float64)
+    W = (torch.randn(vocab_n, w.d, generator=torch.Generator().manual_seed(w.seed + 1)) * w.w_std)
+    W = W.to(torch.bfloat16).float().numpy()
+    tokens = rng.integers(0, vocab_n, T)
+    mask = np.ones(T, np.uint8)
+    offs = np.arange(S + 1) * per
+    rewards = (rng.random(S) < w.reward_p).astype(np.float64)
+    t0 = time.perf_counter()
+    oais.full_path(H, W, tokens, mask, offs, rewards, P, G, w.block)
+    dt = time.perf_counter() - t0
+    rate = T / dt * (vocab_n / w.V)
+    return rate, dt, f"{T} tokens x d={w.d} x {vocab_n} of V={w.V} vocabulary rows, rate scaled by {vocab_n}/{w.V}"
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+
+
+def _ld_u(V: int) -> int:
+    return (V + 63) // 64 * 64
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def run_ours(args) -> None:
+    import torch.distributed as dist
+    import paper_2605_13907_b200 as ais
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    base = workloads.WORKLOADS[args.workload]
+    w = workloads.scaled(base, seed=base.seed + 7919 * rank)          # every rank owns its own prompts (weak scaling)
+    batch = workloads.make_batch(w, device=dev)
+    T, n_valid = batch.T, batch.n_valid
+    params = ais.default_params(vocab_chunk=w.vocab_chunk)
+    step = ais.AisStep(T, w.d, w.V, w.P, w.G, w.block, device=dev, params=params, workspace_bytes_cap=args.workspace_gb << 30)
+    offs = batch.seq_offsets.to(dev)
+    rew = batch.rewards.to(dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def one_step(ev=None):
+        marks = []
+
+        def mark():
+            if ev is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record(stream)
+                marks.append(e)
+        mark()
+        ais.quantize_fp8(batch.H, w.block, step.qH, step.sH)
+        ais.quantize_fp8(batch.W, w.block, step.qW, step.sW)
+        mark()
+        ais.logprob_fwd(step.shape, step.params, batch.H, batch.W, None, None, None, None, batch.tokens, batch.mask,
+                        step.lp_train, step.lse_train, None, None, step.status, step.workspace)
+        mark()
+        ais.logprob_fwd(step.shape, step.params, None, None, step.qH, step.sH, step.qW, step.sW, batch.tokens, batch.mask,
+                        None, None, step.lp_roll, step.lse_roll, step.status, step.workspace)
+        mark()
+        step.diagnose(batch.mask, offs, rew)
+        mark()
+        step.backward(batch.H, batch.W, batch.tokens, batch.mask, offs)
+        mark()
+        if ev is not None:
+            ev.append(marks)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    events = []
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for _ in range(args.steps):
+        one_step(events)
+    t_end.record(stream)
+    barrier()
+    total_ms = t_start.elapsed_time(t_end)
+    clocks = sampler.stop() if sampler else None
+    status = int(step.status.item())
+    if status != 0:
+        raise RuntimeError(f"device status word {status}")
+    diag = step.read_diag()
+
+    names = ["quantize", "fwd_train_bf16", "fwd_roll_fp8", "diagnostics", "loss_bwd"]
+    seg = {n: 0.0 for n in names}
+    for marks in events:
+        for i, n in enumerate(names):
+            seg[n] += marks[i].elapsed_time(marks[i + 1])
+    seg = {n: v / args.steps for n, v in seg.items()}
+
+    # ---- end to end through host buffers
+    pin = dict(H=batch.H.cpu().pin_memory(), tokens=batch.tokens.cpu().pin_memory(), mask=batch.mask.cpu().pin_memory(),
+               offs=batch.seq_offsets.pin_memory(), rew=batch.rewards.pin_memory())
+    dH_host = torch.empty(step.dH.shape, dtype=step.dH.dtype).pin_memory()
+    small_host = torch.empty(step.diag.numel() + 1, dtype=torch.float64).pin_memory()
+    H2 = torch.empty_like(batch.H)
+    tok2, msk2 = torch.empty_like(batch.tokens), torch.empty_like(batch.mask)
+    offs2, rew2 = torch.empty_like(offs), torch.empty_like(rew)
+    h2d = sum(t.numel() * t.element_size() for t in pin.values())
+    d2h = dH_host.numel() * dH_host.element_size() + small_host.numel() * 8
+
+    def e2e_step():
+        H2.copy_(pin["H"], non_blocking=True)
+        tok2.copy_(pin["tokens"], non_blocking=True)
+        msk2.copy_(pin["mask"], non_blocking=True)
+        offs2.copy_(pin["offs"], non_blocking=True)
+        rew2.copy_(pin["rew"], non_blocking=True)
+        step.step(H2, batch.W, tok2, msk2, offs2, rew2)
+        dH_host.copy_(step.dH, non_blocking=True)
+        small_host[:-1].copy_(step.diag, non_blocking=True)
+        small_host[-1:].copy_(step.loss.double(), non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    ms_per_step = total_ms / args.steps
+    stats = torch.tensor([ms_per_step, e2e_ms, float(n_valid)], dtype=torch.float64, device=dev)
+    if world > 1:
+        mx = stats.clone()
+        dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = stats.clone()
+        dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        ms_per_step, e2e_ms, tokens_all = float(mx[0]), float(mx[1]), float(sm[2])
+    else:
+        tokens_all = float(n_valid)
+
+    if rank == 0:
+        peaks = _peaks()
+        flops_pass = 2.0 * T * w.d * w.V                      # algorithmic FLOPs of one T x d x V contraction
+        t_dom = seg["fwd_train_bf16"] * 1e-3
+        achieved = flops_pass / t_dom / 1e12
+        peak = peaks["bf16_tflops_sustained"]
+        fixed = ais.workspace_min_bytes(step.shape, step.params) - 128 * _ld_u(w.V) * 2
+        blk_rows = (step.workspace.numel() - fixed) // (_ld_u(w.V) * 2) // 128 * 128
+        blk_rows = max(128, min(blk_rows, (T + 127) // 128 * 128))
+        chunks = -(-T // blk_rows)
+        launches = 2 + 2 + 2 + 4 + 3 + 2 * chunks
+        out = {
+            "metric": METRIC, "value": tokens_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16+fp8_e4m3", "data": "synthetic",
+            "config": {"workload": f"{w.name}: d={w.d} V={w.V} P={w.P} G={w.G} block={w.block} lengths={w.lengths}",
+                       "rows": T, "valid_tokens_per_gpu": n_valid,
+                       "l2": "inputs larger than L2 (H %.2f GB, W %.2f GB)" % (T * w.d * 2 / 1e9, w.V * w.d * 2 / 1e9),
+                       "parallelism": f"dp{world} (independent batches per GPU)", "bwd_row_chunks": chunks,
+                       "alpha": diag["alpha"], "d_bar": diag["d_bar"]},
+            "segments_ms": seg,
+            "roofline": {"bound": "tensor", "kernel": "lmhead_kernel<bf16 forward> (trainer log-probs)", "achieved": achieved,
+                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "peak_source": peaks["source"] + " bf16 sustained (kernel timed inside a long step)",
+                         "passes": {"fwd_roll_fp8_tflops": flops_pass / (seg["fwd_roll_fp8"] * 1e-3) / 1e12,
+                                    "bwd_two_passes_tflops": 2 * flops_pass / (seg["loss_bwd"] * 1e-3) / 1e12,
+                                    "quantize_gbs": (T + w.V) * w.d * 3.03 / (seg["quantize"] * 1e-3) / 1e9}},
+            "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches * args.steps,
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            rate, dt, sample = oracle_sample(w)
+            out["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": sample,
+                                   "seconds": dt}
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------ reference arm (CPU oracle)
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    w = workloads.WORKLOADS[args.workload]
+    steps, warm = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    for _ in range(warm):
+        oracle_sample(w, tokens_n=64, vocab_n=2048)
+    rates, secs, sample = [], [], ""
+    for _ in range(steps):
+        r, dt, sample = oracle_sample(w)
+        rates.append(r)
+        secs.append(dt)
+    value = len(rates) / sum(1.0 / r for r in rates)
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+           "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{w.name}: d={w.d} V={w.V} P={w.P} G={w.G} block={w.block} lengths={w.lengths}"},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out), flush=True)
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="qwen3_8b", choices=sorted(workloads.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workspace-gb", type=int, default=48)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        args.warmup = max(args.warmup, 3)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -104,6 +104,11 @@ def quantize_blocks(x, block: int):
     R, K = x32.shape
     if K % block:
         raise ValueError("block must divide the last dimension")
+    slab = max(1, (1 << 22) // max(K, 1))
+    if R > slab:
+        # rows are independent: walk the matrix in row slabs only to keep the integer temporaries small
+        parts = [quantize_blocks(x32[r0:r0 + slab], block) for r0 in range(0, R, slab)]
+        return np.concatenate([p[0] for p in parts], axis=0), np.concatenate([p[1] for p in parts], axis=0)
     xb = x32.reshape(R, K // block, block)
     amax = np.max(np.abs(xb), axis=2).astype(np.float32)
     scales = (amax / np.float32(E4M3_MAX)).astype(np.float32)

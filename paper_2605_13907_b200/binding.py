@@ -179,10 +179,14 @@ class AisStep:
         dev = self.device
         nkb = d // fp8_block
         ws = workspace_bytes(self.shape, self.params)
-        if workspace_bytes_cap is not None:
-            ws = max(workspace_min_bytes(self.shape, self.params), min(ws, workspace_bytes_cap))
         if ws == 0:
             raise AisError("invalid shape or parameters")
+        if workspace_bytes_cap is not None:
+            # room for every row's backward scratch in one pass, limited by the cap, never below the minimum
+            ws_min = workspace_min_bytes(self.shape, self.params)
+            ld_u = (V + 63) // 64 * 64
+            ws_all = ws_min + max(0, (T + 127) // 128 * 128 - 128) * ld_u * 2
+            ws = max(ws_min, min(ws_all, workspace_bytes_cap))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
         self.qH = torch.empty(max(T, 1), d, dtype=torch.uint8, device=dev)
         self.sH = torch.empty(nkb, max((T + 3) // 4 * 4, 4), dtype=torch.float32, device=dev)
