@@ -190,6 +190,35 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params,
                  void* dH, float* loss, ais_diag* diag,
                  uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Trainer log-probabilities for callers that cannot hand over a workspace (the paper has no counterpart;
+ * this is a packaging variant of the trainer pass of ais_logprob_fwd, same kernels, same results).
+ *
+ * Who needs it: code that runs where device memory cannot be obtained at call time - a plug-in or
+ * callback that receives only its input and output buffers, a process whose HBM has been handed in
+ * full to another pool (a serving engine's KV cache, a training framework's caching allocator), or a
+ * latency-critical loop that must avoid cudaMalloc because it stalls the whole device.  Such a caller
+ * has nowhere to get the workspace that ais_logprob_fwd asks for.
+ *
+ * The partial (max, sum-exp, target-logit) triples of the vocabulary ranges are kept in a fixed array of
+ * 3 x 8 x AIS_STATIC_MAX_ROWS floats (1.5 MiB) that is part of the library image; every GPU on which
+ * the library is loaded holds it until the process exits.  The call allocates and frees nothing.
+ *   - T must not exceed AIS_STATIC_MAX_ROWS; a larger T returns AIS_ERR_LIMIT and enqueues nothing.
+ *   - shape->d must be a multiple of 64 and V of 8; P, G and fp8_block are not read.  The vocabulary
+ *     is always streamed in 4 ranges.
+ *   - The first call on each device resolves the array's device address and prepares the kernels; make
+ *     that first call with the device current and before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps what the last call left in it.  Each call
+ *     overwrites every slot it later reads, so nothing has to be cleared; but two calls that overlap on
+ *     the GPU (different streams, no ordering between them) race on it and give undefined results.
+ * Inputs and outputs as in ais_logprob_fwd: H [T, ldh] bf16, W [V, ldw] bf16, tokens [T], mask [T],
+ * lp_train [T] (written), lse_train [T] (written, may be NULL), dev_status (OR-ed into, may be NULL).
+ */
+#define AIS_STATIC_MAX_ROWS 16384
+int ais_logprob_train_static(const ais_shape* shape, const void* H, const void* W, const int32_t* tokens,
+                             const uint8_t* mask, float* lp_train, float* lse_train, uint32_t* dev_status,
+                             void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -70,6 +70,8 @@ def lib() -> C.CDLL:
         L.ais_diagnostics.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.ais_loss_bwd.restype = C.c_int
         L.ais_loss_bwd.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 14 + [vp, sz, vp]
+        L.ais_logprob_train_static.restype = C.c_int
+        L.ais_logprob_train_static.argtypes = [C.POINTER(Shape)] + [vp] * 8
         _lib = L
     return _lib
 
@@ -155,6 +157,17 @@ def loss_bwd(shape: Shape, params: Params, H, W, tokens, mask, seq_offsets, lse_
                               _ptr(lse_train), _ptr(lp_train), _ptr(lp_old), _ptr(adv), _ptr(w_tilde), _ptr(dH), _ptr(loss),
                               _ptr(diag), _ptr(dev_status), _ptr(workspace), workspace.numel() * workspace.element_size(),
                               _stream(workspace)), "ais_loss_bwd")
+
+
+def logprob_train_static(shape: Shape, H, W, tokens, mask, lp_train, lse_train=None, dev_status=None):
+    """Trainer log-probs with the library's built-in scratch: no workspace argument and no allocation, for
+    callers that only own their inputs and outputs.  At most STATIC_MAX_ROWS rows; calls must not overlap."""
+    _require_cuda(H, W, tokens, mask, lp_train, lse_train, dev_status)
+    _check(lib().ais_logprob_train_static(C.byref(shape), _ptr(H), _ptr(W), _ptr(tokens), _ptr(mask), _ptr(lp_train),
+                                          _ptr(lse_train), _ptr(dev_status), _stream(H)), "ais_logprob_train_static")
+
+
+STATIC_MAX_ROWS = 16384
 
 
 def read_diag(diag_buf: torch.Tensor) -> dict:
