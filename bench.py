@@ -45,7 +45,7 @@ def _peaks():
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle sample
-def oracle_sample(w: workloads.Workload, tokens_n: int = 192, vocab_n: int = 8192):
+def oracle_sample(w: workloads.Workload, tokens_n: int = 192, vocab_n: int = 32768):
     """Times the oracle, as it stands, on `tokens_n` rows against `vocab_n` vocabulary rows of the workload's
     shape and scales the rate to the full vocabulary (every stage of the path costs O(V) per token)."""
     from oracle import ais as oais
@@ -138,6 +138,8 @@ def run_ours(args) -> None:
 
     base = workloads.WORKLOADS[args.workload]
     w = workloads.scaled(base, seed=base.seed + 7919 * rank)          # every rank owns its own prompts (weak scaling)
+    if args.prompts:
+        w = workloads.scaled(w, P=args.prompts)                       # reduced case for profiler captures
     batch = workloads.make_batch(w, device=dev)
     T, n_valid = batch.T, batch.n_valid
     params = ais.default_params(vocab_chunk=w.vocab_chunk)
@@ -321,6 +323,7 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workspace-gb", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (small profiling case)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

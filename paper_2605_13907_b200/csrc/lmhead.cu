@@ -1,9 +1,10 @@
 // LM-head tensor-core passes for sm_100a: TMA-fed tcgen05.mma with accumulators in tensor memory and
 // fused epilogues (streaming log-sum-exp + target pick, softmax-minus-onehot scratch, dH scaling).
 //
-// One persistent CTA per SM.  Warp 0 issues TMA tile loads, warp 1 issues the MMAs, warps 2..9 are the
-// epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (one row per thread) and column half (w-2)/4 of the
-// 256-column accumulator.  Two 256-column accumulators alternate so that the epilogue of one tile (or,
+// One persistent CTA of three warpgroups per SM.  Warp 0 issues TMA tile loads, warp 1 issues the MMAs
+// (warps 2, 3 idle), warps 4..11 are the epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (one row per
+// thread) and column half (w-4)/4 of the 256-column accumulator.  In the FP8 pass the first warpgroup gives
+// registers to the two epilogue warpgroups, which keep 128 fp32 accumulators per thread.  Two 256-column accumulators alternate so that the epilogue of one tile (or,
 // in the FP8 pass, the promotion of one scale block) overlaps the MMAs of the next.
 #include "lmhead.cuh"
 #include "ptx.cuh"
@@ -37,6 +38,40 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Packed pairs of fp32 in one 64-bit register and the two-wide arithmetic of sm_100 on them.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+template <int N>
+__device__ __forceinline__ void reg_alloc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void reg_dealloc() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -109,6 +144,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+
+    // FP8 pass: 384 threads x 168 registers at launch = 128 x 56 + 256 x 224 after the split below.
+    if (warp < 4) {
+    if (MODE == kFwdFp8) reg_dealloc<56>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -213,10 +252,12 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             // everything issued has to finish before the tensor memory is given back
             tc_commit(done);
         }
+    }
     } else {
         // ------------------------------------------------------------------ epilogue warps
+        if (MODE == kFwdFp8) reg_alloc<224>();
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;             // column half of the accumulator
+        const int half = (warp - 4) >> 2;             // column half of the accumulator
         const int r_in_tile = q * 32 + lane;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
         Pipe tb(2), sc(kScaleSlots);
@@ -241,10 +282,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
             for (int t = w.t0; t < w.t1 && ok; ++t) {
                 const int col_base = t * kBN + half * 128;    // first output column of this thread's half
-                float acc[128];
+                uint64_t acc2[64];                             // FP8 pass: 128 fp32 accumulators as packed pairs
                 if (MODE == kFwdFp8) {
 #pragma unroll
-                    for (int i = 0; i < 128; ++i) acc[i] = 0.f;
+                    for (int i = 0; i < 64; ++i) acc2[i] = 0ull;
                     for (int ks = 0; ks < a.ksteps && ok; ++ks) {
                         if (!mbar_wait_warp(&sfull[sc.idx], sc.phase, abort_flag)) { ok = false; break; }
                         const float* sS = reinterpret_cast<const float*>(scale_base + sc.idx * kScaleSlotBytes);
@@ -252,25 +293,28 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
                             tc_fence_after();
                             const float sh = sS[g * kBM + r_in_tile];
-                            const float4* sw4 = reinterpret_cast<const float4*>(sS + (kScaleBOffset / 4) + g * kBN + half * 128);
+                            const uint64_t sh2 = pack2(sh, sh);
+                            const ulonglong2* sw2 = reinterpret_cast<const ulonglong2*>(sS + (kScaleBOffset / 4) + g * kBN + half * 128);
                             const uint32_t taddr = tmem_base + lane_addr + tb.idx * kBN + half * 128;
 #pragma unroll
                             for (int c = 0; c < 4; ++c) {
                                 uint32_t v[32];
                                 tmem_ld32(taddr + c * 32, v);
                                 tmem_ld_wait();
+                                if (c == 3) {
+                                    // the partial sums are in registers: hand the buffer back before the arithmetic
+                                    tc_fence_before();
+                                    __syncwarp();
+                                    if (lane == 0) mbar_arrive(&tempty[tb.idx]);
+                                }
 #pragma unroll
                                 for (int i = 0; i < 32; i += 4) {
-                                    const float4 sw = sw4[(c * 32 + i) >> 2];
-                                    acc[c * 32 + i + 0] = fmaf(sh * sw.x, __uint_as_float(v[i + 0]), acc[c * 32 + i + 0]);
-                                    acc[c * 32 + i + 1] = fmaf(sh * sw.y, __uint_as_float(v[i + 1]), acc[c * 32 + i + 1]);
-                                    acc[c * 32 + i + 2] = fmaf(sh * sw.z, __uint_as_float(v[i + 2]), acc[c * 32 + i + 2]);
-                                    acc[c * 32 + i + 3] = fmaf(sh * sw.w, __uint_as_float(v[i + 3]), acc[c * 32 + i + 3]);
+                                    const ulonglong2 sw = sw2[(c * 32 + i) >> 2];      // scales of 4 columns, two packed pairs
+                                    const int j = (c * 32 + i) >> 1;
+                                    acc2[j] = fma2(mul2(sh2, sw.x), pack2u(v[i], v[i + 1]), acc2[j]);
+                                    acc2[j + 1] = fma2(mul2(sh2, sw.y), pack2u(v[i + 2], v[i + 3]), acc2[j + 1]);
                                 }
                             }
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(&tempty[tb.idx]);
                             tb.advance();
                         }
                         __syncwarp();
@@ -290,7 +334,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     float x[32];
                     if (MODE == kFwdFp8) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) x[i] = acc[c * 32 + i];
+                        for (int i = 0; i < 32; i += 2) unpack2(acc2[(c * 32 + i) >> 1], x[i], x[i + 1]);
                     } else {
                         uint32_t v[32];
                         tmem_ld32(taddr + c * 32, v);

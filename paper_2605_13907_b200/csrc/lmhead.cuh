@@ -25,7 +25,7 @@ constexpr int kScaleSlots = 4;
 constexpr int kScaleSlotBytes = 4 * (kBM + kBN) * 4;   // up to 4 scale blocks per stage
 constexpr int kScaleBOffset = 4 * kBM * 4;
 constexpr int kNumBarriers = 2 * kStages + 4 + 2 * kScaleSlots + 1;
-constexpr int kThreads = 320;            // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int kThreads = 384;            // warp 0 TMA, warp 1 MMA, warps 2..3 idle, warps 4..11 epilogue
 constexpr int kEpiWarps = 8;
 constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kScaleSlots * kScaleSlotBytes + kNumBarriers * 8 + 64;
 

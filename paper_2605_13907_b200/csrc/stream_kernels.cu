@@ -65,8 +65,24 @@ __global__ void __launch_bounds__(kQThreads) quantize_kernel(const __nv_bfloat16
             const float s = (amax == 0.f) ? 1.0f : __fdiv_rn(amax, 448.0f);
             if (col < cols) {
                 float qv[8];
+                if (s > 0x1p-100f && s < 0x1p100f) {
+                    // Correctly rounded x / s from the correctly rounded reciprocal y = RN(1/s): two residual
+                    // corrections with fused multiply-adds; the first makes the quotient faithful, and a faithful
+                    // quotient corrected once more with the exact residual is the round-to-nearest quotient
+                    // (Markstein's division theorem).  |x / s| <= 448 here, so nothing overflows; a quotient that
+                    // underflows encodes to zero either way; the sign of x is restored explicitly.
+                    const float y = __frcp_rn(s);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) qv[i] = __fdiv_rn(v[i], s);
+                    for (int i = 0; i < 8; ++i) {
+                        float q = v[i] * y;
+                        q = __fmaf_rn(__fmaf_rn(-s, q, v[i]), y, q);
+                        q = __fmaf_rn(__fmaf_rn(-s, q, v[i]), y, q);
+                        qv[i] = copysignf(q, v[i]);          // a zero residual sum would turn -0 into +0
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) qv[i] = __fdiv_rn(v[i], s);
+                }
                 uint2 out;
                 out.x = static_cast<uint32_t>(cvt_e4m3x2(qv[1], qv[0])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[3], qv[2])) << 16);
                 out.y = static_cast<uint32_t>(cvt_e4m3x2(qv[5], qv[4])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[7], qv[6])) << 16);

@@ -120,6 +120,27 @@ def test_quantize_every_bf16_value():
         assert np.array_equal(scales.cpu().numpy()[:, :x.shape[0]].T.view(np.uint32), rs.view(np.uint32))
 
 
+def test_quantize_every_bf16_value_random_scales():
+    """Every finite bf16 value against 60 block scales spread over 60 decades (the quotient x / s must be the
+    correctly rounded one for the code to match, whatever the scale's mantissa)."""
+    ais = _lib()
+    bits = torch.arange(0, 1 << 16, dtype=torch.int32)
+    vals = (bits << 16).view(torch.float32)
+    vals = vals[torch.isfinite(vals)]
+    n = (vals.numel() // 127) * 127
+    rng = np.random.default_rng(0)
+    for _ in range(60):
+        amax = float(torch.tensor(np.exp(rng.uniform(np.log(1e-30), np.log(1e30))), dtype=torch.float32).to(torch.bfloat16))
+        x = vals[:n].clone().reshape(-1, 127)
+        x = torch.where(x.abs() > amax, torch.full_like(x, amax * 0.5), x)
+        x = torch.cat([torch.full((x.shape[0], 1), amax), x], dim=1).to(torch.bfloat16).cuda()
+        codes, scales = ais.quantize_fp8(x, 128)
+        torch.cuda.synchronize()
+        rc, rs = e4m3.quantize_blocks(x.float().cpu().numpy(), 128)
+        assert np.array_equal(codes.cpu().numpy(), rc)
+        assert np.array_equal(scales.cpu().numpy()[:, :x.shape[0]].T.view(np.uint32), rs.view(np.uint32))
+
+
 # ------------------------------------------------------------------ whole path
 def test_tiny_config_full_parity():
     batch = workloads.make_batch(workloads.WORKLOADS["tiny"], device="cpu")
