@@ -1,0 +1,48 @@
+"""The built library loads without a GPU and exports every entry point that include/ais.h declares (CPU only)."""
+
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "ais.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ais_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_path():
+    names = _declared()
+    for must in ("ais_quantize_fp8", "ais_logprob_fwd", "ais_diagnostics", "ais_loss_bwd", "ais_workspace_bytes"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2605_13907_b200 import build
+    lib_path = build.build_library()
+    lib = ctypes.CDLL(lib_path)
+    for name in _declared():
+        assert hasattr(lib, name), name
+    lib.ais_version.restype = ctypes.c_int
+    assert lib.ais_version() >= 100
+    lib.ais_strerror.restype = ctypes.c_char_p
+    assert b"workspace" in lib.ais_strerror(-4)
+
+
+def test_host_side_validation_needs_no_gpu():
+    import paper_2605_13907_b200 as ais
+    p = ais.default_params()
+    assert p.C == 5.0 and abs(p.delta - 0.02) < 1e-7 and abs(p.gamma - 1.2) < 1e-6 and p.alpha_override != p.alpha_override
+    good = ais.binding.make_shape(1000, 4096, 151936, 8, 8, 128)
+    assert ais.workspace_bytes(good, p) >= ais.workspace_min_bytes(good, p) > 0
+    bad = ais.binding.make_shape(1000, 4100, 151936, 8, 8, 128)        # d not a multiple of 128
+    assert ais.workspace_bytes(bad, p) == 0
+    p.C = 0.5                                                           # truncation below 1 is rejected
+    assert ais.workspace_bytes(good, p) == 0
+    import torch
+    with pytest.raises(ais.AisError):                                   # CPU tensors are refused: no CPU path
+        ais.quantize_fp8(torch.zeros(4, 128, dtype=torch.bfloat16), 128)
