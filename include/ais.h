@@ -65,7 +65,7 @@ typedef struct ais_shape {
     int32_t P;            /* prompts in the batch                                            */
     int32_t G;            /* responses per prompt; sequence s belongs to prompt s / G        */
     int32_t fp8_block;    /* elements along d sharing one FP8 scale: 32, 64 or 128           */
-    int32_t reserved;
+    int32_t P_total;      /* prompts over all data-parallel ranks (loss normaliser); 0 = P    */
     int64_t ldh;          /* row stride of H (and of its codes) in elements                  */
     int64_t ldw;          /* row stride of W (and of its codes) in elements                  */
 } ais_shape;
@@ -173,11 +173,32 @@ int ais_diagnostics(const ais_shape* shape, const ais_params* params,
                     void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same step in two halves, for data-parallel use (each rank holds whole prompts; alpha is one number
+ * per global batch, Eq. alpha-final).  ais_diag_moments writes adv, n_valid_seq and this rank's AIS_NUM_MOMENTS
+ * masked sums (double, on the device):
+ *   0 N   1 sum w_bar   2 sum w_bar^2   3 sum |lp_train - lp_roll|   4 sum A   5 sum A^2   6 sum A w_bar
+ *   7 sum (A w_bar)^2   8 sum (lp_roll - lp_train)   9 sum |exp(lp_train) - exp(lp_roll)|   10, 11 unused (zero)
+ * The caller sums the vectors of all ranks (one all-reduce of 12 doubles) and hands the result to
+ * ais_diag_finalize, which derives the diagnostics, alpha, rho and w_tilde from it.  With one rank the two
+ * calls give bit-identical results to ais_diagnostics.
+ */
+#define AIS_NUM_MOMENTS 12
+int ais_diag_moments(const ais_shape* shape, const ais_params* params,
+                     const float* lp_train, const float* lp_roll, const uint8_t* mask,
+                     const int32_t* seq_offsets, const float* rewards,
+                     float* adv, int32_t* n_valid_seq, double* moments,
+                     void* workspace, size_t workspace_bytes, void* stream);
+int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const double* moments,
+                      const float* lp_train, const float* lp_roll, const uint8_t* mask,
+                      float* rho, float* w_tilde, ais_diag* diag, void* stream);
+
+/*
  * AIS-GRPO surrogate loss and its gradient with respect to H (Eq. ais-grpo without the KL term;
  * the objective is maximised, so loss = -J).  With rho_on = exp(lp_train - lp_old)
  * (lp_old == NULL means rho_on = 1) and n_s the valid rows of sequence s:
  *     loss  = - sum_s 1/(P G n_s) sum_{t in s, mask} w_tilde[t] min(rho_on A_s, clip(rho_on, 1 +- clip_eps) A_s)
  *     c_t   = mask[t] w_tilde[t] A_s rho_on [unclipped branch active] / (P G n_s)
+ * (P is shape->P_total when that is set, so that the losses of all data-parallel ranks add up to the global one)
  *     dH[t,:] = c_t (softmax(z[t,:]) - onehot(tokens[t])) W
  * The softmax is recomputed from H, W and lse_train; w_tilde, A and lp_old are constants.
  * dH [T, ldh] bf16 (written, zero rows where mask = 0), loss: one float on the device (may be NULL),

@@ -13,6 +13,7 @@ _LIB_PATH = os.path.join(_HERE, "libais_b200.so")
 _lib = None
 
 FLAG_EMPTY, FLAG_TOKEN_RANGE, FLAG_NONFINITE, FLAG_TIMEOUT = 1, 2, 4, 8
+NUM_MOMENTS = 12
 
 
 class AisError(RuntimeError):
@@ -21,7 +22,7 @@ class AisError(RuntimeError):
 
 class Shape(C.Structure):
     _fields_ = [("T", C.c_int64), ("d", C.c_int32), ("V", C.c_int32), ("P", C.c_int32), ("G", C.c_int32),
-                ("fp8_block", C.c_int32), ("reserved", C.c_int32), ("ldh", C.c_int64), ("ldw", C.c_int64)]
+                ("fp8_block", C.c_int32), ("P_total", C.c_int32), ("ldh", C.c_int64), ("ldw", C.c_int64)]
 
 
 class Params(C.Structure):
@@ -70,6 +71,10 @@ def lib() -> C.CDLL:
         L.ais_diagnostics.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.ais_loss_bwd.restype = C.c_int
         L.ais_loss_bwd.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 14 + [vp, sz, vp]
+        L.ais_diag_moments.restype = C.c_int
+        L.ais_diag_moments.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 8 + [vp, sz, vp]
+        L.ais_diag_finalize.restype = C.c_int
+        L.ais_diag_finalize.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 8
         L.ais_logprob_train_static.restype = C.c_int
         L.ais_logprob_train_static.argtypes = [C.POINTER(Shape)] + [vp] * 8
         _lib = L
@@ -99,8 +104,9 @@ def default_params(**overrides) -> Params:
     return p
 
 
-def make_shape(T: int, d: int, V: int, P: int, G: int, fp8_block: int, ldh: int | None = None, ldw: int | None = None) -> Shape:
-    return Shape(T=T, d=d, V=V, P=P, G=G, fp8_block=fp8_block, reserved=0, ldh=ldh or d, ldw=ldw or d)
+def make_shape(T: int, d: int, V: int, P: int, G: int, fp8_block: int, ldh: int | None = None, ldw: int | None = None,
+               P_total: int = 0) -> Shape:
+    return Shape(T=T, d=d, V=V, P=P, G=G, fp8_block=fp8_block, P_total=P_total, ldh=ldh or d, ldw=ldw or d)
 
 
 def workspace_bytes(shape: Shape, params: Params) -> int:
@@ -150,6 +156,19 @@ def diagnostics(shape: Shape, params: Params, lp_train, lp_roll, mask, seq_offse
            "ais_diagnostics")
 
 
+def diag_moments(shape: Shape, params: Params, lp_train, lp_roll, mask, seq_offsets, rewards, adv, n_valid_seq, moments, workspace):
+    _require_cuda(lp_train, lp_roll, mask, seq_offsets, rewards, adv, n_valid_seq, moments, workspace)
+    _check(lib().ais_diag_moments(C.byref(shape), C.byref(params), _ptr(lp_train), _ptr(lp_roll), _ptr(mask), _ptr(seq_offsets),
+                                  _ptr(rewards), _ptr(adv), _ptr(n_valid_seq), _ptr(moments), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream(workspace)), "ais_diag_moments")
+
+
+def diag_finalize(shape: Shape, params: Params, moments, lp_train, lp_roll, mask, rho, w_tilde, diag):
+    _require_cuda(moments, lp_train, lp_roll, mask, rho, w_tilde, diag)
+    _check(lib().ais_diag_finalize(C.byref(shape), C.byref(params), _ptr(moments), _ptr(lp_train), _ptr(lp_roll), _ptr(mask),
+                                   _ptr(rho), _ptr(w_tilde), _ptr(diag), _stream(moments)), "ais_diag_finalize")
+
+
 def loss_bwd(shape: Shape, params: Params, H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, adv, w_tilde, dH, loss,
              diag, dev_status, workspace):
     _require_cuda(H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, adv, w_tilde, dH, loss, diag, dev_status, workspace)
@@ -184,9 +203,10 @@ class AisStep:
     """
 
     def __init__(self, T: int, d: int, V: int, P: int, G: int, fp8_block: int, device="cuda", params: Params | None = None,
-                 workspace_bytes_cap: int | None = None, want_grad: bool = True):
+                 workspace_bytes_cap: int | None = None, want_grad: bool = True, group=None, P_total: int = 0):
         self.device = torch.device(device)
-        self.shape = make_shape(T, d, V, P, G, fp8_block)
+        self.group = group                       # torch.distributed process group: alpha over all its ranks
+        self.shape = make_shape(T, d, V, P, G, fp8_block, P_total=P_total)
         self.params = params or default_params()
         S = P * G
         dev = self.device
@@ -217,6 +237,7 @@ class AisStep:
         self.loss = torch.zeros(1, **f32)
         self.diag = torch.zeros((C.sizeof(Diag) + 7) // 8, dtype=torch.float64, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.moments = torch.zeros(NUM_MOMENTS, dtype=torch.float64, device=dev)
         self.dH = torch.empty(max(T, 1), d, dtype=torch.bfloat16, device=dev) if want_grad else None
         self.w_quantized = False
 
@@ -233,8 +254,16 @@ class AisStep:
                     self.lse_train, self.lp_roll, self.lse_roll, self.status, self.workspace)
 
     def diagnose(self, mask, seq_offsets, rewards) -> None:
-        diagnostics(self.shape, self.params, self.lp_train, self.lp_roll, mask, seq_offsets, rewards, self.adv,
-                    self.n_valid_seq, self.rho, self.w_tilde, self.diag, self.workspace)
+        if self.group is None:
+            diagnostics(self.shape, self.params, self.lp_train, self.lp_roll, mask, seq_offsets, rewards, self.adv,
+                        self.n_valid_seq, self.rho, self.w_tilde, self.diag, self.workspace)
+            return
+        # data parallel: this rank's masked sums, one all-reduce of 12 doubles, then alpha / w_tilde from the global sums
+        from . import dist as _dist
+        diag_moments(self.shape, self.params, self.lp_train, self.lp_roll, mask, seq_offsets, rewards, self.adv,
+                     self.n_valid_seq, self.moments, self.workspace)
+        _dist.allreduce_moments(self.moments, self.group)
+        diag_finalize(self.shape, self.params, self.moments, self.lp_train, self.lp_roll, mask, self.rho, self.w_tilde, self.diag)
 
     def backward(self, H, W, tokens, mask, seq_offsets, lp_old=None) -> None:
         loss_bwd(self.shape, self.params, H, W, tokens, mask, seq_offsets, self.lse_train, self.lp_train, lp_old, self.adv,

@@ -82,6 +82,7 @@ int check_shape(const ais_shape* s) {
     if (s->ldh < s->d || s->ldw < s->d) return AIS_ERR_SHAPE;
     if (s->ldh % 16 != 0 || s->ldw % 16 != 0) return AIS_ERR_ALIGN;
     if (static_cast<int64_t>(s->P) * s->G > (1 << 24)) return AIS_ERR_SHAPE;
+    if (s->P_total != 0 && (s->P_total < s->P || static_cast<int64_t>(s->P_total) * s->G > (int64_t(1) << 30))) return AIS_ERR_SHAPE;
     return AIS_OK;
 }
 
@@ -300,6 +301,47 @@ int ais_diagnostics(const ais_shape* shape, const ais_params* params, const floa
     return AIS_OK;
 }
 
+int ais_diag_moments(const ais_shape* shape, const ais_params* params, const float* lp_train, const float* lp_roll,
+                     const uint8_t* mask, const int32_t* seq_offsets, const float* rewards, float* adv, int32_t* n_valid_seq,
+                     double* moments, void* workspace, size_t workspace_bytes, void* stream) {
+    int st = check_shape(shape);
+    if (st != AIS_OK) return st;
+    st = check_params(params);
+    if (st != AIS_OK) return st;
+    if (!lp_train || !lp_roll || !mask || !seq_offsets || !rewards || !adv || !moments) return AIS_ERR_NULL;
+    if (!aligned(moments, 8)) return AIS_ERR_ALIGN;
+    const Layout L = make_layout(shape, params);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.off_coef) return AIS_ERR_WORKSPACE;
+    st = device_setup(nullptr);
+    if (st != AIS_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const int S = shape->P * shape->G;
+    if (launch_seq_stats(mask, seq_offsets, rewards, S, shape->G, params->adv_std_norm, params->eps, adv, n_valid_seq, s) !=
+        cudaSuccess)
+        return AIS_ERR_DEVICE;
+    if (launch_moments(lp_train, lp_roll, mask, seq_offsets, adv, shape->T, S, *params, reinterpret_cast<double*>(ws + L.off_diag),
+                       moments, s) != cudaSuccess)
+        return AIS_ERR_DEVICE;
+    return AIS_OK;
+}
+
+int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const double* moments, const float* lp_train,
+                      const float* lp_roll, const uint8_t* mask, float* rho, float* w_tilde, ais_diag* diag, void* stream) {
+    int st = check_shape(shape);
+    if (st != AIS_OK) return st;
+    st = check_params(params);
+    if (st != AIS_OK) return st;
+    if (!moments || !lp_train || !lp_roll || !mask || !w_tilde || !diag) return AIS_ERR_NULL;
+    if (!aligned(moments, 8) || !aligned(diag, 8)) return AIS_ERR_ALIGN;
+    st = device_setup(nullptr);
+    if (st != AIS_OK) return st;
+    if (launch_finalize(moments, lp_train, lp_roll, mask, shape->T, *params, rho, w_tilde, diag,
+                        static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return AIS_ERR_DEVICE;
+    return AIS_OK;
+}
+
 int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H, const void* W, const int32_t* tokens,
                  const uint8_t* mask, const int32_t* seq_offsets, const float* lse_train, const float* lp_train,
                  const float* lp_old, const float* adv, const float* w_tilde, void* dH, float* loss, ais_diag* diag,
@@ -323,7 +365,8 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
     float* coef = reinterpret_cast<float*>(ws + L.off_coef);
     int32_t* nseq = reinterpret_cast<int32_t*>(ws + L.off_nseq);
     if (launch_seq_stats(mask, seq_offsets, nullptr, S, shape->G, 0, 0.f, nullptr, nseq, s) != cudaSuccess) return AIS_ERR_DEVICE;
-    if (launch_loss_coef(lp_train, lp_old, mask, seq_offsets, adv, w_tilde, nseq, shape->T, S, params->clip_eps,
+    const int P_norm = shape->P_total > 0 ? shape->P_total : shape->P;
+    if (launch_loss_coef(lp_train, lp_old, mask, seq_offsets, adv, w_tilde, nseq, shape->T, S, P_norm * shape->G, params->clip_eps,
                          reinterpret_cast<double*>(ws + L.off_diag), coef, loss, diag, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     if (shape->T == 0) return AIS_OK;

@@ -300,7 +300,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             for (int c = 0; c < 4; ++c) {
                                 uint32_t v[32];
                                 tmem_ld32(taddr + c * 32, v);
-                                tmem_ld_wait();
+                                tmem_ld_wait(v);
                                 if (c == 3) {
                                     // the partial sums are in registers: hand the buffer back before the arithmetic
                                     tc_fence_before();
@@ -338,7 +338,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     } else {
                         uint32_t v[32];
                         tmem_ld32(taddr + c * 32, v);
-                        tmem_ld_wait();
+                        tmem_ld_wait(v);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(v[i]);
                     }

@@ -276,6 +276,16 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
     *diag = d;
 }
 
+// Sums the per-block partial moments in block order into one vector of kNumMoments doubles.
+__global__ void moments_reduce_kernel(const double* __restrict__ partials, int nblocks, double* __restrict__ moments) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    for (int i = 0; i < kNumMoments; ++i) {
+        double m = 0.0;
+        for (int b = 0; b < nblocks; ++b) m += partials[b * kNumMoments + i];
+        moments[i] = m;
+    }
+}
+
 __global__ void rectify_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
                                const uint8_t* __restrict__ mask, int64_t T, double logC, const ais_diag* __restrict__ diag,
                                float* __restrict__ rho, float* __restrict__ w_tilde) {
@@ -301,7 +311,7 @@ __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __
                                                                   const int32_t* __restrict__ seq_offsets,
                                                                   const float* __restrict__ adv, const float* __restrict__ w_tilde,
                                                                   const int32_t* __restrict__ n_valid_seq, int64_t T, int S,
-                                                                  double clip_eps, double* __restrict__ partials,
+                                                                  int S_norm, double clip_eps, double* __restrict__ partials,
                                                                   float* __restrict__ coef) {
     __shared__ double scratch[32];
     double J = 0.0;
@@ -312,7 +322,7 @@ __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __
             const int s = seq_of_row(seq_offsets, S, t);
             const double A = adv[s];
             const int n = n_valid_seq[s] > 0 ? n_valid_seq[s] : 1;
-            const double norm = 1.0 / (static_cast<double>(S) * static_cast<double>(n));
+            const double norm = 1.0 / (static_cast<double>(S_norm) * static_cast<double>(n));
             const double rho_on = lp_old ? exp(static_cast<double>(lp_train[t]) - static_cast<double>(lp_old[t])) : 1.0;
             const double un = rho_on * A;
             const double cl = fmin(fmax(rho_on, 1.0 - clip_eps), 1.0 + clip_eps) * A;
@@ -379,11 +389,31 @@ cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8
     return cudaGetLastError();
 }
 
+cudaError_t launch_moments(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
+                           const float* adv, int64_t T, int S, const ais_params& p, double* partials, double* moments,
+                           cudaStream_t stream) {
+    const double logC = log(static_cast<double>(p.C));
+    moments_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, logC, partials);
+    moments_reduce_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, moments);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finalize(const double* moments, const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T,
+                            const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream) {
+    const double logC = log(static_cast<double>(p.C));
+    diag_finalize_kernel<<<1, 32, 0, stream>>>(moments, 1, p, diag);
+    if (T > 0) {
+        const int blocks = static_cast<int>(((T + 255) / 256) < 1184 ? ((T + 255) / 256) : 1184);
+        rectify_kernel<<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, logC, diag, rho, w_tilde);
+    }
+    return cudaGetLastError();
+}
+
 cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const uint8_t* mask, const int32_t* seq_offsets,
-                             const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S,
+                             const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S, int S_norm,
                              float clip_eps, double* partials, float* coef, float* loss, ais_diag* diag, cudaStream_t stream) {
     loss_coef_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, mask, seq_offsets, adv, w_tilde, n_valid_seq,
-                                                                 T, S, static_cast<double>(clip_eps), partials, coef);
+                                                                 T, S, S_norm, static_cast<double>(clip_eps), partials, coef);
     loss_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, loss, diag);
     return cudaGetLastError();
 }

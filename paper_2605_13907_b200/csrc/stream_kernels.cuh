@@ -28,9 +28,18 @@ cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8
                         const float* adv, int64_t T, int S, const ais_params& p, double* partials /*[kDiagBlocks][kNumMoments]*/,
                         float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
 
-// coef[t] and the loss; n_valid_seq must already hold the valid counts.
+// The two halves of launch_diag: partial moments summed into `moments` [kNumMoments], and everything that follows
+// from a (possibly all-reduced) moment vector.
+cudaError_t launch_moments(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
+                           const float* adv, int64_t T, int S, const ais_params& p, double* partials, double* moments,
+                           cudaStream_t stream);
+cudaError_t launch_finalize(const double* moments, const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T,
+                            const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
+
+// coef[t] and the loss; n_valid_seq must already hold the valid counts.  S_norm is the number of sequences the
+// objective averages over (all data-parallel ranks together).
 cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const uint8_t* mask, const int32_t* seq_offsets,
-                             const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S,
+                             const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S, int S_norm,
                              float clip_eps, double* partials /*[kDiagBlocks]*/, float* coef, float* loss, ais_diag* diag,
                              cudaStream_t stream);
 
