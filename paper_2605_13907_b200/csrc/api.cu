@@ -418,6 +418,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
         // dH = c (.) (U W)
         a.ncols = shape->d;
         a.n_col_tiles = (shape->d + kBN - 1) / kBN;
+        a.n_row_tiles = static_cast<int32_t>((rows + kDhRows - 1) / kDhRows);
         a.nsplit = 1;
         a.ksteps = (shape->V + 63) / 64;
         units = a.n_row_tiles * a.n_col_tiles;

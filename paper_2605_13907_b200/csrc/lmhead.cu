@@ -3,7 +3,9 @@
 //
 // One persistent CTA of three warpgroups per SM.  Warp 0 issues TMA tile loads, warp 1 issues the MMAs
 // (warps 2, 3 idle), warps 4..11 are the epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (one row per
-// thread) and column half (w-4)/4 of the 256-column accumulator.  In the FP8 pass the first warpgroup gives
+// thread) and column half (w-4)/4 of the 256-column accumulator.  The dH pass gives a CTA two row tiles
+// (256 rows, both accumulators) so that every W slice it loads is used twice; its contraction over the
+// vocabulary is so long that the one epilogue per unit need not overlap anything.  In the FP8 pass the first warpgroup gives
 // registers to the two epilogue warpgroups, which keep 128 fp32 accumulators per thread.  Two 256-column accumulators alternate so that the epilogue of one tile (or,
 // in the FP8 pass, the promotion of one scale block) overlaps the MMAs of the next.
 #include "lmhead.cuh"
@@ -121,6 +123,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBarriers);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+    constexpr int STG = (MODE == kBwdDh) ? kDhStages : kStages;                 // depth of the stage ring
+    constexpr int STG_BYTES = (MODE == kBwdDh) ? kDhStageBytes : kStageBytes;
+    constexpr int A_BYTES = (MODE == kBwdDh) ? 2 * kAStageBytes : kAStageBytes;
+    constexpr int NBUF = (MODE == kBwdDh) ? 1 : 2;                              // accumulator sets that alternate
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int num_units = (MODE == kBwdDh) ? a.n_row_tiles * a.n_col_tiles : a.n_row_tiles * a.nsplit;
@@ -151,7 +157,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            Pipe st(kStages), sc(kScaleSlots);
+            Pipe st(STG), sc(kScaleSlots);
             uint32_t issued = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
@@ -159,11 +165,16 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
                     for (int ks = 0; ks < a.ksteps; ++ks) {
                         if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag)) { ok = false; break; }
-                        uint8_t* sA = stage_base + st.idx * kStageBytes;
-                        uint8_t* sB = sA + kAStageBytes;
-                        mbar_expect_tx(&full[st.idx], kStageBytes);
+                        uint8_t* sA = stage_base + st.idx * STG_BYTES;
+                        uint8_t* sB = sA + A_BYTES;
+                        mbar_expect_tx(&full[st.idx], STG_BYTES);
                         const int kelem = (MODE == kFwdFp8) ? ks * 128 : ks * 64;
-                        tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kBM);
+                        if (MODE == kBwdDh) {
+                            tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kDhRows);
+                            tma_load_2d(sA + kAStageBytes, &tmA, &full[st.idx], kelem, w.rt * kDhRows + kBM);
+                        } else {
+                            tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kBM);
+                        }
                         if (MODE == kBwdDh) {
                             // B is W[v, n]: n (the output column) is the contiguous axis -> four 64-column boxes
 #pragma unroll
@@ -187,10 +198,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             }
             if (!ok) {
                 // another role gave up: let the copies already in flight land before the CTA exits
-                const uint32_t pending = issued < static_cast<uint32_t>(kStages) ? issued : kStages;
+                const uint32_t pending = issued < static_cast<uint32_t>(STG) ? issued : STG;
                 for (uint32_t i = 0; i < pending; ++i) {
                     const uint32_t n = issued - 1 - i;                 // n-th load overall
-                    mbar_wait_drain(&full[n % kStages], (n / kStages) & 1u);
+                    mbar_wait_drain(&full[n % STG], (n / STG) & 1u);
                 }
             }
         }
@@ -200,7 +211,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             constexpr uint32_t idesc =
                 (MODE == kFwdFp8) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
                                   : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, 0, MODE == kBwdDh ? 1 : 0);
-            Pipe st(kStages), tb(2);
+            Pipe st(STG), tb(NBUF);
             bool ok = true;
             for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit<MODE>(a, u);
@@ -212,8 +223,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     for (int ks = 0; ks < a.ksteps; ++ks) {
                         if (!mbar_wait(&full[st.idx], st.phase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t sA = smem_u32(stage_base + st.idx * kStageBytes);
-                        const uint32_t sB = sA + kAStageBytes;
+                        const uint32_t sA = smem_u32(stage_base + st.idx * STG_BYTES);
+                        const uint32_t sB = sA + A_BYTES;
                         if (MODE == kFwdFp8) {
                             const int per = 4 / a.sgroups;             // MMAs per scale block
                             for (int g = 0; g < a.sgroups && ok; ++g) {
@@ -229,16 +240,21 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                 tb.advance();
                             }
                             if (!ok) break;
+                        } else if (MODE == kBwdDh) {
+                            // two row tiles share every B slice: accumulators at TMEM columns 0 and 256
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const uint64_t bdesc = smem_desc_sw128(sB + j * 2048, kBStageBytes / 4, 1024);
+                                const uint32_t accum = (ks > 0 || j > 0) ? 1u : 0u;
+                                mma_f16(tmem_base, smem_desc_sw128(sA + j * 32, 16, 1024), bdesc, idesc, accum);
+                                mma_f16(tmem_base + kBN, smem_desc_sw128(sA + kAStageBytes + j * 32, 16, 1024), bdesc, idesc, accum);
+                            }
                         } else {
                             const uint32_t dcol = tmem_base + tb.idx * kBN;
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const uint64_t adesc = smem_desc_sw128(sA + j * 32, 16, 1024);
-                                const uint64_t bdesc = (MODE == kBwdDh)
-                                                           ? smem_desc_sw128(sB + j * 2048, kBStageBytes / 4, 1024)
-                                                           : smem_desc_sw128(sB + j * 32, 16, 1024);
-                                mma_f16(dcol, adesc, bdesc, idesc, (ks > 0 || j > 0) ? 1u : 0u);
-                            }
+                            for (int j = 0; j < 4; ++j)
+                                mma_f16(dcol, smem_desc_sw128(sA + j * 32, 16, 1024), smem_desc_sw128(sB + j * 32, 16, 1024), idesc,
+                                        (ks > 0 || j > 0) ? 1u : 0u);
                         }
                         tc_commit(&empty[st.idx]);
                         st.advance();
@@ -260,11 +276,49 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         const int half = (warp - 4) >> 2;             // column half of the accumulator
         const int r_in_tile = q * 32 + lane;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        Pipe tb(2), sc(kScaleSlots);
+        Pipe tb(NBUF), sc(kScaleSlots);
         bool ok = true;
         uint32_t flags = 0;
         for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
             const Unit w = decode_unit<MODE>(a, u);
+            if (MODE == kBwdDh) {
+                // one unit = 256 rows x 256 columns of dH, finished after the whole contraction over the vocabulary
+                if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int sub = 0; sub < 2; ++sub) {
+                    const int64_t lrow2 = static_cast<int64_t>(w.rt) * kDhRows + sub * kBM + r_in_tile;
+                    const bool in = lrow2 < a.rows;
+                    const int64_t grow2 = a.row0 + lrow2;
+                    const float cf = in ? a.coef[grow2] : 0.f;
+                    const uint32_t taddr2 = tmem_base + lane_addr + sub * kBN + half * 128;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int col0 = w.t0 * kBN + half * 128 + c * 32;
+                        uint32_t v[32];
+                        tmem_ld32(taddr2 + c * 32, v);
+                        tmem_ld_wait(v);
+                        if (in && col0 < a.ncols) {
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int i = 0; i < 32; i += 2) {
+                                const float v0 = (cf == 0.f) ? 0.f : cf * __uint_as_float(v[i]);
+                                const float v1 = (cf == 0.f) ? 0.f : cf * __uint_as_float(v[i + 1]);
+                                pk[i >> 1] = pack_bf16(v0, v1);
+                            }
+                            uint4* dst = reinterpret_cast<uint4*>(a.dH + grow2 * a.lddh + col0);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                if (col0 + j * 8 < a.ncols) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tempty[0]);
+                tb.advance();
+                continue;
+            }
             const int64_t lrow = static_cast<int64_t>(w.rt) * kBM + r_in_tile;   // row inside this launch
             const bool row_ok = lrow < a.rows;
             const int64_t grow = a.row0 + lrow;
@@ -276,9 +330,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (valid && (y < 0 || y >= a.ncols)) { flags |= AIS_FLAG_TOKEN_RANGE; y = -1; }
             }
             float m2 = kNegBig, s = 0.f, zy = -INFINITY;       // log2-domain running max, sum, target logit
-            float lse2 = 0.f, coef = 0.f;
+            float lse2 = 0.f;
             if (MODE == kBwdP && row_ok) lse2 = a.lse[grow] * kLog2e;
-            if (MODE == kBwdDh && row_ok) coef = a.coef[grow];
 
             for (int t = w.t0; t < w.t1 && ok; ++t) {
                 const int col_base = t * kBN + half * 128;    // first output column of this thread's half
@@ -374,20 +427,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                 pk[i >> 1] = pack_bf16(p0, p1);
                             }
                             uint4* dst = reinterpret_cast<uint4*>(a.U + lrow * a.ldU + col0);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                if (col0 + j * 8 < a.ncols) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                        }
-                    } else {   // kBwdDh
-                        if (row_ok && col0 < a.ncols) {
-                            uint32_t pk[16];
-#pragma unroll
-                            for (int i = 0; i < 32; i += 2) {
-                                const float v0 = (coef == 0.f) ? 0.f : coef * x[i];
-                                const float v1 = (coef == 0.f) ? 0.f : coef * x[i + 1];
-                                pk[i >> 1] = pack_bf16(v0, v1);
-                            }
-                            uint4* dst = reinterpret_cast<uint4*>(a.dH + grow * a.lddh + col0);
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
                                 if (col0 + j * 8 < a.ncols) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);

@@ -21,6 +21,11 @@ constexpr int kAStageBytes = kBM * kStageKBytes;
 constexpr int kBStageBytes = kBN * kStageKBytes;
 constexpr int kStageBytes = kAStageBytes + kBStageBytes;
 constexpr int kStages = 4;
+// dH pass: a CTA owns two row tiles (256 rows) so that every W tile it loads feeds two accumulators
+constexpr int kDhRows = 2 * kBM;
+constexpr int kDhStageBytes = 2 * kAStageBytes + kBStageBytes;
+constexpr int kDhStages = 3;
+static_assert(kDhStages * kDhStageBytes <= kStages * kStageBytes, "the dH stage ring must fit the same shared memory");
 constexpr int kScaleSlots = 4;
 constexpr int kScaleSlotBytes = 4 * (kBM + kBN) * 4;   // up to 4 scale blocks per stage
 constexpr int kScaleBOffset = 4 * kBM * 4;
@@ -32,7 +37,7 @@ constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kScaleSlots * kScaleSl
 struct LmheadArgs {
     int64_t rows;          // valid rows handled by this launch
     int64_t row0;          // global index of local row 0 (per-row vectors are indexed globally)
-    int32_t n_row_tiles;
+    int32_t n_row_tiles;   // row tiles of 128 rows (dH pass: of 256 rows)
     int32_t ncols;         // output columns: V (forward, recompute) or d (dH)
     int32_t n_col_tiles;
     int32_t ksteps;        // shared-memory stages per accumulator tile
