@@ -30,6 +30,10 @@ sys.path.insert(0, ROOT)
 
 import workloads  # noqa: E402
 
+# DRAM bytes (read + write) of one launch of the bf16 forward kernel, from the ncu capture summarised in
+# profiles/ncu_full_all_kernels_small_case.md: 3.829 GB for 3 sweeps over W on the 1-prompt case, scaled to the
+# 15 sweeps of the full workload (the traffic is W re-read once per group of 37 row tiles, plus H once).
+TRAFFIC_BF16_FWD = {"qwen3_8b": 3.829e9 * 15 / 3}
 METRIC = "AIS-corrected fwd+bwd tokens/sec"
 UNIT = "tokens/s"
 
@@ -272,7 +276,7 @@ def run_ours(args) -> None:
                        "alpha": diag["alpha"], "d_bar": diag["d_bar"]},
             "segments_ms": seg,
             "roofline": {"bound": "tensor", "kernel": "lmhead_kernel<bf16 forward> (trainer log-probs)", "achieved": achieved,
-                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": TRAFFIC_BF16_FWD.get(args.workload) if not args.prompts else None,
                          "peak_source": peaks["source"] + " bf16 sustained (kernel timed inside a long step)",
                          "passes": {"fwd_roll_fp8_tflops": flops_pass / (seg["fwd_roll_fp8"] * 1e-3) / 1e12,
                                     "bwd_two_passes_tflops": 2 * flops_pass / (seg["loss_bwd"] * 1e-3) / 1e12,

@@ -237,11 +237,16 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
 }
 
 __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nblocks, ais_params p, ais_diag* __restrict__ diag) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    double m[kNumMoments];
-    for (int i = 0; i < kNumMoments; ++i) m[i] = 0.0;
-    for (int b = 0; b < nblocks; ++b)
-        for (int i = 0; i < kNumMoments; ++i) m[i] += partials[b * kNumMoments + i];
+    // one thread per moment sums the partials in block order; thread 0 then derives the diagnostics
+    __shared__ double m[kNumMoments];
+    if (blockIdx.x != 0) return;
+    if (threadIdx.x < kNumMoments) {
+        double acc = 0.0;
+        for (int b = 0; b < nblocks; ++b) acc += partials[b * kNumMoments + threadIdx.x];
+        m[threadIdx.x] = acc;
+    }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
     ais_diag d;
     d.status_flags = 0;
     d.reserved = 0;
@@ -278,12 +283,10 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
 
 // Sums the per-block partial moments in block order into one vector of kNumMoments doubles.
 __global__ void moments_reduce_kernel(const double* __restrict__ partials, int nblocks, double* __restrict__ moments) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    for (int i = 0; i < kNumMoments; ++i) {
-        double m = 0.0;
-        for (int b = 0; b < nblocks; ++b) m += partials[b * kNumMoments + i];
-        moments[i] = m;
-    }
+    if (blockIdx.x != 0 || threadIdx.x >= kNumMoments) return;
+    double m = 0.0;
+    for (int b = 0; b < nblocks; ++b) m += partials[b * kNumMoments + threadIdx.x];
+    moments[threadIdx.x] = m;
 }
 
 __global__ void rectify_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
