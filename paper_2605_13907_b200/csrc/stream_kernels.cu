@@ -9,18 +9,73 @@ namespace ais {
 namespace {
 
 // ------------------------------------------------------------------------------------------------
-// FP8-E4M3 block quantisation.  A CTA covers 32 rows x 2048 columns; each warp walks 4 rows, a lane
+// FP8-E4M3 block quantisation.  A CTA covers 32 rows x 1024 columns; each warp walks 4 rows, a lane
 // holds 8 consecutive bf16 values (16-byte load), the lanes of one block share the block's amax by
 // shuffles, and the block-major scales are staged in shared memory so that they leave coalesced.
 // ------------------------------------------------------------------------------------------------
 constexpr int kQRows = 32;
-constexpr int kQCols = 2048;
+constexpr int kQCols = 1024;
 constexpr int kQThreads = 256;
+constexpr int kQIters = kQCols / 256;      // 16-byte loads per lane and row
 
 __device__ __forceinline__ uint16_t cvt_e4m3x2(float hi, float lo) {
     uint16_t r;
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
     return r;
+}
+
+// Correctly rounded x / s from the correctly rounded reciprocal y = RN(1/s): two residual corrections with
+// fused multiply-adds; the first makes the quotient faithful, and a faithful quotient corrected once more with
+// the exact residual is the round-to-nearest quotient (Markstein's division theorem).  |x / s| <= 448 here, so
+// nothing overflows; a quotient that underflows encodes to zero either way; the sign of x is restored
+// explicitly because a zero residual sum would turn -0 into +0.
+__device__ __forceinline__ float exact_div(float x, float s, float y) {
+    float q = x * y;
+    q = __fmaf_rn(__fmaf_rn(-s, q, x), y, q);
+    q = __fmaf_rn(__fmaf_rn(-s, q, x), y, q);
+    return copysignf(q, x);
+}
+
+// IEEE division kept out of line: it is only reached for scales outside [2^-100, 2^100] and would otherwise
+// be inlined eight times into every copy of the hot loop.
+__device__ __noinline__ float slow_div(float x, float s) { return __fdiv_rn(x, s); }
+
+template <int BLOCK>
+__device__ __forceinline__ void quantize_lane(const uint4 raw, bool in_range, int lane, float& scale_out, uint2& out) {
+    constexpr int kLanesPerBlock = BLOCK / 8;
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+    // amax on the bf16 bit patterns: |x| is the pattern without its sign bit, and patterns of non-negative
+    // values order like the values, so packed 16-bit unsigned maxima do the work of eight float compares
+    uint32_t m = __vmaxu2(__vmaxu2(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu), __vmaxu2(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu));
+    m = max(m & 0xFFFFu, m >> 16);
+#pragma unroll
+    for (int off = 1; off < kLanesPerBlock; off <<= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, off));
+    // the first lane of the block derives the scale and its reciprocal once and hands both to the others
+    float s = 1.0f, y = 1.0f;
+    const int leader = lane & ~(kLanesPerBlock - 1);
+    if (lane == leader && m != 0u) {
+        s = __fdiv_rn(__uint_as_float(m << 16), 448.0f);
+        y = __frcp_rn(s);
+    }
+    s = __shfl_sync(0xffffffffu, s, leader);
+    y = __shfl_sync(0xffffffffu, y, leader);
+    scale_out = s;
+    if (!in_range) return;
+    float v[8], qv[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+    if (s > 0x1p-100f && s < 0x1p100f) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) qv[i] = exact_div(v[i], s, y);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) qv[i] = slow_div(v[i], s);      // rare: scale outside the safe exponent range
+    }
+    out.x = static_cast<uint32_t>(cvt_e4m3x2(qv[1], qv[0])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[3], qv[2])) << 16);
+    out.y = static_cast<uint32_t>(cvt_e4m3x2(qv[5], qv[4])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[7], qv[6])) << 16);
 }
 
 template <int BLOCK>
@@ -35,57 +90,26 @@ __global__ void __launch_bounds__(kQThreads) quantize_kernel(const __nv_bfloat16
     const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kQRows;
     const int64_t col0 = static_cast<int64_t>(blockIdx.x) * kQCols;
 
-#pragma unroll
+    // each warp walks 4 rows; the row loop is kept rolled so that the kernel stays small in the instruction cache
+    // (a fully unrolled version stalled on instruction fetch); occupancy, not prefetching, hides the load latency
+#pragma unroll 1
     for (int rr = 0; rr < 4; ++rr) {
         const int r_local = warp * 4 + rr;
         const int64_t row = row0 + r_local;
-        if (row >= rows) break;
-        const __nv_bfloat16* xr = x + row * ld;
-        uint4 raw[8];
+        uint4 raw[kQIters];
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
+        for (int it = 0; it < kQIters; ++it) {
             const int64_t col = col0 + it * 256 + lane * 8;
-            raw[it] = (col < cols) ? __ldg(reinterpret_cast<const uint4*>(xr + col)) : make_uint4(0, 0, 0, 0);
+            raw[it] = (row < rows && col < cols) ? __ldg(reinterpret_cast<const uint4*>(x + row * ld + col)) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
+        for (int it = 0; it < kQIters; ++it) {
             const int64_t col = col0 + it * 256 + lane * 8;
-            float v[8];
-            const uint32_t w[4] = {raw[it].x, raw[it].y, raw[it].z, raw[it].w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                v[2 * i] = __uint_as_float(w[i] << 16);
-                v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-            }
-            float amax = 0.f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
-#pragma unroll
-            for (int off = 1; off < kLanesPerBlock; off <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
-            const float s = (amax == 0.f) ? 1.0f : __fdiv_rn(amax, 448.0f);
-            if (col < cols) {
-                float qv[8];
-                if (s > 0x1p-100f && s < 0x1p100f) {
-                    // Correctly rounded x / s from the correctly rounded reciprocal y = RN(1/s): two residual
-                    // corrections with fused multiply-adds; the first makes the quotient faithful, and a faithful
-                    // quotient corrected once more with the exact residual is the round-to-nearest quotient
-                    // (Markstein's division theorem).  |x / s| <= 448 here, so nothing overflows; a quotient that
-                    // underflows encodes to zero either way; the sign of x is restored explicitly.
-                    const float y = __frcp_rn(s);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float q = v[i] * y;
-                        q = __fmaf_rn(__fmaf_rn(-s, q, v[i]), y, q);
-                        q = __fmaf_rn(__fmaf_rn(-s, q, v[i]), y, q);
-                        qv[i] = copysignf(q, v[i]);          // a zero residual sum would turn -0 into +0
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) qv[i] = __fdiv_rn(v[i], s);
-                }
-                uint2 out;
-                out.x = static_cast<uint32_t>(cvt_e4m3x2(qv[1], qv[0])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[3], qv[2])) << 16);
-                out.y = static_cast<uint32_t>(cvt_e4m3x2(qv[5], qv[4])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[7], qv[6])) << 16);
+            const bool in = row < rows && col < cols;
+            float s;
+            uint2 out;
+            quantize_lane<BLOCK>(raw[it], in, lane, s, out);
+            if (in) {
                 *reinterpret_cast<uint2*>(codes + row * ldq + col) = out;
                 if ((lane % kLanesPerBlock) == 0) sc[(it * 256 + lane * 8) / BLOCK][r_local] = s;
             }
