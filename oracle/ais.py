@@ -189,9 +189,15 @@ def surrogate_terms(lp_theta, lp_old, adv_tok, clip_eps: float):
     return rho_on, sur, active
 
 
-def loss_and_coeff(lp_theta, lp_old, mask, seq_offsets, adv, w_tilde, P: int, G: int, clip_eps: float):
-    """loss = -J with J = sum_s 1/(P G n_s) sum_{t in s, valid} w_tilde_t * sur_t  (AIS-GRPO objective
-    without the KL term; the expectation over prompts is the mean over the P prompts, |o_i| = n_s).
+def loss_and_coeff(lp_theta, lp_old, mask, seq_offsets, adv, w_tilde, P: int, G: int, clip_eps: float,
+                   lp_ref=None, beta_kl: float = 0.0):
+    """loss = -J with J = sum_s 1/(P G n_s) sum_{t in s, valid} [w_tilde_t * sur_t - beta_kl * kl_t]
+    (AIS-GRPO objective; the expectation over prompts is the mean over the P prompts, |o_i| = n_s).
+
+    kl_t is the per-token estimate of D_KL(pi_theta || pi_ref).  The paper writes the term but not its
+    estimator; the reading here is the one of the GRPO paper it builds on,
+    kl_t = r - log r - 1 with r = pi_ref / pi_theta = exp(lp_ref - lp_theta), which is non-negative and
+    zero only when the two log-probs agree.  lp_ref = None (or beta_kl = 0) drops the term.
 
     Also returns c_t, the per-token factor of the logit gradient
     d loss / d z[t, :] = c_t (softmax(z_t) - onehot(y_t)), with w_tilde, A and lp_old held constant
@@ -208,7 +214,25 @@ def loss_and_coeff(lp_theta, lp_old, mask, seq_offsets, adv, w_tilde, P: int, G:
     wt = np.asarray(w_tilde, np.float64)
     J = np.sum(np.where(valid, wt * sur * norm, 0.0))
     c = np.where(valid & active, wt * adv_tok * rho_on * norm, 0.0)
+    if lp_ref is not None and beta_kl != 0.0:
+        log_r = np.asarray(lp_ref, np.float64) - np.asarray(lp_theta, np.float64)
+        r = np.exp(log_r)
+        kl = r - log_r - 1.0
+        J = J - beta_kl * np.sum(np.where(valid, kl * norm, 0.0))
+        # d kl / d lp_theta = 1 - r ; d loss / d lp_theta = +beta * norm * (1 - r) ; d lp / d z = onehot - p
+        c = c - np.where(valid, beta_kl * (1.0 - r) * norm, 0.0)
     return -J, c
+
+
+def kl_term(lp_theta, lp_ref, mask, seq_offsets, P: int, G: int) -> float:
+    """sum_s 1/(P G n_s) sum_t kl_t : the value of the KL term of the objective (without beta)."""
+    T = len(mask)
+    valid = np.asarray(mask).astype(bool)
+    sid = seq_ids(seq_offsets, T)
+    n_tok = np.maximum(valid_counts(mask, seq_offsets)[sid], 1).astype(np.float64)
+    log_r = np.asarray(lp_ref, np.float64) - np.asarray(lp_theta, np.float64)
+    kl = np.exp(log_r) - log_r - 1.0
+    return float(np.sum(np.where(valid, kl / (P * G * n_tok), 0.0)))
 
 
 def grad_hidden(H, W, tokens, c) -> np.ndarray:
@@ -225,7 +249,7 @@ def grad_hidden(H, W, tokens, c) -> np.ndarray:
 
 # --------------------------------------------------------------------------- whole path
 def full_path(H, W, tokens, mask, seq_offsets, rewards, P: int, G: int, block: int,
-              params: Params | None = None, lp_old=None, want_grad: bool = True) -> dict:
+              params: Params | None = None, lp_old=None, want_grad: bool = True, lp_ref=None, beta_kl: float = 0.0) -> dict:
     """Algorithm 1, 'Adaptive Coefficient Estimation' through 'Policy Update' (loss and dH only)."""
     p = params or Params()
     T = np.asarray(H).shape[0]
@@ -238,7 +262,7 @@ def full_path(H, W, tokens, mask, seq_offsets, rewards, P: int, G: int, block: i
     diag = diagnostics(lp_t, lp_r, mask, adv_tok, p)
     w_tilde = rectify(wbar, diag["alpha"], mask)
     old = lp_t if lp_old is None else lp_old
-    loss, c = loss_and_coeff(lp_t, old, mask, seq_offsets, adv, w_tilde, P, G, p.clip_eps)
+    loss, c = loss_and_coeff(lp_t, old, mask, seq_offsets, adv, w_tilde, P, G, p.clip_eps, lp_ref=lp_ref, beta_kl=beta_kl)
     diag["loss"] = float(loss)
     out = dict(lp_train=lp_t, lse_train=lse_t, lp_roll=lp_r, lse_roll=lse_r, qH=qH, sH=sH, qW=qW, sW=sW,
                adv=adv, rho=rho, wbar=wbar, w_tilde=w_tilde, diag=diag, loss=loss, c=c)

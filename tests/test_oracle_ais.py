@@ -316,6 +316,42 @@ def test_gradient_matches_central_differences(shift_old):
     assert np.all(dH[mask == 0] == 0)
 
 
+def test_kl_term_value_sign_and_gradient():
+    """kl_t = r - log r - 1 >= 0 with equality at r = 1; closed form on hand values; the gradient including the
+    KL term matches central differences (the reference log-probs come from a second, perturbed LM head)."""
+    H, W, tok, mask, offs, rewards, P, G = _tiny_problem(seed=16)
+    rng = np.random.default_rng(17)
+    adv = ais.advantages(rewards, G)
+    w_tilde = np.ones(len(tok))
+    lp0, _ = ais.logprob_train(H, W, tok, mask)
+    W_ref = W + rng.normal(0, 0.2, W.shape)
+    lp_ref, _ = ais.logprob_train(H, W_ref, tok, mask)
+    # value: identical policies give zero, otherwise positive; one token worked by hand
+    assert ais.kl_term(lp0, lp0, mask, offs, P, G) == 0.0
+    assert ais.kl_term(lp0, lp_ref, mask, offs, P, G) > 0.0
+    one = ais.kl_term(np.array([math.log(0.5)]), np.array([math.log(0.25)]), np.ones(1), np.array([0, 1]), 1, 1)
+    assert one == pytest.approx(0.5 - math.log(0.5) - 1.0, abs=1e-15)            # r = 1/2
+    beta = 0.7
+    l0, c0 = ais.loss_and_coeff(lp0, lp0, mask, offs, adv, w_tilde, P, G, 0.2)
+    l1, c1 = ais.loss_and_coeff(lp0, lp0, mask, offs, adv, w_tilde, P, G, 0.2, lp_ref=lp_ref, beta_kl=beta)
+    assert l1 - l0 == pytest.approx(beta * ais.kl_term(lp0, lp_ref, mask, offs, P, G), abs=1e-14)
+    dH = ais.grad_hidden(H, W, tok, c1)
+    num = np.zeros_like(H)
+    h = 1e-5
+
+    def f(Hx):
+        lp, _ = ais.logprob_train(Hx, W, tok, mask)
+        return ais.loss_and_coeff(lp, lp0, mask, offs, adv, w_tilde, P, G, 0.2, lp_ref=lp_ref, beta_kl=beta)[0]
+    for t in range(H.shape[0]):
+        for k in range(H.shape[1]):
+            Hp, Hm = H.copy(), H.copy()
+            Hp[t, k] += h
+            Hm[t, k] -= h
+            num[t, k] = (f(Hp) - f(Hm)) / (2 * h)
+    assert np.linalg.norm(dH - num) <= 1e-6 * np.linalg.norm(num) + 1e-10
+    assert np.linalg.norm(ais.grad_hidden(H, W, tok, c1 - c0)) > 0                 # the KL part is not a no-op
+
+
 def test_logit_gradient_rows_sum_to_zero_and_weight_layout():
     H, W, tok, mask, offs, rewards, P, G = _tiny_problem(seed=12)
     c = np.random.default_rng(0).normal(size=len(tok))
