@@ -87,7 +87,8 @@ typedef struct ais_params {
     int32_t vocab_chunk;  /* 0: library default.  Otherwise the vocabulary is streamed in
                              independent chunks of about this many columns whose partial
                              (max, sum-exp, target logit) triples are merged afterwards.     */
-    int32_t reserved;
+    float beta_kl;        /* weight of the KL(pi_theta || pi_ref) term of the objective (0: no term;
+                             the paper gives no value).  Used only when ais_loss_bwd gets lp_ref.  */
 } ais_params;
 
 /* Everything the reductions produce; lives in DEVICE memory, the caller copies it back. */
@@ -109,6 +110,7 @@ typedef struct ais_diag {
     double loss;          /* written by ais_loss_bwd                                         */
     double kl_k1;         /* monitor: mean(lp_roll - lp_train)                               */
     double mean_abs_dp;   /* monitor: mean |exp(lp_train) - exp(lp_roll)|                    */
+    double kl_ref;        /* written by ais_loss_bwd: value of the KL term (without beta_kl) */
     uint32_t status_flags;
     uint32_t reserved;
 } ais_diag;
@@ -193,21 +195,26 @@ int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const do
                       float* rho, float* w_tilde, ais_diag* diag, void* stream);
 
 /*
- * AIS-GRPO surrogate loss and its gradient with respect to H (Eq. ais-grpo without the KL term;
- * the objective is maximised, so loss = -J).  With rho_on = exp(lp_train - lp_old)
+ * AIS-GRPO loss and its gradient with respect to H (Eq. ais-grpo; the objective is maximised, so
+ * loss = -J).  With rho_on = exp(lp_train - lp_old)
  * (lp_old == NULL means rho_on = 1) and n_s the valid rows of sequence s:
  *     loss  = - sum_s 1/(P G n_s) sum_{t in s, mask} w_tilde[t] min(rho_on A_s, clip(rho_on, 1 +- clip_eps) A_s)
  *     c_t   = mask[t] w_tilde[t] A_s rho_on [unclipped branch active] / (P G n_s)
  * (P is shape->P_total when that is set, so that the losses of all data-parallel ranks add up to the global one)
  *     dH[t,:] = c_t (softmax(z[t,:]) - onehot(tokens[t])) W
- * The softmax is recomputed from H, W and lse_train; w_tilde, A and lp_old are constants.
+ * With lp_ref != NULL and beta_kl != 0 the KL term is included.  The paper does not name its estimator; this
+ * library uses the one of the GRPO paper it builds on, per token kl_t = r - log r - 1 with
+ * r = exp(lp_ref[t] - lp_train[t]) (lp_ref: log-probs of the sampled tokens under the reference policy, e.g.
+ * from another ais_logprob_fwd call with the reference LM head):
+ *     loss += beta_kl sum_s 1/(P G n_s) sum_t kl_t ,   c_t -= mask[t] beta_kl (1 - r) / (P G n_s)
+ * The softmax is recomputed from H, W and lse_train; w_tilde, A, lp_old and lp_ref are constants.
  * dH [T, ldh] bf16 (written, zero rows where mask = 0), loss: one float on the device (may be NULL),
  * diag: if not NULL its `loss` field is written too.
  */
 int ais_loss_bwd(const ais_shape* shape, const ais_params* params,
                  const void* H, const void* W, const int32_t* tokens, const uint8_t* mask,
                  const int32_t* seq_offsets, const float* lse_train, const float* lp_train,
-                 const float* lp_old, const float* adv, const float* w_tilde,
+                 const float* lp_old, const float* lp_ref, const float* adv, const float* w_tilde,
                  void* dH, float* loss, ais_diag* diag,
                  uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
 

@@ -28,13 +28,13 @@ class Shape(C.Structure):
 class Params(C.Structure):
     _fields_ = [("C", C.c_float), ("delta", C.c_float), ("gamma", C.c_float), ("eps", C.c_float),
                 ("beta_var", C.c_float), ("clip_eps", C.c_float), ("alpha_override", C.c_float),
-                ("adv_std_norm", C.c_int32), ("vocab_chunk", C.c_int32), ("reserved", C.c_int32)]
+                ("adv_std_norm", C.c_int32), ("vocab_chunk", C.c_int32), ("beta_kl", C.c_float)]
 
 
 class Diag(C.Structure):
     _fields_ = [(n, C.c_double) for n in
                 ("n_valid", "mean_w", "cv2", "ess", "ess_ratio", "alpha_ess", "d_bar", "alpha_mis", "std_A", "std_Aw",
-                 "delta_sigma", "alpha_var", "alpha_adaptive", "alpha", "loss", "kl_k1", "mean_abs_dp")] + \
+                 "delta_sigma", "alpha_var", "alpha_adaptive", "alpha", "loss", "kl_k1", "mean_abs_dp", "kl_ref")] + \
                [("status_flags", C.c_uint32), ("reserved", C.c_uint32)]
 
     def as_dict(self) -> dict:
@@ -70,7 +70,7 @@ def lib() -> C.CDLL:
         L.ais_diagnostics.restype = C.c_int
         L.ais_diagnostics.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.ais_loss_bwd.restype = C.c_int
-        L.ais_loss_bwd.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 14 + [vp, sz, vp]
+        L.ais_loss_bwd.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 15 + [vp, sz, vp]
         L.ais_diag_moments.restype = C.c_int
         L.ais_diag_moments.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 8 + [vp, sz, vp]
         L.ais_diag_finalize.restype = C.c_int
@@ -170,10 +170,11 @@ def diag_finalize(shape: Shape, params: Params, moments, lp_train, lp_roll, mask
 
 
 def loss_bwd(shape: Shape, params: Params, H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, adv, w_tilde, dH, loss,
-             diag, dev_status, workspace):
-    _require_cuda(H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, adv, w_tilde, dH, loss, diag, dev_status, workspace)
+             diag, dev_status, workspace, lp_ref=None):
+    _require_cuda(H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, lp_ref, adv, w_tilde, dH, loss, diag, dev_status,
+                  workspace)
     _check(lib().ais_loss_bwd(C.byref(shape), C.byref(params), _ptr(H), _ptr(W), _ptr(tokens), _ptr(mask), _ptr(seq_offsets),
-                              _ptr(lse_train), _ptr(lp_train), _ptr(lp_old), _ptr(adv), _ptr(w_tilde), _ptr(dH), _ptr(loss),
+                              _ptr(lse_train), _ptr(lp_train), _ptr(lp_old), _ptr(lp_ref), _ptr(adv), _ptr(w_tilde), _ptr(dH), _ptr(loss),
                               _ptr(diag), _ptr(dev_status), _ptr(workspace), workspace.numel() * workspace.element_size(),
                               _stream(workspace)), "ais_loss_bwd")
 
@@ -265,15 +266,15 @@ class AisStep:
         _dist.allreduce_moments(self.moments, self.group)
         diag_finalize(self.shape, self.params, self.moments, self.lp_train, self.lp_roll, mask, self.rho, self.w_tilde, self.diag)
 
-    def backward(self, H, W, tokens, mask, seq_offsets, lp_old=None) -> None:
+    def backward(self, H, W, tokens, mask, seq_offsets, lp_old=None, lp_ref=None) -> None:
         loss_bwd(self.shape, self.params, H, W, tokens, mask, seq_offsets, self.lse_train, self.lp_train, lp_old, self.adv,
-                 self.w_tilde, self.dH, self.loss, self.diag, self.status, self.workspace)
+                 self.w_tilde, self.dH, self.loss, self.diag, self.status, self.workspace, lp_ref=lp_ref)
 
-    def step(self, H, W, tokens, mask, seq_offsets, rewards, lp_old=None, requantize_w: bool = True) -> None:
+    def step(self, H, W, tokens, mask, seq_offsets, rewards, lp_old=None, requantize_w: bool = True, lp_ref=None) -> None:
         self.forward(H, W, tokens, mask, requantize_w)
         self.diagnose(mask, seq_offsets, rewards)
         if self.dH is not None:
-            self.backward(H, W, tokens, mask, seq_offsets, lp_old)
+            self.backward(H, W, tokens, mask, seq_offsets, lp_old, lp_ref)
 
     def read_diag(self) -> dict:
         return read_diag(self.diag)

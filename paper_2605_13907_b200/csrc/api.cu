@@ -92,7 +92,7 @@ int check_params(const ais_params* p) {
         !(p->beta_var >= 0.f))
         return AIS_ERR_PARAM;
     if (!isnan(p->alpha_override) && !(p->alpha_override >= 0.f && p->alpha_override <= 1.f)) return AIS_ERR_PARAM;
-    if (p->vocab_chunk < 0) return AIS_ERR_PARAM;
+    if (p->vocab_chunk < 0 || !(p->beta_kl >= 0.f)) return AIS_ERR_PARAM;
     return AIS_OK;
 }
 
@@ -171,7 +171,7 @@ void ais_default_params(ais_params* p) {
     p->alpha_override = NAN;
     p->adv_std_norm = 0;
     p->vocab_chunk = 0;
-    p->reserved = 0;
+    p->beta_kl = 0.0f;
 }
 
 size_t ais_workspace_min_bytes(const ais_shape* shape, const ais_params* params) {
@@ -344,7 +344,8 @@ int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const do
 
 int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H, const void* W, const int32_t* tokens,
                  const uint8_t* mask, const int32_t* seq_offsets, const float* lse_train, const float* lp_train,
-                 const float* lp_old, const float* adv, const float* w_tilde, void* dH, float* loss, ais_diag* diag,
+                 const float* lp_old, const float* lp_ref, const float* adv, const float* w_tilde, void* dH, float* loss,
+                 ais_diag* diag,
                  uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream) {
     int st = check_shape(shape);
     if (st != AIS_OK) return st;
@@ -366,7 +367,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
     int32_t* nseq = reinterpret_cast<int32_t*>(ws + L.off_nseq);
     if (launch_seq_stats(mask, seq_offsets, nullptr, S, shape->G, 0, 0.f, nullptr, nseq, s) != cudaSuccess) return AIS_ERR_DEVICE;
     const int P_norm = shape->P_total > 0 ? shape->P_total : shape->P;
-    if (launch_loss_coef(lp_train, lp_old, mask, seq_offsets, adv, w_tilde, nseq, shape->T, S, P_norm * shape->G, params->clip_eps,
+    if (launch_loss_coef(lp_train, lp_old, lp_ref, params->beta_kl, mask, seq_offsets, adv, w_tilde, nseq, shape->T, S, P_norm * shape->G, params->clip_eps,
                          reinterpret_cast<double*>(ws + L.off_diag), coef, loss, diag, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     if (shape->T == 0) return AIS_OK;

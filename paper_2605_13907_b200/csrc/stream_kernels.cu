@@ -275,6 +275,7 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
     d.status_flags = 0;
     d.reserved = 0;
     d.loss = 0.0;
+    d.kl_ref = 0.0;
     const double N = m[0];
     d.n_valid = N;
     if (N <= 0.0) {
@@ -334,6 +335,7 @@ __global__ void rectify_kernel(const float* __restrict__ lp_train, const float* 
 // Per-token gradient factor c_t and the surrogate loss (Eq. ais-grpo without the KL term).
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_old,
+                                                                  const float* __restrict__ lp_ref, double beta_kl,
                                                                   const uint8_t* __restrict__ mask,
                                                                   const int32_t* __restrict__ seq_offsets,
                                                                   const float* __restrict__ adv, const float* __restrict__ w_tilde,
@@ -341,7 +343,7 @@ __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __
                                                                   int S_norm, double clip_eps, double* __restrict__ partials,
                                                                   float* __restrict__ coef) {
     __shared__ double scratch[32];
-    double J = 0.0;
+    double J = 0.0, KL = 0.0;
     for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T;
          t += static_cast<int64_t>(gridDim.x) * blockDim.x) {
         double c = 0.0;
@@ -356,19 +358,38 @@ __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __
             const double wt = w_tilde[t];
             J += wt * fmin(un, cl) * norm;
             if (un <= cl) c = wt * A * rho_on * norm;
+            if (lp_ref) {
+                // KL(pi_theta || pi_ref) estimate r - log r - 1, r = pi_ref / pi_theta; its slope in lp_theta is 1 - r
+                const double log_r = static_cast<double>(lp_ref[t]) - static_cast<double>(lp_train[t]);
+                const double r = exp(log_r);
+                KL += (r - log_r - 1.0) * norm;
+                c -= beta_kl * (1.0 - r) * norm;
+            }
         }
         coef[t] = static_cast<float>(c);
     }
     const double tot = block_sum(J, scratch);
-    if (threadIdx.x == 0) partials[blockIdx.x] = tot;
+    const double tot_kl = block_sum(KL, scratch);
+    if (threadIdx.x == 0) {
+        partials[2 * blockIdx.x] = tot;
+        partials[2 * blockIdx.x + 1] = tot_kl;
+    }
 }
 
-__global__ void loss_finalize_kernel(const double* __restrict__ partials, int nblocks, float* loss, ais_diag* diag) {
+__global__ void loss_finalize_kernel(const double* __restrict__ partials, int nblocks, double beta_kl, float* loss,
+                                     ais_diag* diag) {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    double J = 0.0;
-    for (int b = 0; b < nblocks; ++b) J += partials[b];
-    if (loss) *loss = static_cast<float>(-J);
-    if (diag) diag->loss = -J;
+    double J = 0.0, KL = 0.0;
+    for (int b = 0; b < nblocks; ++b) {
+        J += partials[2 * b];
+        KL += partials[2 * b + 1];
+    }
+    const double total = -J + beta_kl * KL;
+    if (loss) *loss = static_cast<float>(total);
+    if (diag) {
+        diag->loss = total;
+        diag->kl_ref = KL;
+    }
 }
 
 }  // namespace
@@ -436,12 +457,15 @@ cudaError_t launch_finalize(const double* moments, const float* lp_train, const 
     return cudaGetLastError();
 }
 
-cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const uint8_t* mask, const int32_t* seq_offsets,
+cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const float* lp_ref, float beta_kl, const uint8_t* mask,
+                             const int32_t* seq_offsets,
                              const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S, int S_norm,
                              float clip_eps, double* partials, float* coef, float* loss, ais_diag* diag, cudaStream_t stream) {
-    loss_coef_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, mask, seq_offsets, adv, w_tilde, n_valid_seq,
-                                                                 T, S, S_norm, static_cast<double>(clip_eps), partials, coef);
-    loss_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, loss, diag);
+    const float* ref = (beta_kl != 0.f) ? lp_ref : nullptr;
+    loss_coef_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, ref, static_cast<double>(beta_kl), mask, seq_offsets,
+                                                                 adv, w_tilde, n_valid_seq, T, S, S_norm,
+                                                                 static_cast<double>(clip_eps), partials, coef);
+    loss_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, ref ? static_cast<double>(beta_kl) : 0.0, loss, diag);
     return cudaGetLastError();
 }
 

@@ -38,9 +38,10 @@ cudaError_t launch_finalize(const double* moments, const float* lp_train, const 
 
 // coef[t] and the loss; n_valid_seq must already hold the valid counts.  S_norm is the number of sequences the
 // objective averages over (all data-parallel ranks together).
-cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const uint8_t* mask, const int32_t* seq_offsets,
+cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const float* lp_ref, float beta_kl, const uint8_t* mask,
+                             const int32_t* seq_offsets,
                              const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S, int S_norm,
-                             float clip_eps, double* partials /*[kDiagBlocks]*/, float* coef, float* loss, ais_diag* diag,
+                             float clip_eps, double* partials /*[kDiagBlocks][2]*/, float* coef, float* loss, ais_diag* diag,
                              cudaStream_t stream);
 
 }  // namespace ais

@@ -203,6 +203,37 @@ def test_alpha_endpoints_and_clip_on_gpu():
     _compare_all(batch, step, ref, a)
 
 
+def test_kl_term_on_gpu():
+    """Eq. ais-grpo with its KL term: reference log-probs from a perturbed LM head (computed by the library's own
+    forward pass on the GPU side and by the oracle on the CPU side), beta_kl = 0.5."""
+    ais = _lib()
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], V=768, lengths="uniform:30:70", seed=33)
+    batch = _to_cuda(workloads.make_batch(w, device="cpu"))
+    a = workloads.to_numpy(batch)
+    g = torch.Generator().manual_seed(7)
+    W_ref = (batch.W.float().cpu() + 0.02 * torch.randn(batch.W.shape, generator=g)).to(torch.bfloat16)
+    lp_ref_oracle, _ = oais.logprob_train(a["H"], W_ref.float().numpy(), a["tokens"], a["mask"])
+    # reference pass on the GPU: the trainer kernel with the reference weights
+    ref_step = ais.AisStep(batch.T, w.d, w.V, w.P, w.G, w.block)
+    ais.logprob_fwd(ref_step.shape, ref_step.params, batch.H, W_ref.cuda(), None, None, None, None, batch.tokens, batch.mask,
+                    ref_step.lp_train, ref_step.lse_train, None, None, ref_step.status, ref_step.workspace)
+    torch.cuda.synchronize()
+    assert np.max(np.abs(ref_step.lp_train.cpu().numpy()[:batch.T] - lp_ref_oracle)) <= LP_ATOL
+    beta = 0.5
+    step = ais.AisStep(batch.T, w.d, w.V, w.P, w.G, w.block, params=ais.default_params(beta_kl=beta))
+    step.step(batch.H, batch.W, batch.tokens, batch.mask, batch.seq_offsets.cuda(), batch.rewards.cuda(),
+              lp_ref=ref_step.lp_train)
+    torch.cuda.synchronize()
+    ref = oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, w.block,
+                         lp_ref=lp_ref_oracle, beta_kl=beta)
+    d = _compare_all(batch, step, ref, a)
+    kl = oais.kl_term(ref["lp_train"], lp_ref_oracle, a["mask"], a["seq_offsets"], w.P, w.G)
+    assert kl > 1e-4 and abs(d["kl_ref"] - kl) <= 2e-2 * kl + 1e-6
+    # the term really moves the gradient: without it dH differs
+    plain = _run_gpu(batch)
+    assert _rel_fro(plain.dH.float().cpu().numpy(), step.dH.float().cpu().numpy()) > 1e-2
+
+
 def test_on_policy_recovery_on_gpu():
     """Feeding the trainer's log-probs as the rollout's: rho == 1 exactly, alpha == 0 (Proposition 'on-policy recovery')."""
     ais = _lib()
