@@ -70,11 +70,18 @@ def logprob_train(H, W, tokens, mask):
 def logprob_rollout(H, W, tokens, mask, block: int):
     """Rollout pass: weights and activations quantised to E4M3 per block along d
     (Section 2.1: 'we quantize both the weights and activations of the rollout model'),
-    then the same log-softmax.  Returns (lp, lse, (qH, sH, qW, sW))."""
-    qH, sH = e4m3.quantize_blocks(H, block)
-    qW, sW = e4m3.quantize_blocks(W, block)
-    Hq = e4m3.dequantize_blocks(qH, sH, block)
-    Wq = e4m3.dequantize_blocks(qW, sW, block)
+    then the same log-softmax.  block = 0 selects one scale per tensor (Appendix 'FP8 rollout': per-tensor
+    dynamic scaling).  Returns (lp, lse, (qH, sH, qW, sW))."""
+    if block == 0:
+        qH, sH = e4m3.quantize_tensor(H)
+        qW, sW = e4m3.quantize_tensor(W)
+        Hq = e4m3.decode(qH) * np.float64(sH)
+        Wq = e4m3.decode(qW) * np.float64(sW)
+    else:
+        qH, sH = e4m3.quantize_blocks(H, block)
+        qW, sW = e4m3.quantize_blocks(W, block)
+        Hq = e4m3.dequantize_blocks(qH, sH, block)
+        Wq = e4m3.dequantize_blocks(qW, sW, block)
     lp, lse = log_softmax_gather(logits(Hq, Wq), tokens, mask)
     return lp, lse, (qH, sH, qW, sW)
 

@@ -121,6 +121,23 @@ def quantize_blocks(x, block: int):
     return codes, scales
 
 
+def quantize_tensor(x):
+    """Per-tensor dynamic scaling (what the paper's own rollouts used): one scale s = fl32(max|x| / 448) for the
+    whole matrix, same code rule as quantize_blocks.  Returns (codes uint8 [R, K], scale float32 scalar)."""
+    x32 = np.asarray(x, dtype=np.float32)
+    R, K = x32.shape
+    amax = np.float32(np.max(np.abs(x32))) if x32.size else np.float32(0)
+    s = np.float32(1.0) if amax == 0 else (amax / np.float32(E4M3_MAX)).astype(np.float32)
+    rows = max(1, (1 << 22) // max(K, 1))
+    parts = []
+    for r0 in range(0, max(R, 1), rows):
+        with np.errstate(over="ignore"):
+            quot = (x32[r0:r0 + rows] / s).astype(np.float32)
+        parts.append(encode(np.clip(quot, -3.0e38, 3.0e38).astype(np.float32)))
+    codes = np.concatenate(parts, axis=0).reshape(R, K) if parts else np.zeros((R, K), np.uint8)
+    return codes, np.float32(s)
+
+
 def dequantize_blocks(codes, scales, block: int) -> np.ndarray:
     """codes [R, K], scales [R, K // block] -> float64 [R, K] = decode(q) * s (exact product)."""
     codes = np.asarray(codes, dtype=np.uint8)

@@ -188,3 +188,18 @@ def test_block_axis_is_last_axis_only():
     diff = (s0 != s1)
     assert diff.sum() == 1 and diff[2, 1]
     assert np.array_equal(c0[:, :128], c1[:, :128]) and np.array_equal(c0[[0, 1, 3]], c1[[0, 1, 3]])
+
+
+def test_per_tensor_quantisation():
+    """One scale for the whole matrix: equals block quantisation of the flattened matrix as a single block; the
+    global maximum lands on +-448; an all-zero matrix gets scale 1."""
+    rng = np.random.default_rng(9)
+    x = _bf16_round(rng.normal(size=(6, 96)) * 3)
+    codes, s = e4m3.quantize_tensor(x)
+    c1, s1 = e4m3.quantize_blocks(x.reshape(1, -1), x.size)
+    assert s == s1[0, 0] and np.array_equal(codes.reshape(1, -1), c1)
+    assert s == np.float32(np.abs(x).max()) / np.float32(448)
+    i = np.unravel_index(np.abs(x).argmax(), x.shape)
+    assert codes[i] & 0x7F == 0x7E
+    z, sz = e4m3.quantize_tensor(np.zeros((3, 8), np.float32))
+    assert sz == 1.0 and not z.any()
