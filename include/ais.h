@@ -64,7 +64,8 @@ typedef struct ais_shape {
     int32_t V;            /* vocabulary size                                                 */
     int32_t P;            /* prompts in the batch                                            */
     int32_t G;            /* responses per prompt; sequence s belongs to prompt s / G        */
-    int32_t fp8_block;    /* elements along d sharing one FP8 scale: 32, 64 or 128           */
+    int32_t fp8_block;    /* elements along d sharing one FP8 scale: 32, 64 or 128;
+                             0 = one scale per tensor (ais_quantize_fp8_tensor)              */
     int32_t P_total;      /* prompts over all data-parallel ranks (loss normaliser); 0 = P    */
     int64_t ldh;          /* row stride of H (and of its codes) in elements                  */
     int64_t ldw;          /* row stride of W (and of its codes) in elements                  */
@@ -139,6 +140,16 @@ size_t ais_workspace_min_bytes(const ais_shape* shape, const ais_params* params)
  */
 int ais_quantize_fp8(const void* x, int64_t rows, int64_t cols, int64_t ld, int block,
                      uint8_t* codes, int64_t ldq, float* scales, int64_t lds, void* stream);
+
+/*
+ * Per-tensor dynamic scaling, the setting of the paper's own rollouts (Appendix "FP8 rollout"): one scale
+ * s = fl32(max|x| / 448) for the whole matrix (s = 1 for an all-zero matrix), same code rule.  `scale` is one
+ * float on the device (written).  With shape->fp8_block == 0, ais_logprob_fwd takes such codes and reads sH / sW
+ * as pointers to one float each (ldsH / ldsW are ignored); the contraction then accumulates entirely in tensor
+ * memory and the two scales are applied once per logit.
+ */
+int ais_quantize_fp8_tensor(const void* x, int64_t rows, int64_t cols, int64_t ld,
+                            uint8_t* codes, int64_t ldq, float* scale, void* stream);
 
 /*
  * Trainer and rollout log-probabilities (Algorithm 1: "full-precision log-probs" and the sampler's

@@ -64,6 +64,8 @@ def lib() -> C.CDLL:
             f.argtypes = [C.POINTER(Shape), C.POINTER(Params)]
         L.ais_quantize_fp8.restype = C.c_int
         L.ais_quantize_fp8.argtypes = [vp, i64, i64, i64, C.c_int, vp, i64, vp, i64, vp]
+        L.ais_quantize_fp8_tensor.restype = C.c_int
+        L.ais_quantize_fp8_tensor.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp]
         L.ais_logprob_fwd.restype = C.c_int
         L.ais_logprob_fwd.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, i64, vp, vp, i64, vp, vp,
                                       vp, vp, vp, vp, vp, vp, sz, vp]
@@ -129,6 +131,12 @@ def quantize_fp8(x: torch.Tensor, block: int, codes: torch.Tensor | None = None,
     rows, cols = x.shape
     if codes is None:
         codes = torch.empty(rows, cols, dtype=torch.uint8, device=x.device)
+    if block == 0:                                   # one scale per tensor; scales holds it in its first element
+        if scales is None:
+            scales = torch.empty(1, 4, dtype=torch.float32, device=x.device)
+        _check(lib().ais_quantize_fp8_tensor(_ptr(x), rows, cols, x.stride(0), _ptr(codes), codes.stride(0), _ptr(scales),
+                                             _stream(x)), "ais_quantize_fp8_tensor")
+        return codes, scales
     if scales is None:
         lds = (rows + 3) // 4 * 4
         scales = torch.empty(cols // block, max(lds, 4), dtype=torch.float32, device=x.device)
@@ -211,7 +219,7 @@ class AisStep:
         self.params = params or default_params()
         S = P * G
         dev = self.device
-        nkb = d // fp8_block
+        nkb = d // fp8_block if fp8_block else 1
         ws = workspace_bytes(self.shape, self.params)
         if ws == 0:
             raise AisError("invalid shape or parameters")

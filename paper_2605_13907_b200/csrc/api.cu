@@ -77,8 +77,8 @@ int check_shape(const ais_shape* s) {
     if (s->T < 0 || s->T > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
     if (s->d <= 0 || s->V <= 0 || s->P <= 0 || s->G <= 0) return AIS_ERR_SHAPE;
     if (s->d % 128 != 0 || s->V % 8 != 0) return AIS_ERR_SHAPE;
-    if (s->fp8_block != 32 && s->fp8_block != 64 && s->fp8_block != 128) return AIS_ERR_SHAPE;
-    if (s->d % s->fp8_block != 0) return AIS_ERR_SHAPE;
+    if (s->fp8_block != 0 && s->fp8_block != 32 && s->fp8_block != 64 && s->fp8_block != 128) return AIS_ERR_SHAPE;
+    if (s->fp8_block != 0 && s->d % s->fp8_block != 0) return AIS_ERR_SHAPE;
     if (s->ldh < s->d || s->ldw < s->d) return AIS_ERR_SHAPE;
     if (s->ldh % 16 != 0 || s->ldw % 16 != 0) return AIS_ERR_ALIGN;
     if (static_cast<int64_t>(s->P) * s->G > (1 << 24)) return AIS_ERR_SHAPE;
@@ -202,6 +202,19 @@ int ais_quantize_fp8(const void* x, int64_t rows, int64_t cols, int64_t ld, int 
                : AIS_ERR_DEVICE;
 }
 
+int ais_quantize_fp8_tensor(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq, float* scale,
+                            void* stream) {
+    if (!x || !codes || !scale) return AIS_ERR_NULL;
+    if (rows < 0 || cols < 0 || cols % 8 != 0 || ld < cols || ldq < cols) return AIS_ERR_SHAPE;
+    if (ld % 8 != 0 || ldq % 8 != 0 || !aligned(x, 16) || !aligned(codes, 8) || !aligned(scale, 4)) return AIS_ERR_ALIGN;
+    if (rows > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
+    int st = device_setup(nullptr);
+    if (st != AIS_OK) return st;
+    return launch_quantize_tensor(x, rows, cols, ld, codes, ldq, scale, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? AIS_OK
+               : AIS_ERR_DEVICE;
+}
+
 int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void* H, const void* W, const uint8_t* qH,
                     const float* sH, int64_t ldsH, const uint8_t* qW, const float* sW, int64_t ldsW, const int32_t* tokens,
                     const uint8_t* mask, float* lp_train, float* lse_train, float* lp_roll, float* lse_roll,
@@ -215,10 +228,14 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     if (do_train && (!H || !W)) return AIS_ERR_NULL;
     if (do_roll && (!qH || !sH || !qW || !sW)) return AIS_ERR_NULL;
     if (do_train && (!aligned(H, 16) || !aligned(W, 16))) return AIS_ERR_ALIGN;
+    const bool per_tensor = shape->fp8_block == 0;
     if (do_roll) {
-        if (!aligned(qH, 16) || !aligned(qW, 16) || !aligned(sH, 16) || !aligned(sW, 16)) return AIS_ERR_ALIGN;
-        if (ldsH < shape->T || ldsW < shape->V) return AIS_ERR_SHAPE;
-        if (ldsH % 4 != 0 || ldsW % 4 != 0) return AIS_ERR_ALIGN;
+        if (!aligned(qH, 16) || !aligned(qW, 16) || !aligned(sH, 4) || !aligned(sW, 4)) return AIS_ERR_ALIGN;
+        if (!per_tensor) {
+            if (!aligned(sH, 16) || !aligned(sW, 16)) return AIS_ERR_ALIGN;
+            if (ldsH < shape->T || ldsW < shape->V) return AIS_ERR_SHAPE;
+            if (ldsH % 4 != 0 || ldsW % 4 != 0) return AIS_ERR_ALIGN;
+        }
     }
     const Layout L = make_layout(shape, params);
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.off_diag) return AIS_ERR_WORKSPACE;
@@ -237,7 +254,7 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     a.ncols = shape->V;
     a.n_col_tiles = (shape->V + kBN - 1) / kBN;
     a.nsplit = L.nsplit;
-    a.sgroups = 128 / shape->fp8_block;
+    a.sgroups = per_tensor ? 1 : 128 / shape->fp8_block;
     a.tokens = tokens;
     a.mask = mask;
     a.part_m = reinterpret_cast<float*>(ws + L.off_part_m);
@@ -260,7 +277,19 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
             cudaSuccess)
             return AIS_ERR_DEVICE;
     }
-    if (do_roll) {
+    if (do_roll && per_tensor) {
+        // one scale per tensor: the whole contraction accumulates in tensor memory, the scales meet in the epilogue
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
+            return AIS_ERR_DEVICE;
+        a.ksteps = shape->d / 128;
+        a.scale_a = sH;
+        a.scale_b = sW;
+        if (launch_lmhead(kFwdFp8T, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
+        if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_roll, lse_roll, dev_status, s) !=
+            cudaSuccess)
+            return AIS_ERR_DEVICE;
+    } else if (do_roll) {
         const uint64_t nkb = d / shape->fp8_block;
         if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
             !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||

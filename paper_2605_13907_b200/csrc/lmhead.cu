@@ -168,7 +168,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         uint8_t* sA = stage_base + st.idx * STG_BYTES;
                         uint8_t* sB = sA + A_BYTES;
                         mbar_expect_tx(&full[st.idx], STG_BYTES);
-                        const int kelem = (MODE == kFwdFp8) ? ks * 128 : ks * 64;
+                        const int kelem = (MODE == kFwdFp8 || MODE == kFwdFp8T) ? ks * 128 : ks * 64;
                         if (MODE == kBwdDh) {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kDhRows);
                             tma_load_2d(sA + kAStageBytes, &tmA, &full[st.idx], kelem, w.rt * kDhRows + kBM);
@@ -209,7 +209,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc =
-                (MODE == kFwdFp8) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
+                (MODE == kFwdFp8 || MODE == kFwdFp8T) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
                                   : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, 0, MODE == kBwdDh ? 1 : 0);
             Pipe st(STG), tb(NBUF);
             bool ok = true;
@@ -252,9 +252,12 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         } else {
                             const uint32_t dcol = tmem_base + tb.idx * kBN;
 #pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                mma_f16(dcol, smem_desc_sw128(sA + j * 32, 16, 1024), smem_desc_sw128(sB + j * 32, 16, 1024), idesc,
-                                        (ks > 0 || j > 0) ? 1u : 0u);
+                            for (int j = 0; j < 4; ++j) {
+                                const uint64_t adesc = smem_desc_sw128(sA + j * 32, 16, 1024);
+                                const uint64_t bdesc = smem_desc_sw128(sB + j * 32, 16, 1024);
+                                if (MODE == kFwdFp8T) mma_f8(dcol, adesc, bdesc, idesc, (ks > 0 || j > 0) ? 1u : 0u);
+                                else mma_f16(dcol, adesc, bdesc, idesc, (ks > 0 || j > 0) ? 1u : 0u);
+                            }
                         }
                         tc_commit(&empty[st.idx]);
                         st.advance();
@@ -330,6 +333,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (valid && (y < 0 || y >= a.ncols)) { flags |= AIS_FLAG_TOKEN_RANGE; y = -1; }
             }
             float m2 = kNegBig, s = 0.f, zy = -INFINITY;       // log2-domain running max, sum, target logit
+            const float tscale = (MODE == kFwdFp8T) ? (*a.scale_a) * (*a.scale_b) : 1.f;
             float lse2 = 0.f;
             if (MODE == kBwdP && row_ok) lse2 = a.lse[grow] * kLog2e;
 
@@ -394,8 +398,12 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         tmem_ld_wait(v);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(v[i]);
+                        if (MODE == kFwdFp8T) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) x[i] *= tscale;
+                        }
                     }
-                    if (MODE == kFwdBf16 || MODE == kFwdFp8) {
+                    if (MODE == kFwdBf16 || MODE == kFwdFp8 || MODE == kFwdFp8T) {
                         if (y >= col0 && y < col0 + 32) {
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
@@ -440,7 +448,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     tb.advance();
                 }
             }
-            if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8)) {
+            if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8 || MODE == kFwdFp8T)) {
                 const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow;
                 a.part_m[o] = m2 * kLn2;
                 a.part_s[o] = s;
@@ -478,6 +486,7 @@ cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& t
         case kFwdFp8:  return launch_mode<kFwdFp8>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
         case kBwdP:    return launch_mode<kBwdP>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
         case kBwdDh:   return launch_mode<kBwdDh>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
+        case kFwdFp8T: return launch_mode<kFwdFp8T>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
     }
     return cudaErrorInvalidValue;
 }
@@ -490,7 +499,9 @@ cudaError_t lmhead_prepare() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lmhead_kernel<kBwdP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(lmhead_kernel<kBwdDh>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(lmhead_kernel<kBwdDh>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(lmhead_kernel<kFwdFp8T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
 }  // namespace ais

@@ -11,7 +11,8 @@ enum LmheadMode : int {
     kFwdBf16 = 0,   // z = H W^T (bf16), streaming log-sum-exp + target pick -> partial triples
     kFwdFp8  = 1,   // z^ from E4M3 codes with per-block scale promotion, same epilogue
     kBwdP    = 2,   // recompute z (bf16), write u = softmax - onehot as bf16 scratch
-    kBwdDh   = 3    // dH = c (.) (U W), contraction over the vocabulary
+    kBwdDh   = 3,   // dH = c (.) (U W), contraction over the vocabulary
+    kFwdFp8T = 4    // E4M3 codes with one scale per tensor: whole contraction in tensor memory, one multiply after
 };
 
 constexpr int kBM = 128;                 // rows per tile (TMEM lanes)
@@ -52,6 +53,8 @@ struct LmheadArgs {
     const float* lse;      // recompute: log-sum-exp of the trainer pass
     __nv_bfloat16* U;      // recompute output / dH input scratch [rows_pad, ldU]
     int64_t ldU;
+    const float* scale_a;  // per-tensor FP8: the two scales (one float each, on the device)
+    const float* scale_b;
     const float* coef;     // dH: per-row factor c_t
     __nv_bfloat16* dH;
     int64_t lddh;

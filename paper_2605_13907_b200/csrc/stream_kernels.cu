@@ -125,6 +125,61 @@ __global__ void __launch_bounds__(kQThreads) quantize_kernel(const __nv_bfloat16
 }
 
 // ------------------------------------------------------------------------------------------------
+// Per-tensor dynamic scaling: one scale for the whole matrix.  Pass 1 folds max|x| (as a bf16 bit pattern; the
+// patterns of non-negative values order like the values, so an integer atomicMax is exact and order-free)
+// into the word that will hold the scale, pass 2 turns it into s = amax / 448, pass 3 quantises.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) tensor_amax_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols, int64_t ld,
+                                                           uint32_t* __restrict__ amax_bits) {
+    const int64_t vec_per_row = cols / 8;
+    const int64_t total = rows * vec_per_row;
+    uint32_t m = 0;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = i / vec_per_row, c = (i % vec_per_row) * 8;
+        const uint4 w = __ldg(reinterpret_cast<const uint4*>(x + r * ld + c));
+        m = __vmaxu2(m, __vmaxu2(__vmaxu2(w.x & 0x7FFF7FFFu, w.y & 0x7FFF7FFFu), __vmaxu2(w.z & 0x7FFF7FFFu, w.w & 0x7FFF7FFFu)));
+    }
+    m = max(m & 0xFFFFu, m >> 16);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if ((threadIdx.x & 31) == 0 && m != 0u) atomicMax(amax_bits, m);
+}
+
+__global__ void tensor_scale_kernel(uint32_t* scale_word) {
+    const uint32_t m = *scale_word;                        // bf16 pattern of max|x|
+    const float s = (m == 0u) ? 1.0f : __fdiv_rn(__uint_as_float(m << 16), 448.0f);
+    *reinterpret_cast<float*>(scale_word) = s;
+}
+
+__global__ void __launch_bounds__(256) tensor_quantize_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols,
+                                                               int64_t ld, uint8_t* __restrict__ codes, int64_t ldq,
+                                                               const float* __restrict__ scale) {
+    const float s = *scale;
+    const bool fast = s > 0x1p-100f && s < 0x1p100f;
+    const float y = fast ? __frcp_rn(s) : 0.f;
+    const int64_t vec_per_row = cols / 8;
+    const int64_t total = rows * vec_per_row;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = i / vec_per_row, c = (i % vec_per_row) * 8;
+        const uint4 raw = __ldg(reinterpret_cast<const uint4*>(x + r * ld + c));
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        float qv[8];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xFFFF0000u);
+            qv[2 * k] = fast ? exact_div(lo, s, y) : slow_div(lo, s);
+            qv[2 * k + 1] = fast ? exact_div(hi, s, y) : slow_div(hi, s);
+        }
+        uint2 out;
+        out.x = static_cast<uint32_t>(cvt_e4m3x2(qv[1], qv[0])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[3], qv[2])) << 16);
+        out.y = static_cast<uint32_t>(cvt_e4m3x2(qv[5], qv[4])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[7], qv[6])) << 16);
+        *reinterpret_cast<uint2*>(codes + r * ldq + c) = out;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Merge of the per-split (max, sum-exp, target-logit) triples into lp and lse.
 // ------------------------------------------------------------------------------------------------
 __global__ void combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_s,
@@ -406,6 +461,19 @@ cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t l
         case 128: quantize_kernel<128><<<grid, kQThreads, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scales, lds); break;
         default: return cudaErrorInvalidValue;
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_tensor(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,
+                                   float* scale, cudaStream_t stream) {
+    cudaError_t e = cudaMemsetAsync(scale, 0, sizeof(float), stream);
+    if (e != cudaSuccess) return e;
+    const __nv_bfloat16* xp = static_cast<const __nv_bfloat16*>(x);
+    const int64_t total = rows * (cols / 8);
+    const int blocks = static_cast<int>(total <= 0 ? 1 : ((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16));
+    if (total > 0) tensor_amax_kernel<<<blocks, 256, 0, stream>>>(xp, rows, cols, ld, reinterpret_cast<uint32_t*>(scale));
+    tensor_scale_kernel<<<1, 1, 0, stream>>>(reinterpret_cast<uint32_t*>(scale));
+    if (total > 0) tensor_quantize_kernel<<<blocks, 256, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scale);
     return cudaGetLastError();
 }
 

@@ -16,6 +16,10 @@ constexpr int kNumMoments = 12;
 cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes,
                             int64_t ldq, float* scales, int64_t lds, cudaStream_t stream);
 
+// One scale for the whole matrix (written to *scale on the device), then the codes.
+cudaError_t launch_quantize_tensor(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,
+                                   float* scale, cudaStream_t stream);
+
 // lp[t] = z_y - lse, lse[t] from nparts partial triples laid out [nparts][part_ld].
 cudaError_t launch_combine(const float* part_m, const float* part_s, const float* part_z, int nparts, int64_t part_ld,
                            const uint8_t* mask, int64_t T, float* lp, float* lse, uint32_t* status, cudaStream_t stream);

@@ -234,6 +234,34 @@ def test_kl_term_on_gpu():
     assert _rel_fro(plain.dH.float().cpu().numpy(), step.dH.float().cpu().numpy()) > 1e-2
 
 
+@pytest.mark.parametrize("case", ["tiny", "ragged"])
+def test_per_tensor_fp8_scaling(case):
+    """fp8_block = 0: one scale per tensor (the paper's own rollout setting).  Codes and the two scales bit-exact,
+    the rest of the path within the usual tolerances."""
+    ais = _lib()
+    base = workloads.WORKLOADS["tiny"]
+    w = workloads.scaled(base, block=0) if case == "tiny" else \
+        workloads.scaled(base, block=0, d=384, V=1336, P=3, G=4, lengths="uniform:5:90", seed=81)
+    batch = _to_cuda(workloads.make_batch(w, device="cpu"))
+    step = _run_gpu(batch)
+    a = workloads.to_numpy(batch)
+    ref = oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, 0)
+    T = batch.T
+    assert np.array_equal(step.qH.cpu().numpy()[:T], ref["qH"]) and np.array_equal(step.qW.cpu().numpy(), ref["qW"])
+    assert np.float32(step.sH[0, 0].item()).view(np.uint32) == np.float32(ref["sH"]).view(np.uint32)
+    assert np.float32(step.sW[0, 0].item()).view(np.uint32) == np.float32(ref["sW"]).view(np.uint32)
+    assert np.max(np.abs(step.lp_roll.cpu().numpy()[:T] - ref["lp_roll"])) <= LP_ATOL
+    assert np.max(np.abs(step.lp_train.cpu().numpy()[:T] - ref["lp_train"])) <= LP_ATOL
+    d = step.read_diag()
+    assert abs(d["alpha"] - ref["diag"]["alpha"]) <= ALPHA_ATOL and int(step.status.item()) == 0
+    dH = step.dH.float().cpu().numpy()[:T].astype(np.float64)
+    assert _rel_fro(dH, ref["dH"]) <= DH_REL
+    # degenerate input: an all-zero tensor gets scale 1 and zero codes
+    z = torch.zeros(8, 128, dtype=torch.bfloat16, device="cuda")
+    codes, scale = ais.quantize_fp8(z, 0)
+    assert float(scale[0, 0]) == 1.0 and not codes.any()
+
+
 def test_on_policy_recovery_on_gpu():
     """Feeding the trainer's log-probs as the rollout's: rho == 1 exactly, alpha == 0 (Proposition 'on-policy recovery')."""
     ais = _lib()
