@@ -254,6 +254,18 @@ def grad_hidden(H, W, tokens, c) -> np.ndarray:
     return p @ np.asarray(W, np.float64)
 
 
+def grad_weight(H, W, tokens, c) -> np.ndarray:
+    """dW[v, :] = sum_t c_t (softmax(z_t)[v] - [v = y_t]) H[t, :]   in float64 (same layout as W: [V, d])."""
+    z = logits(H, W)
+    z = z - z.max(axis=1, keepdims=True)
+    p = np.exp(z)
+    p /= p.sum(axis=1, keepdims=True)
+    T = z.shape[0]
+    p[np.arange(T), np.asarray(tokens, np.int64)] -= 1.0
+    p *= np.asarray(c, np.float64)[:, None]
+    return p.T @ np.asarray(H, np.float64)
+
+
 # --------------------------------------------------------------------------- whole path
 def full_path(H, W, tokens, mask, seq_offsets, rewards, P: int, G: int, block: int,
               params: Params | None = None, lp_old=None, want_grad: bool = True, lp_ref=None, beta_kl: float = 0.0) -> dict:
@@ -275,4 +287,5 @@ def full_path(H, W, tokens, mask, seq_offsets, rewards, P: int, G: int, block: i
                adv=adv, rho=rho, wbar=wbar, w_tilde=w_tilde, diag=diag, loss=loss, c=c)
     if want_grad:
         out["dH"] = grad_hidden(H, W, tokens, c)
+        out["dW"] = grad_weight(H, W, tokens, c)
     return out

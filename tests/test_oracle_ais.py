@@ -352,6 +352,35 @@ def test_kl_term_value_sign_and_gradient():
     assert np.linalg.norm(ais.grad_hidden(H, W, tok, c1 - c0)) > 0                 # the KL part is not a no-op
 
 
+def test_weight_gradient_matches_central_differences():
+    """dW against central differences of the loss in every entry of W (clip active, KL term on)."""
+    H, W, tok, mask, offs, rewards, P, G = _tiny_problem(seed=18, T=12, d=5, V=7)
+    rng = np.random.default_rng(19)
+    adv = ais.advantages(rewards, G)
+    w_tilde = 1.0 + 0.5 * (np.minimum(np.exp(rng.normal(0, 0.5, len(tok))), 5.0) - 1.0)
+    lp0, _ = ais.logprob_train(H, W, tok, mask)
+    lp_old = lp0 + 0.3 * rng.choice([-1.0, 1.0], len(tok))
+    lp_ref = lp0 + rng.normal(0, 0.3, len(tok))
+
+    def f(Wx):
+        lp, _ = ais.logprob_train(H, Wx, tok, mask)
+        return ais.loss_and_coeff(lp, lp_old, mask, offs, adv, w_tilde, P, G, 0.2, lp_ref=lp_ref, beta_kl=0.3)[0]
+    _, c = ais.loss_and_coeff(lp0, lp_old, mask, offs, adv, w_tilde, P, G, 0.2, lp_ref=lp_ref, beta_kl=0.3)
+    dW = ais.grad_weight(H, W, tok, c)
+    assert dW.shape == W.shape
+    num = np.zeros_like(W)
+    h = 1e-5
+    for v in range(W.shape[0]):
+        for k in range(W.shape[1]):
+            Wp, Wm = W.copy(), W.copy()
+            Wp[v, k] += h
+            Wm[v, k] -= h
+            num[v, k] = (f(Wp) - f(Wm)) / (2 * h)
+    assert np.linalg.norm(dW - num) <= 1e-6 * np.linalg.norm(num) + 1e-10
+    # columns of (p - onehot) sum to zero over the vocabulary, so the rows of dW sum to zero over v
+    assert np.abs(dW.sum(axis=0)).max() < 1e-12
+
+
 def test_logit_gradient_rows_sum_to_zero_and_weight_layout():
     H, W, tok, mask, offs, rewards, P, G = _tiny_problem(seed=12)
     c = np.random.default_rng(0).normal(size=len(tok))
