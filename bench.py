@@ -155,6 +155,9 @@ def run_ours(args) -> None:
     rew = batch.rewards.to(dev)
     stream = torch.cuda.current_stream(dev)
 
+    # variant (not the headline step): also produce the LM-head weight gradient, one more T x d x V pass
+    dW_buf = torch.empty(w.V, w.d, dtype=torch.float32, device=dev) if args.with_dw else None
+
     def one_step(ev=None):
         marks = []
 
@@ -175,7 +178,7 @@ def run_ours(args) -> None:
         mark()
         step.diagnose(batch.mask, offs, rew)
         mark()
-        step.backward(batch.H, batch.W, batch.tokens, batch.mask, offs)
+        step.backward(batch.H, batch.W, batch.tokens, batch.mask, offs, dW=dW_buf)
         mark()
         if ev is not None:
             ev.append(marks)
@@ -266,7 +269,7 @@ def run_ours(args) -> None:
         blk_rows = (step.workspace.numel() - fixed) // (_ld_u(w.V) * 2) // 128 * 128
         blk_rows = max(128, min(blk_rows, (T + 127) // 128 * 128))
         chunks = -(-T // blk_rows)
-        launches = (2 if w.block else 6) + 2 + 2 + (4 if world == 1 else 5) + 3 + 2 * chunks
+        launches = (2 if w.block else 6) + 2 + 2 + (4 if world == 1 else 5) + 3 + (3 if args.with_dw else 2) * chunks
         out = {
             "metric": METRIC, "value": tokens_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -281,7 +284,7 @@ def run_ours(args) -> None:
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": TRAFFIC_BF16_FWD.get(args.workload) if not args.prompts else None,
                          "peak_source": peaks["source"] + " bf16 sustained (kernel timed inside a long step)",
                          "passes": {"fwd_roll_fp8_tflops": flops_pass / (seg["fwd_roll_fp8"] * 1e-3) / 1e12,
-                                    "bwd_two_passes_tflops": 2 * flops_pass / (seg["loss_bwd"] * 1e-3) / 1e12,
+                                    "bwd_two_passes_tflops": (3 if args.with_dw else 2) * flops_pass / (seg["loss_bwd"] * 1e-3) / 1e12,
                                     "quantize_gbs": (T + w.V) * w.d * (3.03 if w.block else 5.0) / (seg["quantize"] * 1e-3) / 1e9}},
             "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches * args.steps,
@@ -331,6 +334,7 @@ def main() -> None:
     ap.add_argument("--workspace-gb", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (small profiling case)")
+    ap.add_argument("--with-dw", action="store_true", help="variant: ais_loss_bwd also writes dW (a fifth tensor-core pass)")
     ap.add_argument("--fp8-per-tensor", action="store_true",
                     help="variant (not the headline workload): per-tensor dynamic FP8 scaling instead of per-block scales")
     args = ap.parse_args()

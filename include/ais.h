@@ -220,13 +220,18 @@ int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const do
  *     loss += beta_kl sum_s 1/(P G n_s) sum_t kl_t ,   c_t -= mask[t] beta_kl (1 - r) / (P G n_s)
  * The softmax is recomputed from H, W and lse_train; w_tilde, A, lp_old and lp_ref are constants.
  * dH [T, ldh] bf16 (written, zero rows where mask = 0), loss: one float on the device (may be NULL),
- * diag: if not NULL its `loss` field is written too.
+ * diag: if not NULL its `loss` and `kl_ref` fields are written too.
+ * dW (may be NULL): gradient with respect to the LM head in W's layout, [V, lddw] fp32,
+ *     dW[v,:] = sum_t c_t (softmax(z[t,:])[v] - [v == tokens[t]]) H[t,:]
+ * overwritten when dw_accumulate == 0, added to otherwise (micro-batch accumulation); costs one more
+ * T x d x V tensor-core pass over the scratch that dH uses.
  */
 int ais_loss_bwd(const ais_shape* shape, const ais_params* params,
                  const void* H, const void* W, const int32_t* tokens, const uint8_t* mask,
                  const int32_t* seq_offsets, const float* lse_train, const float* lp_train,
                  const float* lp_old, const float* lp_ref, const float* adv, const float* w_tilde,
                  void* dH, float* loss, ais_diag* diag,
+                 float* dW, int64_t lddw, int dw_accumulate,
                  uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*

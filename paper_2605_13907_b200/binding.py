@@ -72,7 +72,7 @@ def lib() -> C.CDLL:
         L.ais_diagnostics.restype = C.c_int
         L.ais_diagnostics.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.ais_loss_bwd.restype = C.c_int
-        L.ais_loss_bwd.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 15 + [vp, sz, vp]
+        L.ais_loss_bwd.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 15 + [i64, C.c_int] + [vp, vp, sz, vp]
         L.ais_diag_moments.restype = C.c_int
         L.ais_diag_moments.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 8 + [vp, sz, vp]
         L.ais_diag_finalize.restype = C.c_int
@@ -178,12 +178,13 @@ def diag_finalize(shape: Shape, params: Params, moments, lp_train, lp_roll, mask
 
 
 def loss_bwd(shape: Shape, params: Params, H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, adv, w_tilde, dH, loss,
-             diag, dev_status, workspace, lp_ref=None):
+             diag, dev_status, workspace, lp_ref=None, dW=None, dw_accumulate: bool = False):
     _require_cuda(H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, lp_ref, adv, w_tilde, dH, loss, diag, dev_status,
-                  workspace)
+                  workspace, dW)
     _check(lib().ais_loss_bwd(C.byref(shape), C.byref(params), _ptr(H), _ptr(W), _ptr(tokens), _ptr(mask), _ptr(seq_offsets),
                               _ptr(lse_train), _ptr(lp_train), _ptr(lp_old), _ptr(lp_ref), _ptr(adv), _ptr(w_tilde), _ptr(dH), _ptr(loss),
-                              _ptr(diag), _ptr(dev_status), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                              _ptr(diag), _ptr(dW), dW.stride(0) if dW is not None else 0, 1 if dw_accumulate else 0,
+                              _ptr(dev_status), _ptr(workspace), workspace.numel() * workspace.element_size(),
                               _stream(workspace)), "ais_loss_bwd")
 
 
@@ -274,9 +275,10 @@ class AisStep:
         _dist.allreduce_moments(self.moments, self.group)
         diag_finalize(self.shape, self.params, self.moments, self.lp_train, self.lp_roll, mask, self.rho, self.w_tilde, self.diag)
 
-    def backward(self, H, W, tokens, mask, seq_offsets, lp_old=None, lp_ref=None) -> None:
+    def backward(self, H, W, tokens, mask, seq_offsets, lp_old=None, lp_ref=None, dW=None, dw_accumulate: bool = False) -> None:
         loss_bwd(self.shape, self.params, H, W, tokens, mask, seq_offsets, self.lse_train, self.lp_train, lp_old, self.adv,
-                 self.w_tilde, self.dH, self.loss, self.diag, self.status, self.workspace, lp_ref=lp_ref)
+                 self.w_tilde, self.dH, self.loss, self.diag, self.status, self.workspace, lp_ref=lp_ref, dW=dW,
+                 dw_accumulate=dw_accumulate)
 
     def step(self, H, W, tokens, mask, seq_offsets, rewards, lp_old=None, requantize_w: bool = True, lp_ref=None) -> None:
         self.forward(H, W, tokens, mask, requantize_w)

@@ -374,7 +374,7 @@ int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const do
 int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H, const void* W, const int32_t* tokens,
                  const uint8_t* mask, const int32_t* seq_offsets, const float* lse_train, const float* lp_train,
                  const float* lp_old, const float* lp_ref, const float* adv, const float* w_tilde, void* dH, float* loss,
-                 ais_diag* diag,
+                 ais_diag* diag, float* dW, int64_t lddw, int dw_accumulate,
                  uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream) {
     int st = check_shape(shape);
     if (st != AIS_OK) return st;
@@ -382,6 +382,8 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
     if (st != AIS_OK) return st;
     if (!H || !W || !tokens || !mask || !seq_offsets || !lse_train || !lp_train || !adv || !w_tilde || !dH) return AIS_ERR_NULL;
     if (!aligned(H, 16) || !aligned(W, 16) || !aligned(dH, 16)) return AIS_ERR_ALIGN;
+    if (dW && (!aligned(dW, 16) || lddw % 4 != 0)) return AIS_ERR_ALIGN;
+    if (dW && lddw < shape->d) return AIS_ERR_SHAPE;
     const Layout L = make_layout(shape, params);
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.fixed_bytes + static_cast<size_t>(kBM) * L.u_row_bytes)
         return AIS_ERR_WORKSPACE;
@@ -454,6 +456,29 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
         units = a.n_row_tiles * a.n_col_tiles;
         if (launch_lmhead(kBwdDh, tmU, tmW_n, tmU, tmW_n, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
             return AIS_ERR_DEVICE;
+        if (dW) {
+            // dW (+)= U^T H over the rows of this pass: both operands are read with the rows as contraction axis;
+            // the maps end at `rows`, so rows the scratch still holds from an earlier pass read as zeros
+            CUtensorMap tmU_t, tmH_t;
+            if (!make_tmap(&tmU_t, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, U, V, static_cast<uint64_t>(rows), L.ldU * 2, 64, 64,
+                           CU_TENSOR_MAP_SWIZZLE_128B) ||
+                !make_tmap(&tmH_t, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Hc, d, static_cast<uint64_t>(rows), shape->ldh * 2, 64, 64,
+                           CU_TENSOR_MAP_SWIZZLE_128B))
+                return AIS_ERR_DEVICE;
+            LmheadArgs w = a;
+            w.rows = shape->V;
+            w.row0 = 0;
+            w.n_row_tiles = static_cast<int32_t>((shape->V + kDhRows - 1) / kDhRows);
+            w.ncols = shape->d;
+            w.n_col_tiles = (shape->d + kBN - 1) / kBN;
+            w.ksteps = static_cast<int32_t>((rows + 63) / 64);
+            w.dW = dW;
+            w.lddw = lddw;
+            w.dw_accumulate = (dw_accumulate || r0 > 0) ? 1 : 0;
+            units = w.n_row_tiles * w.n_col_tiles;
+            if (launch_lmhead(kBwdDw, tmU_t, tmH_t, tmU_t, tmH_t, w, units < num_sms ? units : num_sms, s) != cudaSuccess)
+                return AIS_ERR_DEVICE;
+        }
     }
     return AIS_OK;
 }

@@ -88,7 +88,7 @@ struct Unit {
 template <int MODE>
 __device__ __forceinline__ Unit decode_unit(const LmheadArgs& a, int u) {
     Unit w;
-    if (MODE == kBwdDh) {
+    if (MODE == kBwdDh || MODE == kBwdDw) {
         w.rt = u / a.n_col_tiles;
         w.t0 = u % a.n_col_tiles;
         w.t1 = w.t0 + 1;
@@ -123,13 +123,14 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBarriers);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    constexpr int STG = (MODE == kBwdDh) ? kDhStages : kStages;                 // depth of the stage ring
-    constexpr int STG_BYTES = (MODE == kBwdDh) ? kDhStageBytes : kStageBytes;
-    constexpr int A_BYTES = (MODE == kBwdDh) ? 2 * kAStageBytes : kAStageBytes;
-    constexpr int NBUF = (MODE == kBwdDh) ? 1 : 2;                              // accumulator sets that alternate
+    constexpr bool TWO_ACC = (MODE == kBwdDh || MODE == kBwdDw);                // two 128-row tiles per CTA, one B slice
+    constexpr int STG = TWO_ACC ? kDhStages : kStages;                          // depth of the stage ring
+    constexpr int STG_BYTES = TWO_ACC ? kDhStageBytes : kStageBytes;
+    constexpr int A_BYTES = TWO_ACC ? 2 * kAStageBytes : kAStageBytes;
+    constexpr int NBUF = TWO_ACC ? 1 : 2;                                       // accumulator sets that alternate
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int num_units = (MODE == kBwdDh) ? a.n_row_tiles * a.n_col_tiles : a.n_row_tiles * a.nsplit;
+    const int num_units = TWO_ACC ? a.n_row_tiles * a.n_col_tiles : a.n_row_tiles * a.nsplit;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
@@ -172,11 +173,17 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         if (MODE == kBwdDh) {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kDhRows);
                             tma_load_2d(sA + kAStageBytes, &tmA, &full[st.idx], kelem, w.rt * kDhRows + kBM);
+                        } else if (MODE == kBwdDw) {
+                            // A is U[t, v]: the output row v is the contiguous axis -> four 64-wide boxes of 64 rows t
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                tma_load_2d(sA + j * (kAStageBytes / 2), &tmA, &full[st.idx], w.rt * kDhRows + j * 64, kelem);
                         } else {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kBM);
                         }
-                        if (MODE == kBwdDh) {
-                            // B is W[v, n]: n (the output column) is the contiguous axis -> four 64-column boxes
+                        if (MODE == kBwdDh || MODE == kBwdDw) {
+                            // B is W[v, n] (dH) or H[t, n] (dW): n (the output column) is the contiguous axis -> four
+                            // 64-column boxes
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
                                 tma_load_2d(sB + j * (kBStageBytes / 4), &tmB, &full[st.idx], t * kBN + j * 64, kelem);
@@ -210,7 +217,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         if (lane == 0) {
             constexpr uint32_t idesc =
                 (MODE == kFwdFp8 || MODE == kFwdFp8T) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
-                                  : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, 0, MODE == kBwdDh ? 1 : 0);
+                                  : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, MODE == kBwdDw ? 1 : 0, TWO_ACC ? 1 : 0);
             Pipe st(STG), tb(NBUF);
             bool ok = true;
             for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
@@ -248,6 +255,17 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                 const uint32_t accum = (ks > 0 || j > 0) ? 1u : 0u;
                                 mma_f16(tmem_base, smem_desc_sw128(sA + j * 32, 16, 1024), bdesc, idesc, accum);
                                 mma_f16(tmem_base + kBN, smem_desc_sw128(sA + kAStageBytes + j * 32, 16, 1024), bdesc, idesc, accum);
+                            }
+                        } else if (MODE == kBwdDw) {
+                            // both operands have the contraction axis t as rows of 128 bytes: 16 rows (2048 bytes) per
+                            // MMA; 64-wide chunks of the output axis are 8 KB apart
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const uint64_t bdesc = smem_desc_sw128(sB + j * 2048, kBStageBytes / 4, 1024);
+                                const uint32_t accum = (ks > 0 || j > 0) ? 1u : 0u;
+                                mma_f16(tmem_base, smem_desc_sw128(sA + j * 2048, kAStageBytes / 2, 1024), bdesc, idesc, accum);
+                                mma_f16(tmem_base + kBN, smem_desc_sw128(sA + kAStageBytes + j * 2048, kAStageBytes / 2, 1024), bdesc,
+                                        idesc, accum);
                             }
                         } else {
                             const uint32_t dcol = tmem_base + tb.idx * kBN;
@@ -293,7 +311,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     const int64_t lrow2 = static_cast<int64_t>(w.rt) * kDhRows + sub * kBM + r_in_tile;
                     const bool in = lrow2 < a.rows;
                     const int64_t grow2 = a.row0 + lrow2;
-                    const float cf = in ? a.coef[grow2] : 0.f;
                     const uint32_t taddr2 = tmem_base + lane_addr + sub * kBN + half * 128;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -305,9 +322,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             uint32_t pk[16];
 #pragma unroll
                             for (int i = 0; i < 32; i += 2) {
-                                const float v0 = (cf == 0.f) ? 0.f : cf * __uint_as_float(v[i]);
-                                const float v1 = (cf == 0.f) ? 0.f : cf * __uint_as_float(v[i + 1]);
-                                pk[i >> 1] = pack_bf16(v0, v1);
+                                pk[i >> 1] = pack_bf16(__uint_as_float(v[i]), __uint_as_float(v[i + 1]));
                             }
                             uint4* dst = reinterpret_cast<uint4*>(a.dH + grow2 * a.lddh + col0);
 #pragma unroll
@@ -322,12 +337,50 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 tb.advance();
                 continue;
             }
+            if (MODE == kBwdDw) {
+                // one unit = 256 vocabulary rows x 256 columns of dW after the contraction over this launch's rows
+                if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int sub = 0; sub < 2; ++sub) {
+                    const int64_t vrow = static_cast<int64_t>(w.rt) * kDhRows + sub * kBM + r_in_tile;
+                    const bool in = vrow < a.rows;
+                    const uint32_t taddr2 = tmem_base + lane_addr + sub * kBN + half * 128;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int col0 = w.t0 * kBN + half * 128 + c * 32;
+                        uint32_t v[32];
+                        tmem_ld32(taddr2 + c * 32, v);
+                        tmem_ld_wait(v);
+                        if (in && col0 < a.ncols) {
+                            float4* dst = reinterpret_cast<float4*>(a.dW + vrow * a.lddw + col0);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                if (col0 + j * 4 < a.ncols) {
+                                    float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                           __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                                    if (a.dw_accumulate) {
+                                        const float4 old = dst[j];
+                                        o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                    }
+                                    dst[j] = o;
+                                }
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tempty[0]);
+                tb.advance();
+                continue;
+            }
             const int64_t lrow = static_cast<int64_t>(w.rt) * kBM + r_in_tile;   // row inside this launch
             const bool row_ok = lrow < a.rows;
             const int64_t grow = a.row0 + lrow;
             int y = -1;
             bool valid = false;
-            if (row_ok && MODE != kBwdDh) {
+            if (row_ok) {
                 y = a.tokens[grow];
                 valid = a.mask[grow] != 0;
                 if (valid && (y < 0 || y >= a.ncols)) { flags |= AIS_FLAG_TOKEN_RANGE; y = -1; }
@@ -335,7 +388,12 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             float m2 = kNegBig, s = 0.f, zy = -INFINITY;       // log2-domain running max, sum, target logit
             const float tscale = (MODE == kFwdFp8T) ? (*a.scale_a) * (*a.scale_b) : 1.f;
             float lse2 = 0.f;
-            if (MODE == kBwdP && row_ok) lse2 = a.lse[grow] * kLog2e;
+            float cf = 0.f;                                    // recompute: c_t, folded into the scratch
+            if (MODE == kBwdP && row_ok) {
+                lse2 = a.lse[grow] * kLog2e;
+                cf = a.coef[grow];
+                if (cf == 0.f) valid = false;                  // rows without gradient are written as exact zeros
+            }
 
             for (int t = w.t0; t < w.t1 && ok; ++t) {
                 const int col_base = t * kBN + half * 128;    // first output column of this thread's half
@@ -432,7 +490,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                 float p1 = valid ? ex2(fmaf(x[i + 1], kLog2e, -lse2)) : 0.f;
                                 if (col0 + i == y) p0 -= 1.f;
                                 if (col0 + i + 1 == y) p1 -= 1.f;
-                                pk[i >> 1] = pack_bf16(p0, p1);
+                                pk[i >> 1] = pack_bf16(valid ? cf * p0 : 0.f, valid ? cf * p1 : 0.f);
                             }
                             uint4* dst = reinterpret_cast<uint4*>(a.U + lrow * a.ldU + col0);
 #pragma unroll
@@ -487,6 +545,7 @@ cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& t
         case kBwdP:    return launch_mode<kBwdP>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
         case kBwdDh:   return launch_mode<kBwdDh>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
         case kFwdFp8T: return launch_mode<kFwdFp8T>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
+        case kBwdDw:   return launch_mode<kBwdDw>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
     }
     return cudaErrorInvalidValue;
 }
@@ -501,7 +560,9 @@ cudaError_t lmhead_prepare() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lmhead_kernel<kBwdDh>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(lmhead_kernel<kFwdFp8T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(lmhead_kernel<kFwdFp8T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(lmhead_kernel<kBwdDw>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
 }  // namespace ais

@@ -12,7 +12,8 @@ enum LmheadMode : int {
     kFwdFp8  = 1,   // z^ from E4M3 codes with per-block scale promotion, same epilogue
     kBwdP    = 2,   // recompute z (bf16), write u = softmax - onehot as bf16 scratch
     kBwdDh   = 3,   // dH = c (.) (U W), contraction over the vocabulary
-    kFwdFp8T = 4    // E4M3 codes with one scale per tensor: whole contraction in tensor memory, one multiply after
+    kFwdFp8T = 4,   // E4M3 codes with one scale per tensor: whole contraction in tensor memory, one multiply after
+    kBwdDw   = 5    // dW += U^T H, contraction over the rows (both operands read with the contraction axis as rows)
 };
 
 constexpr int kBM = 128;                 // rows per tile (TMEM lanes)
@@ -55,7 +56,10 @@ struct LmheadArgs {
     int64_t ldU;
     const float* scale_a;  // per-tensor FP8: the two scales (one float each, on the device)
     const float* scale_b;
-    const float* coef;     // dH: per-row factor c_t
+    const float* coef;     // recompute: per-row factor c_t folded into the scratch
+    float* dW;             // dW pass: [V, lddw] fp32
+    int64_t lddw;
+    int32_t dw_accumulate; // dW pass: add to what dW holds instead of overwriting it
     __nv_bfloat16* dH;
     int64_t lddh;
     uint32_t* status;

@@ -129,6 +129,20 @@ def test_fullsize_sampled_parity(name):
         if nz.any():      # row by row as well, so that one bad row cannot hide in the norm of the others
             rel = np.linalg.norm((dH - dH_ref)[nz], axis=1) / np.linalg.norm(dH_ref[nz], axis=1)
             assert rel.max() <= 2 * DH_REL
+
+        # ---- dW at full size: two identities that hold at any size.  The oracle cannot form dW here (it needs the
+        # softmax of every row), so: columns of dW sum to zero over the vocabulary (rows of softmax - onehot do), and
+        # <dW, W> = sum_t g_t . z_t = <dH, H> ties dW to the dH that was checked row by row above.
+        if name in ("qwen3_8b", "llada_8b"):
+            dW = torch.empty(w.V, w.d, dtype=torch.float32, device="cuda")
+            step.backward(batch.H, batch.W, batch.tokens, batch.mask, offs_d, dW=dW)
+            torch.cuda.synchronize()
+            assert int(step.status.item()) == 0
+            norm = float(dW.double().norm())
+            assert norm > 0 and float(dW.double().sum(dim=0).norm()) <= 2e-2 * norm
+            ip_w = float((dW.double() * batch.W.double()).sum())
+            ip_h = float((step.dH[:T].double() * batch.H.double()).sum())
+            assert abs(ip_w - ip_h) <= 1e-2 * max(abs(ip_h), 1e-12)
     finally:
         pool.terminate()
         pool.join()

@@ -262,6 +262,32 @@ def test_per_tensor_fp8_scaling(case):
     assert float(scale[0, 0]) == 1.0 and not codes.any()
 
 
+@pytest.mark.parametrize("case", ["tiny", "ragged_chunked"])
+def test_weight_gradient_on_gpu(case):
+    """dW = U^T H against the oracle; with the minimum workspace the rows go through in 128-row passes that
+    accumulate into dW; dw_accumulate adds a second micro-batch on top."""
+    ais = _lib()
+    base = workloads.WORKLOADS["tiny"]
+    w = base if case == "tiny" else workloads.scaled(base, d=384, V=1336, P=3, G=4, lengths="uniform:20:90", seed=91)
+    batch = _to_cuda(workloads.make_batch(w, device="cpu"))
+    a, ref = _oracle(batch)
+    step = ais.AisStep(batch.T, w.d, w.V, w.P, w.G, w.block, workspace_bytes_cap=(1 if case != "tiny" else None))
+    offs, rew = batch.seq_offsets.cuda(), batch.rewards.cuda()
+    dW = torch.full((w.V, w.d), 7.0, dtype=torch.float32, device="cuda")          # must be overwritten, not added to
+    step.forward(batch.H, batch.W, batch.tokens, batch.mask)
+    step.diagnose(batch.mask, offs, rew)
+    step.backward(batch.H, batch.W, batch.tokens, batch.mask, offs, dW=dW)
+    torch.cuda.synchronize()
+    assert int(step.status.item()) == 0
+    got = dW.cpu().numpy().astype(np.float64)
+    assert _rel_fro(got, ref["dW"]) <= DH_REL
+    dH = step.dH.float().cpu().numpy()[:batch.T].astype(np.float64)
+    assert _rel_fro(dH, ref["dH"]) <= DH_REL
+    step.backward(batch.H, batch.W, batch.tokens, batch.mask, offs, dW=dW, dw_accumulate=True)
+    torch.cuda.synchronize()
+    assert _rel_fro(dW.cpu().numpy().astype(np.float64), 2 * ref["dW"]) <= DH_REL
+
+
 def test_on_policy_recovery_on_gpu():
     """Feeding the trainer's log-probs as the rollout's: rho == 1 exactly, alpha == 0 (Proposition 'on-policy recovery')."""
     ais = _lib()
