@@ -147,6 +147,12 @@ def run_ours(args) -> None:
     if args.fp8_per_tensor:
         w = workloads.scaled(w, block=0)                              # variant: one FP8 scale per tensor
     batch = workloads.make_batch(w, device=dev)
+    if args.compact:
+        # scattered masks: pack the valid rows once per batch (inside the step for the end-to-end figure) and run on those
+        rc0 = ais.RowCompaction(batch.mask, batch.seq_offsets.to(dev), n_packed=batch.n_valid)
+        packed = workloads.Batch(w, rc0.gather_rows(batch.H), batch.W, rc0.gather(batch.tokens),
+                                 torch.ones(rc0.n, dtype=torch.uint8, device=dev), rc0.packed_offsets.cpu(), batch.rewards)
+        batch = packed
     T, n_valid = batch.T, batch.n_valid
     params = ais.default_params(vocab_chunk=w.vocab_chunk)
     step = ais.AisStep(T, w.d, w.V, w.P, w.G, w.block, device=dev, params=params, workspace_bytes_cap=args.workspace_gb << 30,
@@ -334,6 +340,8 @@ def main() -> None:
     ap.add_argument("--workspace-gb", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (small profiling case)")
+    ap.add_argument("--compact", action="store_true",
+                    help="pack the valid rows first (for workloads with scattered masks, e.g. llada_8b)")
     ap.add_argument("--with-dw", action="store_true", help="variant: ais_loss_bwd also writes dW (a fifth tensor-core pass)")
     ap.add_argument("--fp8-per-tensor", action="store_true",
                     help="variant (not the headline workload): per-tensor dynamic FP8 scaling instead of per-block scales")

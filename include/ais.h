@@ -235,6 +235,32 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params,
                  uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Row compaction for batches whose valid rows are scattered (masked-diffusion log-probabilities: only the masked
+ * positions of a response take part, Appendix "LLaDA Experiments").  The tensor-core passes work on tiles of 128
+ * consecutive rows, so scattered invalid rows cost as much as valid ones; packing the valid rows first makes the
+ * passes proportional to the number of valid rows.
+ *   ais_compact_index : n_valid_seq [S] (valid rows per sequence), packed_offsets [S+1] (their exclusive scan: row
+ *                       offsets of the packed batch) and row_index [>= N] (original row of packed row i, increasing
+ *                       inside every sequence; N = packed_offsets[S]).
+ *   ais_gather_rows   : dst[i,:] = src[row_index[i],:] for rows of row_bytes bytes (multiple of 16; strides in bytes).
+ *   ais_scatter_rows  : dst is zero-filled (dst_rows rows), then dst[row_index[i],:] = src[i,:].
+ *   ais_gather_words / ais_scatter_words : the same for vectors of 32-bit elements (tokens, log-probs, rho, w_tilde);
+ *                       the scatter first fills dst[0 .. dst_rows) with fill_bits (0 for log-probs, the bits of 1.0f
+ *                       for rho and w_tilde).
+ * The caller runs the path on the packed batch (T = N, mask all ones, seq_offsets = packed_offsets) and scatters
+ * what it needs back.  N is data dependent: the caller either knows it (it made the mask) or reads packed_offsets[S].
+ */
+int ais_compact_index(const uint8_t* mask, const int32_t* seq_offsets, int32_t S, int32_t* n_valid_seq,
+                      int32_t* packed_offsets, int32_t* row_index, void* stream);
+int ais_gather_rows(const void* src, int64_t src_stride_bytes, const int32_t* row_index, int64_t n, int64_t row_bytes,
+                    void* dst, int64_t dst_stride_bytes, void* stream);
+int ais_scatter_rows(const void* src, int64_t src_stride_bytes, const int32_t* row_index, int64_t n, int64_t row_bytes,
+                     void* dst, int64_t dst_stride_bytes, int64_t dst_rows, void* stream);
+int ais_gather_words(const void* src, const int32_t* row_index, int64_t n, void* dst, void* stream);
+int ais_scatter_words(const void* src, const int32_t* row_index, int64_t n, void* dst, int64_t dst_rows,
+                      uint32_t fill_bits, void* stream);
+
+/*
  * Trainer log-probabilities for callers that cannot hand over a workspace (the paper has no counterpart;
  * this is a packaging variant of the trainer pass of ais_logprob_fwd, same kernels, same results).
  *

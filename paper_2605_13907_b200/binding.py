@@ -77,6 +77,16 @@ def lib() -> C.CDLL:
         L.ais_diag_moments.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 8 + [vp, sz, vp]
         L.ais_diag_finalize.restype = C.c_int
         L.ais_diag_finalize.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 8
+        L.ais_compact_index.restype = C.c_int
+        L.ais_compact_index.argtypes = [vp, vp, C.c_int32, vp, vp, vp, vp]
+        L.ais_gather_rows.restype = C.c_int
+        L.ais_gather_rows.argtypes = [vp, i64, vp, i64, i64, vp, i64, vp]
+        L.ais_scatter_rows.restype = C.c_int
+        L.ais_scatter_rows.argtypes = [vp, i64, vp, i64, i64, vp, i64, i64, vp]
+        L.ais_gather_words.restype = C.c_int
+        L.ais_gather_words.argtypes = [vp, vp, i64, vp, vp]
+        L.ais_scatter_words.restype = C.c_int
+        L.ais_scatter_words.argtypes = [vp, vp, i64, vp, i64, C.c_uint32, vp]
         L.ais_logprob_train_static.restype = C.c_int
         L.ais_logprob_train_static.argtypes = [C.POINTER(Shape)] + [vp] * 8
         _lib = L
@@ -197,6 +207,54 @@ def logprob_train_static(shape: Shape, H, W, tokens, mask, lp_train, lse_train=N
 
 
 STATIC_MAX_ROWS = 16384
+
+
+class RowCompaction:
+    """Packing of the valid rows of a batch with a scattered mask, and the way back.
+
+    n_packed is the number of valid rows; pass it when known (the usual case: the caller made the mask), otherwise it
+    is read back from the device, which synchronises once.
+    """
+
+    def __init__(self, mask: torch.Tensor, seq_offsets: torch.Tensor, n_packed: int | None = None):
+        _require_cuda(mask, seq_offsets)
+        self.T = mask.numel()
+        S = seq_offsets.numel() - 1
+        dev = mask.device
+        self.n_valid_seq = torch.empty(S, dtype=torch.int32, device=dev)
+        self.packed_offsets = torch.empty(S + 1, dtype=torch.int32, device=dev)
+        self.row_index = torch.empty(max(self.T, 1), dtype=torch.int32, device=dev)
+        _check(lib().ais_compact_index(_ptr(mask), _ptr(seq_offsets), S, _ptr(self.n_valid_seq), _ptr(self.packed_offsets),
+                                       _ptr(self.row_index), _stream(mask)), "ais_compact_index")
+        self.n = int(self.packed_offsets[-1].item()) if n_packed is None else int(n_packed)
+
+    def gather_rows(self, src: torch.Tensor, dst: torch.Tensor | None = None) -> torch.Tensor:
+        if dst is None:
+            dst = torch.empty(max(self.n, 1), src.shape[1], dtype=src.dtype, device=src.device)
+        es = src.element_size()
+        _check(lib().ais_gather_rows(_ptr(src), src.stride(0) * es, _ptr(self.row_index), self.n, src.shape[1] * es, _ptr(dst),
+                                     dst.stride(0) * es, _stream(src)), "ais_gather_rows")
+        return dst
+
+    def scatter_rows(self, src: torch.Tensor, dst: torch.Tensor) -> torch.Tensor:
+        es = src.element_size()
+        _check(lib().ais_scatter_rows(_ptr(src), src.stride(0) * es, _ptr(self.row_index), self.n, src.shape[1] * es, _ptr(dst),
+                                      dst.stride(0) * es, dst.shape[0], _stream(src)), "ais_scatter_rows")
+        return dst
+
+    def gather(self, src: torch.Tensor) -> torch.Tensor:
+        """1-D tensor of 32-bit elements (tokens, float vectors)."""
+        dst = torch.empty(max(self.n, 1), dtype=src.dtype, device=src.device)
+        _check(lib().ais_gather_words(_ptr(src), _ptr(self.row_index), self.n, _ptr(dst), _stream(src)), "ais_gather_words")
+        return dst
+
+    def scatter(self, src: torch.Tensor, fill: float = 0.0) -> torch.Tensor:
+        import struct
+        dst = torch.empty(self.T, dtype=src.dtype, device=src.device)
+        bits = struct.unpack("<I", struct.pack("<f", fill))[0] if src.dtype == torch.float32 else int(fill) & 0xFFFFFFFF
+        _check(lib().ais_scatter_words(_ptr(src), _ptr(self.row_index), self.n, _ptr(dst), self.T, bits, _stream(src)),
+               "ais_scatter_words")
+        return dst
 
 
 def read_diag(diag_buf: torch.Tensor) -> dict:

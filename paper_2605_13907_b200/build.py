@@ -10,7 +10,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libais_b200.so")
-SOURCES = ["api.cu", "lmhead.cu", "stream_kernels.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "lmhead.cu", "stream_kernels.cu", "noalloc.cu", "compact.cu"]
 HEADERS = ["lmhead.cuh", "ptx.cuh", "stream_kernels.cuh", os.path.join("..", "..", "include", "ais.h")]
 
 
