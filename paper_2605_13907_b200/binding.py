@@ -271,10 +271,12 @@ class AisStep:
     """
 
     def __init__(self, T: int, d: int, V: int, P: int, G: int, fp8_block: int, device="cuda", params: Params | None = None,
-                 workspace_bytes_cap: int | None = None, want_grad: bool = True, group=None, P_total: int = 0):
+                 workspace_bytes_cap: int | None = None, want_grad: bool = True, group=None, P_total: int = 0,
+                 ldh: int | None = None, ldw: int | None = None):
         self.device = torch.device(device)
         self.group = group                       # torch.distributed process group: alpha over all its ranks
-        self.shape = make_shape(T, d, V, P, G, fp8_block, P_total=P_total)
+        ldh, ldw = ldh or d, ldw or d            # row strides of H / W; their codes and dH use the same strides
+        self.shape = make_shape(T, d, V, P, G, fp8_block, ldh=ldh, ldw=ldw, P_total=P_total)
         self.params = params or default_params()
         S = P * G
         dev = self.device
@@ -289,9 +291,9 @@ class AisStep:
             ws_all = ws_min + max(0, (T + 127) // 128 * 128 - 128) * ld_u * 2
             ws = max(ws_min, min(ws_all, workspace_bytes_cap))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
-        self.qH = torch.empty(max(T, 1), d, dtype=torch.uint8, device=dev)
+        self.qH = torch.empty(max(T, 1), ldh, dtype=torch.uint8, device=dev)[:, :d]
         self.sH = torch.empty(nkb, max((T + 3) // 4 * 4, 4), dtype=torch.float32, device=dev)
-        self.qW = torch.empty(V, d, dtype=torch.uint8, device=dev)
+        self.qW = torch.empty(V, ldw, dtype=torch.uint8, device=dev)[:, :d]
         self.sW = torch.empty(nkb, (V + 3) // 4 * 4, dtype=torch.float32, device=dev)
         f32 = dict(dtype=torch.float32, device=dev)
         self.lp_train = torch.empty(max(T, 1), **f32)
@@ -306,7 +308,7 @@ class AisStep:
         self.diag = torch.zeros((C.sizeof(Diag) + 7) // 8, dtype=torch.float64, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.moments = torch.zeros(NUM_MOMENTS, dtype=torch.float64, device=dev)
-        self.dH = torch.empty(max(T, 1), d, dtype=torch.bfloat16, device=dev) if want_grad else None
+        self.dH = torch.empty(max(T, 1), ldh, dtype=torch.bfloat16, device=dev)[:, :d] if want_grad else None
         self.w_quantized = False
 
     def quantize_weights(self, W: torch.Tensor) -> None:

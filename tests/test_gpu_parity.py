@@ -288,6 +288,40 @@ def test_weight_gradient_on_gpu(case):
     assert _rel_fro(dW.cpu().numpy().astype(np.float64), 2 * ref["dW"]) <= DH_REL
 
 
+def test_padded_leading_dimensions_and_empty_batch_of_rows():
+    """H and W as column slices of wider buffers (ldh, ldw > d): codes, dH and every tensor map follow the strides.
+    Also T = 0: every entry point accepts it and alpha comes out 0 with the EMPTY flag."""
+    ais = _lib()
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], d=256, V=776, lengths="uniform:20:70", seed=97)
+    b = workloads.make_batch(w, device="cpu")
+    a, ref = _oracle(b)
+    ldh, ldw = w.d + 64, w.d + 128
+    Hbig = torch.randn(b.T, ldh).to(torch.bfloat16).cuda()
+    Wbig = torch.randn(w.V, ldw).to(torch.bfloat16).cuda()
+    Hbig[:, :w.d] = b.H.cuda()
+    Wbig[:, :w.d] = b.W.cuda()
+    H, W = Hbig[:, :w.d], Wbig[:, :w.d]
+    step = ais.AisStep(b.T, w.d, w.V, w.P, w.G, w.block, ldh=ldh, ldw=ldw)
+    step.dH.fill_(3.0)
+    dW = torch.zeros(w.V, w.d, dtype=torch.float32, device="cuda")
+    step.forward(H, W, b.tokens.cuda(), b.mask.cuda())
+    step.diagnose(b.mask.cuda(), b.seq_offsets.cuda(), b.rewards.cuda())
+    step.backward(H, W, b.tokens.cuda(), b.mask.cuda(), b.seq_offsets.cuda(), dW=dW)
+    torch.cuda.synchronize()
+    batch = workloads.Batch(w, H, W, b.tokens.cuda(), b.mask.cuda(), b.seq_offsets, b.rewards)
+    _compare_all(batch, step, ref, a)
+    assert _rel_fro(dW.cpu().numpy().astype(np.float64), ref["dW"]) <= DH_REL
+    # T = 0
+    e = ais.AisStep(0, w.d, w.V, w.P, w.G, w.block)
+    z8 = torch.zeros(1, dtype=torch.uint8, device="cuda")
+    offs0 = torch.zeros(w.S + 1, dtype=torch.int32, device="cuda")
+    e.step(torch.zeros(1, w.d, dtype=torch.bfloat16, device="cuda"), b.W.cuda(), torch.zeros(1, dtype=torch.int32, device="cuda"),
+           z8, offs0, b.rewards.cuda())
+    torch.cuda.synchronize()
+    d = e.read_diag()
+    assert d["alpha"] == 0.0 and d["status_flags"] & ais.FLAG_EMPTY and float(e.loss.item()) == 0.0
+
+
 def test_on_policy_recovery_on_gpu():
     """Feeding the trainer's log-probs as the rollout's: rho == 1 exactly, alpha == 0 (Proposition 'on-policy recovery')."""
     ais = _lib()
