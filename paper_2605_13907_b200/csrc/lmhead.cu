@@ -8,6 +8,8 @@
 // vocabulary is so long that the one epilogue per unit need not overlap anything.  In the FP8 pass the first warpgroup gives
 // registers to the two epilogue warpgroups, which keep 128 fp32 accumulators per thread.  Two 256-column accumulators alternate so that the epilogue of one tile (or,
 // in the FP8 pass, the promotion of one scale block) overlaps the MMAs of the next.
+#include <type_traits>
+
 #include "lmhead.cuh"
 #include "ptx.cuh"
 #include "../../include/ais.h"
@@ -40,31 +42,6 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-
-// Packed pairs of fp32 in one 64-bit register and the two-wide arithmetic of sm_100 on them.
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
 }
 
 template <int N>
@@ -375,6 +352,136 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 tb.advance();
                 continue;
             }
+            if (MODE == kFwdFp8) {
+                // Per-block scales.  Every scale block's partial sum comes back from tensor memory and is promoted
+                // as acc += (sH[row] sW[col]) * partial.  The partial tile is read in the 16x256b fragment shape:
+                // a thread then owns 4 rows x 32 columns of its warp's 32 x 128 piece, so it needs only 4 + 32 scale
+                // values per block, fetched with lane-distinct shared-memory reads (a row-per-thread layout needs
+                // all 128 column scales in every thread, and those broadcast reads alone saturate shared memory).
+                const int rg = lane >> 2, cp = lane & 3;
+                int64_t grow4[4];
+                bool rok4[4];
+                int y4[4];
+                float m4[4], s4[4], zy4[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int64_t lr = static_cast<int64_t>(w.rt) * kBM + q * 32 + (r >> 1) * 16 + (r & 1) * 8 + rg;
+                    rok4[r] = lr < a.rows;
+                    grow4[r] = a.row0 + lr;
+                    y4[r] = -1;
+                    if (rok4[r]) {
+                        y4[r] = a.tokens[grow4[r]];
+                        if (a.mask[grow4[r]] != 0 && (y4[r] < 0 || y4[r] >= a.ncols)) { flags |= AIS_FLAG_TOKEN_RANGE; y4[r] = -1; }
+                    }
+                    m4[r] = kNegBig; s4[r] = 0.f; zy4[r] = -INFINITY;
+                }
+                for (int t = w.t0; t < w.t1 && ok; ++t) {
+                    float acc[4][16][2];                       // [row][8-column group][column of the pair]
+#pragma unroll
+                    for (int r = 0; r < 4; ++r)
+#pragma unroll
+                        for (int n = 0; n < 16; ++n) { acc[r][n][0] = 0.f; acc[r][n][1] = 0.f; }
+                    for (int ks = 0; ks < a.ksteps && ok; ++ks) {
+                        if (!mbar_wait_warp(&sfull[sc.idx], sc.phase, abort_flag)) { ok = false; break; }
+                        const float* sS = reinterpret_cast<const float*>(scale_base + sc.idx * kScaleSlotBytes);
+                        for (int g = 0; g < a.sgroups; ++g) {
+                            if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                            float sh[4];
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) sh[r] = sS[g * kBM + q * 32 + (r >> 1) * 16 + (r & 1) * 8 + rg];
+                            const float2* sw2 = reinterpret_cast<const float2*>(sS + (kScaleBOffset / 4) + g * kBN + half * 128) + cp;
+                            // four loads: (lane half of the quarter) x (column half of the piece); the indices are
+                            // compile-time constants so that the accumulators stay in registers
+                            auto piece = [&](auto HH, auto NB, auto LAST) {
+                                constexpr int hh = decltype(HH)::value, nb = decltype(NB)::value;
+                                uint32_t v[32];
+                                tmem_ld_16x256b_x8(tmem_base + (static_cast<uint32_t>(q * 32 + hh * 16) << 16) + tb.idx * kBN +
+                                                       half * 128 + nb * 64, v);
+                                tmem_ld_wait(v);
+                                if (decltype(LAST)::value) {
+                                    // the partial sums are in registers: hand the buffer back before the arithmetic
+                                    tc_fence_before();
+                                    __syncwarp();
+                                    if (lane == 0) mbar_arrive(&tempty[tb.idx]);
+                                }
+#pragma unroll
+                                for (int mq = 0; mq < 8; ++mq) {
+                                    const float2 sw = sw2[(nb * 8 + mq) * 4];          // columns 8n + 2cp, +1 of this thread
+#pragma unroll
+                                    for (int u = 0; u < 2; ++u) {
+                                        acc[hh * 2 + u][nb * 8 + mq][0] =
+                                            fmaf(sh[hh * 2 + u] * sw.x, __uint_as_float(v[4 * mq + 2 * u]), acc[hh * 2 + u][nb * 8 + mq][0]);
+                                        acc[hh * 2 + u][nb * 8 + mq][1] =
+                                            fmaf(sh[hh * 2 + u] * sw.y, __uint_as_float(v[4 * mq + 2 * u + 1]), acc[hh * 2 + u][nb * 8 + mq][1]);
+                                    }
+                                }
+                            };
+                            using I0 = std::integral_constant<int, 0>;
+                            using I1 = std::integral_constant<int, 1>;
+                            piece(I0{}, I0{}, std::false_type{});
+                            piece(I0{}, I1{}, std::false_type{});
+                            piece(I1{}, I0{}, std::false_type{});
+                            piece(I1{}, I1{}, std::true_type{});
+                            tb.advance();
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sempty[sc.idx]);
+                        sc.advance();
+                    }
+                    if (!ok) break;
+                    // streaming log-sum-exp over this thread's 32 columns of each of its 4 rows
+                    const int cbase = t * kBN + half * 128 + 2 * cp;           // column of acc[.][0][0]
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const int yy = y4[r] - cbase;                          // = 8n + e for an owned column
+                        if (yy >= 0 && yy < 128 && (yy & 6) == 0) {
+                            // written as a running maximum on purpose: a chain of "if (k == n) z = acc[n]" is folded by
+                            // the compiler into acc[k], and a dynamically indexed array leaves the register file
+#pragma unroll
+                            for (int n = 0; n < 16; ++n) {
+                                zy4[r] = fmaxf(zy4[r], (yy == 8 * n) ? acc[r][n][0] : -INFINITY);
+                                zy4[r] = fmaxf(zy4[r], (yy == 8 * n + 1) ? acc[r][n][1] : -INFINITY);
+                            }
+                        }
+                        if (t * kBN + kBN > a.ncols) {
+#pragma unroll
+                            for (int n = 0; n < 16; ++n) {
+                                if (cbase + 8 * n >= a.ncols) acc[r][n][0] = -INFINITY;
+                                if (cbase + 8 * n + 1 >= a.ncols) acc[r][n][1] = -INFINITY;
+                            }
+                        }
+                        float cm = acc[r][0][0];
+#pragma unroll
+                        for (int n = 0; n < 16; ++n) cm = fmaxf(cm, fmaxf(acc[r][n][0], acc[r][n][1]));
+                        const float m_new = fmaxf(m4[r], cm * kLog2e);
+                        float add = 0.f;
+#pragma unroll
+                        for (int n = 0; n < 16; ++n)
+                            add += ex2(fmaf(acc[r][n][0], kLog2e, -m_new)) + ex2(fmaf(acc[r][n][1], kLog2e, -m_new));
+                        s4[r] = fmaf(s4[r], ex2(m4[r] - m_new), add);
+                        m4[r] = m_new;
+                    }
+                }
+                // the four threads that share a row merge their (max, sum, target) and one of them writes the partial
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    float M = fmaxf(m4[r], __shfl_xor_sync(0xffffffffu, m4[r], 1));
+                    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
+                    float ssum = s4[r] * ex2(m4[r] - M);
+                    ssum += __shfl_xor_sync(0xffffffffu, ssum, 1);
+                    ssum += __shfl_xor_sync(0xffffffffu, ssum, 2);
+                    float z = fmaxf(zy4[r], __shfl_xor_sync(0xffffffffu, zy4[r], 1));
+                    z = fmaxf(z, __shfl_xor_sync(0xffffffffu, z, 2));
+                    if (ok && rok4[r] && cp == 0) {
+                        const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow4[r];
+                        a.part_m[o] = M * kLn2;
+                        a.part_s[o] = ssum;
+                        a.part_z[o] = z;
+                    }
+                }
+                continue;
+            }
             const int64_t lrow = static_cast<int64_t>(w.rt) * kBM + r_in_tile;   // row inside this launch
             const bool row_ok = lrow < a.rows;
             const int64_t grow = a.row0 + lrow;
@@ -395,49 +502,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (cf == 0.f) valid = false;                  // rows without gradient are written as exact zeros
             }
 
-            for (int t = w.t0; t < w.t1 && ok; ++t) {
+            for (int t = w.t0; MODE != kFwdFp8 && t < w.t1 && ok; ++t) {
                 const int col_base = t * kBN + half * 128;    // first output column of this thread's half
-                uint64_t acc2[64];                             // FP8 pass: 128 fp32 accumulators as packed pairs
-                if (MODE == kFwdFp8) {
-#pragma unroll
-                    for (int i = 0; i < 64; ++i) acc2[i] = 0ull;
-                    for (int ks = 0; ks < a.ksteps && ok; ++ks) {
-                        if (!mbar_wait_warp(&sfull[sc.idx], sc.phase, abort_flag)) { ok = false; break; }
-                        const float* sS = reinterpret_cast<const float*>(scale_base + sc.idx * kScaleSlotBytes);
-                        for (int g = 0; g < a.sgroups; ++g) {
-                            if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
-                            tc_fence_after();
-                            const float sh = sS[g * kBM + r_in_tile];
-                            const uint64_t sh2 = pack2(sh, sh);
-                            const ulonglong2* sw2 = reinterpret_cast<const ulonglong2*>(sS + (kScaleBOffset / 4) + g * kBN + half * 128);
-                            const uint32_t taddr = tmem_base + lane_addr + tb.idx * kBN + half * 128;
-#pragma unroll
-                            for (int c = 0; c < 4; ++c) {
-                                uint32_t v[32];
-                                tmem_ld32(taddr + c * 32, v);
-                                tmem_ld_wait(v);
-                                if (c == 3) {
-                                    // the partial sums are in registers: hand the buffer back before the arithmetic
-                                    tc_fence_before();
-                                    __syncwarp();
-                                    if (lane == 0) mbar_arrive(&tempty[tb.idx]);
-                                }
-#pragma unroll
-                                for (int i = 0; i < 32; i += 4) {
-                                    const ulonglong2 sw = sw2[(c * 32 + i) >> 2];      // scales of 4 columns, two packed pairs
-                                    const int j = (c * 32 + i) >> 1;
-                                    acc2[j] = fma2(mul2(sh2, sw.x), pack2u(v[i], v[i + 1]), acc2[j]);
-                                    acc2[j + 1] = fma2(mul2(sh2, sw.y), pack2u(v[i + 2], v[i + 3]), acc2[j + 1]);
-                                }
-                            }
-                            tb.advance();
-                        }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sempty[sc.idx]);
-                        sc.advance();
-                    }
-                    if (!ok) break;
-                } else {
+                {
                     if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                 }
@@ -447,10 +514,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 for (int c = 0; c < 4; ++c) {
                     const int col0 = col_base + c * 32;
                     float x[32];
-                    if (MODE == kFwdFp8) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 2) unpack2(acc2[(c * 32 + i) >> 1], x[i], x[i + 1]);
-                    } else {
+                    {
                         uint32_t v[32];
                         tmem_ld32(taddr + c * 32, v);
                         tmem_ld_wait(v);
@@ -461,7 +525,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             for (int i = 0; i < 32; ++i) x[i] *= tscale;
                         }
                     }
-                    if (MODE == kFwdBf16 || MODE == kFwdFp8 || MODE == kFwdFp8T) {
+                    if (MODE == kFwdBf16 || MODE == kFwdFp8T) {
                         if (y >= col0 && y < col0 + 32) {
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
@@ -499,14 +563,12 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         }
                     }
                 }
-                if (MODE != kFwdFp8) {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&tempty[tb.idx]);
-                    tb.advance();
-                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tempty[tb.idx]);
+                tb.advance();
             }
-            if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8 || MODE == kFwdFp8T)) {
+            if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8T)) {
                 const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow;
                 a.part_m[o] = m2 * kLn2;
                 a.part_s[o] = s;
