@@ -267,6 +267,12 @@ def run_ours(args) -> None:
 
     if rank == 0:
         peaks = _peaks()
+        # rows whose advantage is zero (all responses of their prompt got the same reward): their gradient is exactly zero,
+        # and whole 128-row tiles of such rows are skipped by the backward passes (the forward passes still run on them)
+        r = batch.rewards.numpy().reshape(w.P, w.G)
+        zero_seq = np.repeat(np.all(r == r[:, :1], axis=1), w.G)
+        lens = np.diff(batch.seq_offsets.numpy())
+        zero_rows = int(lens[zero_seq].sum())
         flops_pass = 2.0 * T * w.d * w.V                      # algorithmic FLOPs of one T x d x V contraction
         t_dom = seg["fwd_train_bf16"] * 1e-3
         achieved = flops_pass / t_dom / 1e12
@@ -283,7 +289,7 @@ def run_ours(args) -> None:
             "config": {"workload": f"{w.name}: d={w.d} V={w.V} P={w.P} G={w.G} block={w.block} lengths={w.lengths}",
                        "rows": T, "valid_tokens_per_gpu": n_valid,
                        "l2": "inputs larger than L2 (H %.2f GB, W %.2f GB)" % (T * w.d * 2 / 1e9, w.V * w.d * 2 / 1e9),
-                       "parallelism": f"dp{world} (whole prompts per GPU, LM head replicated, one all-reduce of 12 moments for alpha)", "bwd_row_chunks": chunks,
+                       "zero_gradient_rows": zero_rows, "parallelism": f"dp{world} (whole prompts per GPU, LM head replicated, one all-reduce of 12 moments for alpha)", "bwd_row_chunks": chunks,
                        "alpha": diag["alpha"], "d_bar": diag["d_bar"]},
             "segments_ms": seg,
             "roofline": {"bound": "tensor", "kernel": "lmhead_kernel<bf16 forward> (trainer log-probs)", "achieved": achieved,

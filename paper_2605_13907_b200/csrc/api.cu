@@ -111,6 +111,7 @@ struct Layout {
     int nsplit, nparts;
     size_t off_part_m, off_part_s, off_part_z;   // forward partials
     size_t off_diag;                              // reduction partials (doubles)
+    size_t off_flags;                             // one byte per 128-row tile: anything to compute there?
     size_t off_coef, off_nseq;                    // backward: c_t, valid rows per sequence
     size_t off_u;                                 // backward scratch
     int64_t ldU;
@@ -128,6 +129,7 @@ Layout make_layout(const ais_shape* s, const ais_params* p) {
     L.off_part_m = off; off += part_bytes;
     L.off_part_s = off; off += part_bytes;
     L.off_part_z = off; off += part_bytes;
+    L.off_flags = off;  off += align_up(static_cast<size_t>(L.t_ld / kBM + 2), 256);
     L.off_diag = off;   off += align_up(static_cast<size_t>(kDiagBlocks) * kNumMoments * sizeof(double), 256);
     L.off_coef = off;   off += align_up(static_cast<size_t>(L.t_ld) * sizeof(float), 256);
     L.off_nseq = off;   off += align_up(static_cast<size_t>(s->P) * s->G * sizeof(int32_t), 256);
@@ -262,6 +264,9 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     a.part_z = reinterpret_cast<float*>(ws + L.off_part_z);
     a.part_ld = L.t_ld;
     a.status = dev_status;
+    // row tiles without a single valid row are skipped by the tensor-core passes
+    a.tile_active = ws + L.off_flags;
+    if (launch_tile_flags_mask(mask, shape->T, ws + L.off_flags, s) != cudaSuccess) return AIS_ERR_DEVICE;
     const int units = a.n_row_tiles * a.nsplit;
     const int ctas = units < num_sms ? units : num_sms;
     const uint64_t T = static_cast<uint64_t>(shape->T), V = static_cast<uint64_t>(shape->V), d = static_cast<uint64_t>(shape->d);
@@ -402,6 +407,8 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
                          reinterpret_cast<double*>(ws + L.off_diag), coef, loss, diag, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     if (shape->T == 0) return AIS_OK;
+    // row tiles whose gradient factors are all zero (masked rows, zero advantage) are skipped by the recompute and dH passes
+    if (launch_tile_flags_coef(coef, shape->T, ws + L.off_flags, s) != cudaSuccess) return AIS_ERR_DEVICE;
 
     // rows of scratch the workspace can hold (whole row tiles)
     int64_t blk_rows = static_cast<int64_t>((workspace_bytes - L.fixed_bytes) / L.u_row_bytes) / kBM * kBM;
@@ -438,6 +445,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
         a.dH = static_cast<__nv_bfloat16*>(dH);
         a.lddh = shape->ldh;
         a.status = dev_status;
+        a.tile_active = ws + L.off_flags;
         a.sgroups = 1;
         // recompute softmax - onehot into the scratch
         a.ncols = shape->V;

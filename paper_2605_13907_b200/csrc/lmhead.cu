@@ -80,6 +80,21 @@ __device__ __forceinline__ Unit decode_unit(const LmheadArgs& a, int u) {
     return w;
 }
 
+// Row tiles in which no row needs computing (all rows masked in the forward passes, all gradient factors zero in
+// the backward passes) are skipped by all three roles alike; the epilogue writes the neutral output where one is
+// needed.  The dW pass contracts over rows, so it has nothing to skip.
+template <int MODE>
+__device__ __forceinline__ bool unit_active(const LmheadArgs& a, const Unit& w) {
+    if (MODE == kBwdDw || a.tile_active == nullptr) return true;
+    const int64_t g = a.row0 / kBM;
+    if (MODE == kBwdDh) {
+        const int64_t t0 = g + 2 * static_cast<int64_t>(w.rt);
+        const bool second = (2 * static_cast<int64_t>(w.rt) + 1) * kBM < a.rows;
+        return a.tile_active[t0] != 0 || (second && a.tile_active[t0 + 1] != 0);
+    }
+    return a.tile_active[g + w.rt] != 0;
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -140,6 +155,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             bool ok = true;
             for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit<MODE>(a, u);
+                if (!unit_active<MODE>(a, w)) continue;
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
                     for (int ks = 0; ks < a.ksteps; ++ks) {
                         if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -199,6 +215,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             bool ok = true;
             for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
                 const Unit w = decode_unit<MODE>(a, u);
+                if (!unit_active<MODE>(a, w)) continue;
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
                     if (MODE != kFwdFp8) {
                         if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -279,6 +296,32 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         uint32_t flags = 0;
         for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
             const Unit w = decode_unit<MODE>(a, u);
+            if (!unit_active<MODE>(a, w)) {
+                // nothing was loaded or multiplied for this unit: write the neutral output where later passes read it
+                if (MODE == kBwdDh) {
+#pragma unroll
+                    for (int sub = 0; sub < 2; ++sub) {
+                        const int64_t lr = static_cast<int64_t>(w.rt) * kDhRows + sub * kBM + r_in_tile;
+                        if (lr < a.rows) {
+                            uint4* dst = reinterpret_cast<uint4*>(a.dH + (a.row0 + lr) * a.lddh + w.t0 * kBN + half * 128);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (w.t0 * kBN + half * 128 + j * 8 < a.ncols) dst[j] = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                } else if (MODE == kBwdP) {
+                    const int64_t lr = static_cast<int64_t>(w.rt) * kBM + r_in_tile;
+                    if (lr < a.rows) {
+                        for (int t = w.t0; t < w.t1; ++t) {
+                            uint4* dst = reinterpret_cast<uint4*>(a.U + lr * a.ldU + t * kBN + half * 128);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (t * kBN + half * 128 + j * 8 < a.ncols) dst[j] = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                }
+                continue;       // forward passes: the rows are masked, the merge kernel never reads their partials
+            }
             if (MODE == kBwdDh) {
                 // one unit = 256 rows x 256 columns of dH, finished after the whole contraction over the vocabulary
                 if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag)) { ok = false; break; }

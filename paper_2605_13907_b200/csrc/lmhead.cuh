@@ -45,6 +45,7 @@ struct LmheadArgs {
     int32_t ksteps;        // shared-memory stages per accumulator tile
     int32_t nsplit;        // forward / recompute: independent column ranges per row tile
     int32_t sgroups;       // FP8: scale blocks per stage (128 / fp8_block)
+    const uint8_t* tile_active;   // one byte per global 128-row tile: 0 = nothing to compute there (may be NULL)
     const int32_t* tokens;
     const uint8_t* mask;
     float* part_m;         // [nsplit*2][part_ld] running maxima (natural log units)

@@ -267,6 +267,15 @@ __global__ void seq_stats_kernel(const uint8_t* __restrict__ mask, const int32_t
     }
 }
 
+// One byte per 128-row tile: does any row of the tile need computing?  (mask != 0 / gradient factor != 0)
+template <typename T>
+__global__ void tile_flags_kernel(const T* __restrict__ pred, int64_t n, uint8_t* __restrict__ flags) {
+    const int64_t tile = blockIdx.x;
+    const int64_t i = tile * 128 + threadIdx.x;
+    const int any = __syncthreads_or(i < n && pred[i] != T(0));
+    if (threadIdx.x == 0) flags[tile] = any ? 1 : 0;
+}
+
 __device__ __forceinline__ int seq_of_row(const int32_t* __restrict__ seq_offsets, int S, int64_t t) {
     int lo = 0, hi = S;                 // largest s with seq_offsets[s] <= t
     while (hi - lo > 1) {
@@ -482,6 +491,18 @@ cudaError_t launch_combine(const float* part_m, const float* part_s, const float
     if (T == 0) return cudaSuccess;
     const int blocks = static_cast<int>(((T + 255) / 256) < 1184 ? ((T + 255) / 256) : 1184);
     combine_kernel<<<blocks, 256, 0, stream>>>(part_m, part_s, part_z, nparts, part_ld, mask, T, lp, lse, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tile_flags_mask(const uint8_t* mask, int64_t T, uint8_t* flags, cudaStream_t stream) {
+    if (T <= 0) return cudaSuccess;
+    tile_flags_kernel<uint8_t><<<static_cast<unsigned>((T + 127) / 128), 128, 0, stream>>>(mask, T, flags);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tile_flags_coef(const float* coef, int64_t T, uint8_t* flags, cudaStream_t stream) {
+    if (T <= 0) return cudaSuccess;
+    tile_flags_kernel<float><<<static_cast<unsigned>((T + 127) / 128), 128, 0, stream>>>(coef, T, flags);
     return cudaGetLastError();
 }
 

@@ -24,6 +24,10 @@ cudaError_t launch_quantize_tensor(const void* x, int64_t rows, int64_t cols, in
 cudaError_t launch_combine(const float* part_m, const float* part_s, const float* part_z, int nparts, int64_t part_ld,
                            const uint8_t* mask, int64_t T, float* lp, float* lse, uint32_t* status, cudaStream_t stream);
 
+// flags[i] = 1 when rows 128 i .. 128 i + 127 contain a row with mask != 0 (resp. a non-zero gradient factor).
+cudaError_t launch_tile_flags_mask(const uint8_t* mask, int64_t T, uint8_t* flags, cudaStream_t stream);
+cudaError_t launch_tile_flags_coef(const float* coef, int64_t T, uint8_t* flags, cudaStream_t stream);
+
 // n_valid_seq[s] and (when rewards != nullptr) adv[s].
 cudaError_t launch_seq_stats(const uint8_t* mask, const int32_t* seq_offsets, const float* rewards, int S, int G,
                              int adv_std_norm, float eps, float* adv, int32_t* n_valid_seq, cudaStream_t stream);

@@ -322,6 +322,33 @@ def test_padded_leading_dimensions_and_empty_batch_of_rows():
     assert d["alpha"] == 0.0 and d["status_flags"] & ais.FLAG_EMPTY and float(e.loss.item()) == 0.0
 
 
+def test_whole_row_tiles_without_work_are_skipped_correctly():
+    """A group with equal rewards (zero advantage over ~800 consecutive rows) and a long stretch of masked rows: the
+    tensor-core passes skip such 128-row tiles; outputs must still be exact zeros there and right everywhere else,
+    including dW, which contracts over the skipped rows."""
+    ais = _lib()
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], d=256, V=776, P=3, G=4, lengths="const:200", seed=99)
+    b = workloads.make_batch(w, device="cpu")
+    b.rewards[4:8] = 1.0                                   # prompt 1: all responses rewarded -> A = 0 on rows 800..1599
+    b.rewards[0:4] = torch.tensor([1.0, 0.0, 0.0, 1.0])
+    b.mask[130:520] = 0                                    # rows 130..519 masked: tiles 2 and 3 hold no valid row
+    batch = _to_cuda(b)
+    a, ref = _oracle(batch)
+    assert np.all(ref["c"][800:1600] == 0) and np.any(ref["c"][:130] != 0)
+    step = ais.AisStep(batch.T, w.d, w.V, w.P, w.G, w.block)
+    step.dH.fill_(5.0)
+    dW = torch.full((w.V, w.d), 5.0, dtype=torch.float32, device="cuda")
+    offs, rew = batch.seq_offsets.cuda(), batch.rewards.cuda()
+    step.forward(batch.H, batch.W, batch.tokens, batch.mask)
+    step.diagnose(batch.mask, offs, rew)
+    step.backward(batch.H, batch.W, batch.tokens, batch.mask, offs, dW=dW)
+    torch.cuda.synchronize()
+    _compare_all(batch, step, ref, a)
+    dH = step.dH.float().cpu().numpy()
+    assert np.all(dH[800:1600] == 0) and np.all(dH[130:520] == 0)
+    assert _rel_fro(dW.cpu().numpy().astype(np.float64), ref["dW"]) <= DH_REL
+
+
 def test_on_policy_recovery_on_gpu():
     """Feeding the trainer's log-probs as the rollout's: rho == 1 exactly, alpha == 0 (Proposition 'on-policy recovery')."""
     ais = _lib()
