@@ -281,7 +281,7 @@ def run_ours(args) -> None:
         blk_rows = (step.workspace.numel() - fixed) // (_ld_u(w.V) * 2) // 128 * 128
         blk_rows = max(128, min(blk_rows, (T + 127) // 128 * 128))
         chunks = -(-T // blk_rows)
-        launches = (2 if w.block else 6) + 2 + 2 + (4 if world == 1 else 5) + 3 + (3 if args.with_dw else 2) * chunks
+        launches = (2 if w.block else 6) + 3 + 3 + (4 if world == 1 else 5) + 4 + (3 if args.with_dw else 2) * chunks
         out = {
             "metric": METRIC, "value": tokens_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
