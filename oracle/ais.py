@@ -29,7 +29,7 @@ class Params:
     """Hyper-parameters (Appendix 'AIS hyperparameters' and Table of GRPO settings).
 
     beta_var is listed by Algorithm 1 but the paper prints no value for it;
-    1.0 is this build's reading.  alpha_override = None keeps the adaptive
+    1.0 is the reading taken here.  alpha_override = None keeps the adaptive
     coefficient; a number forces alpha (0 = plain GRPO, 1 = truncated IS).
     """
     C: float = 5.0
