@@ -5,113 +5,30 @@
 // (warps 2, 3 idle), warps 4..11 are the epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 (one row per
 // thread) and column half (w-4)/4 of the 256-column accumulator.  The dH pass gives a CTA two row tiles
 // (256 rows, both accumulators) so that every W slice it loads is used twice; its contraction over the
-// vocabulary is so long that the one epilogue per unit need not overlap anything.  In the FP8 pass the first warpgroup gives
-// registers to the two epilogue warpgroups, which keep 128 fp32 accumulators per thread.  Two 256-column accumulators alternate so that the epilogue of one tile (or,
-// in the FP8 pass, the promotion of one scale block) overlaps the MMAs of the next.
+// vocabulary is so long that the one epilogue per unit need not overlap anything.  Two 256-column accumulators
+// alternate so that the epilogue of one tile overlaps the MMAs of the next.  The rollout pass with per-block
+// scales has a kernel of its own (lmhead_fp8.cu).
 #include <type_traits>
 
-#include "lmhead.cuh"
-#include "ptx.cuh"
+#include "lmhead_common.cuh"
 #include "../../include/ais.h"
 
 namespace ais {
 
 namespace {
 
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kNegBig = -1.0e30f;
-
-struct Pipe {
-    uint32_t idx = 0, phase = 0;
-    int n;
-    __device__ explicit Pipe(int n_) : n(n_) {}
-    __device__ __forceinline__ void advance() {
-        if (++idx == static_cast<uint32_t>(n)) { idx = 0; phase ^= 1u; }
-    }
-};
-
-// Warp-wide wait: every lane polls (so every lane observes the completed phase itself) and the outcome is
-// made uniform, because the tcgen05.ld / __syncwarp that follow need the whole warp.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    const bool r = mbar_wait(bar, parity, abort_flag);
-    return __all_sync(0xffffffffu, r);
-}
-
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-template <int N>
-__device__ __forceinline__ void reg_alloc() {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
-}
-template <int N>
-__device__ __forceinline__ void reg_dealloc() {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// Which row tile and which column tiles a work unit covers.
-struct Unit {
-    int rt, t0, t1, part;
-};
-template <int MODE>
-__device__ __forceinline__ Unit decode_unit(const LmheadArgs& a, int u) {
-    Unit w;
-    if (MODE == kBwdDh || MODE == kBwdDw) {
-        w.rt = u / a.n_col_tiles;
-        w.t0 = u % a.n_col_tiles;
-        w.t1 = w.t0 + 1;
-        w.part = 0;
-    } else {
-        w.rt = u / a.nsplit;
-        const int c = u % a.nsplit;
-        w.t0 = static_cast<int>((static_cast<int64_t>(c) * a.n_col_tiles) / a.nsplit);
-        w.t1 = static_cast<int>((static_cast<int64_t>(c + 1) * a.n_col_tiles) / a.nsplit);
-        w.part = c;
-    }
-    return w;
-}
-
-// Row tiles in which no row needs computing (all rows masked in the forward passes, all gradient factors zero in
-// the backward passes) are skipped by all three roles alike; the epilogue writes the neutral output where one is
-// needed.  The dW pass contracts over rows, so it has nothing to skip.
-template <int MODE>
-__device__ __forceinline__ bool unit_active(const LmheadArgs& a, const Unit& w) {
-    if (MODE == kBwdDw || a.tile_active == nullptr) return true;
-    const int64_t g = a.row0 / kBM;
-    if (MODE == kBwdDh) {
-        const int64_t t0 = g + 2 * static_cast<int64_t>(w.rt);
-        const bool second = (2 * static_cast<int64_t>(w.rt) + 1) * kBM < a.rows;
-        return a.tile_active[t0] != 0 || (second && a.tile_active[t0 + 1] != 0);
-    }
-    return a.tile_active[g + w.rt] != 0;
-}
-
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
-lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-              const __grid_constant__ CUtensorMap tmSA, const __grid_constant__ CUtensorMap tmSB,
-              const LmheadArgs a) {
+lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const LmheadArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* stage_base = smem;
-    uint8_t* scale_base = smem + kStages * kStageBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(scale_base + kScaleSlots * kScaleSlotBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
     uint64_t* full = bars;                       // [kStages]   TMA -> MMA
     uint64_t* empty = full + kStages;            // [kStages]   MMA -> TMA
     uint64_t* tfull = empty + kStages;           // [2]         MMA -> epilogue
     uint64_t* tempty = tfull + 2;                // [2]         epilogue -> MMA
-    uint64_t* sfull = tempty + 2;                // [kScaleSlots] TMA -> epilogue (FP8 scales)
-    uint64_t* sempty = sfull + kScaleSlots;      // [kScaleSlots] epilogue -> TMA
-    uint64_t* done = sempty + kScaleSlots;       // [1]         all MMAs of this CTA have completed
+    uint64_t* done = tempty + 2;                 // [1]         all MMAs of this CTA have completed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBarriers);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -127,7 +44,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
-        for (int i = 0; i < kScaleSlots; ++i) { mbar_init(&sfull[i], 1); mbar_init(&sempty[i], kEpiWarps); }
         mbar_init(done, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -143,14 +59,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-
-    // FP8 pass: 384 threads x 168 registers at launch = 128 x 56 + 256 x 224 after the split below.
-    if (warp < 4) {
-    if (MODE == kFwdFp8) reg_dealloc<56>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            Pipe st(STG), sc(kScaleSlots);
+            Pipe st(STG);
             uint32_t issued = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
@@ -162,7 +74,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         uint8_t* sA = stage_base + st.idx * STG_BYTES;
                         uint8_t* sB = sA + A_BYTES;
                         mbar_expect_tx(&full[st.idx], STG_BYTES);
-                        const int kelem = (MODE == kFwdFp8 || MODE == kFwdFp8T) ? ks * 128 : ks * 64;
+                        const int kelem = (MODE == kFwdFp8T) ? ks * 128 : ks * 64;
                         if (MODE == kBwdDh) {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kDhRows);
                             tma_load_2d(sA + kAStageBytes, &tmA, &full[st.idx], kelem, w.rt * kDhRows + kBM);
@@ -185,14 +97,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         }
                         ++issued;
                         st.advance();
-                        if (MODE == kFwdFp8) {
-                            if (!mbar_wait(&sempty[sc.idx], sc.phase ^ 1u, abort_flag)) { ok = false; break; }
-                            uint8_t* sS = scale_base + sc.idx * kScaleSlotBytes;
-                            mbar_expect_tx(&sfull[sc.idx], static_cast<uint32_t>(a.sgroups) * (kBM + kBN) * 4u);
-                            tma_load_2d(sS, &tmSA, &sfull[sc.idx], w.rt * kBM, ks * a.sgroups);
-                            tma_load_2d(sS + kScaleBOffset, &tmSB, &sfull[sc.idx], t * kBN, ks * a.sgroups);
-                            sc.advance();
-                        }
                     }
                 }
             }
@@ -209,7 +113,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc =
-                (MODE == kFwdFp8 || MODE == kFwdFp8T) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
+                (MODE == kFwdFp8T) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
                                   : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, MODE == kBwdDw ? 1 : 0, TWO_ACC ? 1 : 0);
             Pipe st(STG), tb(NBUF);
             bool ok = true;
@@ -217,31 +121,14 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const Unit w = decode_unit<MODE>(a, u);
                 if (!unit_active<MODE>(a, w)) continue;
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
-                    if (MODE != kFwdFp8) {
-                        if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
-                    }
+                    if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
                     for (int ks = 0; ks < a.ksteps; ++ks) {
                         if (!mbar_wait(&full[st.idx], st.phase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t sA = smem_u32(stage_base + st.idx * STG_BYTES);
                         const uint32_t sB = sA + A_BYTES;
-                        if (MODE == kFwdFp8) {
-                            const int per = 4 / a.sgroups;             // MMAs per scale block
-                            for (int g = 0; g < a.sgroups && ok; ++g) {
-                                if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag)) { ok = false; break; }
-                                tc_fence_after();
-                                const uint32_t dcol = tmem_base + tb.idx * kBN;
-                                for (int j = 0; j < per; ++j) {
-                                    const uint32_t off = (g * per + j) * 32;
-                                    mma_f8(dcol, smem_desc_sw128(sA + off, 16, 1024), smem_desc_sw128(sB + off, 16, 1024),
-                                           idesc, j > 0 ? 1u : 0u);
-                                }
-                                tc_commit(&tfull[tb.idx]);
-                                tb.advance();
-                            }
-                            if (!ok) break;
-                        } else if (MODE == kBwdDh) {
+                        if (MODE == kBwdDh) {
                             // two row tiles share every B slice: accumulators at TMEM columns 0 and 256
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
@@ -274,7 +161,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         tc_commit(&empty[st.idx]);
                         st.advance();
                     }
-                    if (MODE != kFwdFp8 && ok) {
+                    if (ok) {
                         tc_commit(&tfull[tb.idx]);
                         tb.advance();
                     }
@@ -283,15 +170,13 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             // everything issued has to finish before the tensor memory is given back
             tc_commit(done);
         }
-    }
-    } else {
+    } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue warps
-        if (MODE == kFwdFp8) reg_alloc<224>();
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int half = (warp - 4) >> 2;             // column half of the accumulator
         const int r_in_tile = q * 32 + lane;
         const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        Pipe tb(NBUF), sc(kScaleSlots);
+        Pipe tb(NBUF);
         bool ok = true;
         uint32_t flags = 0;
         for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
@@ -395,136 +280,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 tb.advance();
                 continue;
             }
-            if (MODE == kFwdFp8) {
-                // Per-block scales.  Every scale block's partial sum comes back from tensor memory and is promoted
-                // as acc += (sH[row] sW[col]) * partial.  The partial tile is read in the 16x256b fragment shape:
-                // a thread then owns 4 rows x 32 columns of its warp's 32 x 128 piece, so it needs only 4 + 32 scale
-                // values per block, fetched with lane-distinct shared-memory reads (a row-per-thread layout needs
-                // all 128 column scales in every thread, and those broadcast reads alone saturate shared memory).
-                const int rg = lane >> 2, cp = lane & 3;
-                int64_t grow4[4];
-                bool rok4[4];
-                int y4[4];
-                float m4[4], s4[4], zy4[4];
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int64_t lr = static_cast<int64_t>(w.rt) * kBM + q * 32 + (r >> 1) * 16 + (r & 1) * 8 + rg;
-                    rok4[r] = lr < a.rows;
-                    grow4[r] = a.row0 + lr;
-                    y4[r] = -1;
-                    if (rok4[r]) {
-                        y4[r] = a.tokens[grow4[r]];
-                        if (a.mask[grow4[r]] != 0 && (y4[r] < 0 || y4[r] >= a.ncols)) { flags |= AIS_FLAG_TOKEN_RANGE; y4[r] = -1; }
-                    }
-                    m4[r] = kNegBig; s4[r] = 0.f; zy4[r] = -INFINITY;
-                }
-                for (int t = w.t0; t < w.t1 && ok; ++t) {
-                    float acc[4][16][2];                       // [row][8-column group][column of the pair]
-#pragma unroll
-                    for (int r = 0; r < 4; ++r)
-#pragma unroll
-                        for (int n = 0; n < 16; ++n) { acc[r][n][0] = 0.f; acc[r][n][1] = 0.f; }
-                    for (int ks = 0; ks < a.ksteps && ok; ++ks) {
-                        if (!mbar_wait_warp(&sfull[sc.idx], sc.phase, abort_flag)) { ok = false; break; }
-                        const float* sS = reinterpret_cast<const float*>(scale_base + sc.idx * kScaleSlotBytes);
-                        for (int g = 0; g < a.sgroups; ++g) {
-                            if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
-                            tc_fence_after();
-                            float sh[4];
-#pragma unroll
-                            for (int r = 0; r < 4; ++r) sh[r] = sS[g * kBM + q * 32 + (r >> 1) * 16 + (r & 1) * 8 + rg];
-                            const float2* sw2 = reinterpret_cast<const float2*>(sS + (kScaleBOffset / 4) + g * kBN + half * 128) + cp;
-                            // four loads: (lane half of the quarter) x (column half of the piece); the indices are
-                            // compile-time constants so that the accumulators stay in registers
-                            auto piece = [&](auto HH, auto NB, auto LAST) {
-                                constexpr int hh = decltype(HH)::value, nb = decltype(NB)::value;
-                                uint32_t v[32];
-                                tmem_ld_16x256b_x8(tmem_base + (static_cast<uint32_t>(q * 32 + hh * 16) << 16) + tb.idx * kBN +
-                                                       half * 128 + nb * 64, v);
-                                tmem_ld_wait(v);
-                                if (decltype(LAST)::value) {
-                                    // the partial sums are in registers: hand the buffer back before the arithmetic
-                                    tc_fence_before();
-                                    __syncwarp();
-                                    if (lane == 0) mbar_arrive(&tempty[tb.idx]);
-                                }
-#pragma unroll
-                                for (int mq = 0; mq < 8; ++mq) {
-                                    const float2 sw = sw2[(nb * 8 + mq) * 4];          // columns 8n + 2cp, +1 of this thread
-#pragma unroll
-                                    for (int u = 0; u < 2; ++u) {
-                                        acc[hh * 2 + u][nb * 8 + mq][0] =
-                                            fmaf(sh[hh * 2 + u] * sw.x, __uint_as_float(v[4 * mq + 2 * u]), acc[hh * 2 + u][nb * 8 + mq][0]);
-                                        acc[hh * 2 + u][nb * 8 + mq][1] =
-                                            fmaf(sh[hh * 2 + u] * sw.y, __uint_as_float(v[4 * mq + 2 * u + 1]), acc[hh * 2 + u][nb * 8 + mq][1]);
-                                    }
-                                }
-                            };
-                            using I0 = std::integral_constant<int, 0>;
-                            using I1 = std::integral_constant<int, 1>;
-                            piece(I0{}, I0{}, std::false_type{});
-                            piece(I0{}, I1{}, std::false_type{});
-                            piece(I1{}, I0{}, std::false_type{});
-                            piece(I1{}, I1{}, std::true_type{});
-                            tb.advance();
-                        }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sempty[sc.idx]);
-                        sc.advance();
-                    }
-                    if (!ok) break;
-                    // streaming log-sum-exp over this thread's 32 columns of each of its 4 rows
-                    const int cbase = t * kBN + half * 128 + 2 * cp;           // column of acc[.][0][0]
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const int yy = y4[r] - cbase;                          // = 8n + e for an owned column
-                        if (yy >= 0 && yy < 128 && (yy & 6) == 0) {
-                            // written as a running maximum on purpose: a chain of "if (k == n) z = acc[n]" is folded by
-                            // the compiler into acc[k], and a dynamically indexed array leaves the register file
-#pragma unroll
-                            for (int n = 0; n < 16; ++n) {
-                                zy4[r] = fmaxf(zy4[r], (yy == 8 * n) ? acc[r][n][0] : -INFINITY);
-                                zy4[r] = fmaxf(zy4[r], (yy == 8 * n + 1) ? acc[r][n][1] : -INFINITY);
-                            }
-                        }
-                        if (t * kBN + kBN > a.ncols) {
-#pragma unroll
-                            for (int n = 0; n < 16; ++n) {
-                                if (cbase + 8 * n >= a.ncols) acc[r][n][0] = -INFINITY;
-                                if (cbase + 8 * n + 1 >= a.ncols) acc[r][n][1] = -INFINITY;
-                            }
-                        }
-                        float cm = acc[r][0][0];
-#pragma unroll
-                        for (int n = 0; n < 16; ++n) cm = fmaxf(cm, fmaxf(acc[r][n][0], acc[r][n][1]));
-                        const float m_new = fmaxf(m4[r], cm * kLog2e);
-                        float add = 0.f;
-#pragma unroll
-                        for (int n = 0; n < 16; ++n)
-                            add += ex2(fmaf(acc[r][n][0], kLog2e, -m_new)) + ex2(fmaf(acc[r][n][1], kLog2e, -m_new));
-                        s4[r] = fmaf(s4[r], ex2(m4[r] - m_new), add);
-                        m4[r] = m_new;
-                    }
-                }
-                // the four threads that share a row merge their (max, sum, target) and one of them writes the partial
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    float M = fmaxf(m4[r], __shfl_xor_sync(0xffffffffu, m4[r], 1));
-                    M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
-                    float ssum = s4[r] * ex2(m4[r] - M);
-                    ssum += __shfl_xor_sync(0xffffffffu, ssum, 1);
-                    ssum += __shfl_xor_sync(0xffffffffu, ssum, 2);
-                    float z = fmaxf(zy4[r], __shfl_xor_sync(0xffffffffu, zy4[r], 1));
-                    z = fmaxf(z, __shfl_xor_sync(0xffffffffu, z, 2));
-                    if (ok && rok4[r] && cp == 0) {
-                        const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow4[r];
-                        a.part_m[o] = M * kLn2;
-                        a.part_s[o] = ssum;
-                        a.part_z[o] = z;
-                    }
-                }
-                continue;
-            }
             const int64_t lrow = static_cast<int64_t>(w.rt) * kBM + r_in_tile;   // row inside this launch
             const bool row_ok = lrow < a.rows;
             const int64_t grow = a.row0 + lrow;
@@ -545,7 +300,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (cf == 0.f) valid = false;                  // rows without gradient are written as exact zeros
             }
 
-            for (int t = w.t0; MODE != kFwdFp8 && t < w.t1 && ok; ++t) {
+            for (int t = w.t0; t < w.t1 && ok; ++t) {
                 const int col_base = t * kBN + half * 128;    // first output column of this thread's half
                 {
                     if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
@@ -636,21 +391,21 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 }  // namespace
 
 template <int MODE>
-static cudaError_t launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA, const CUtensorMap& tmSB,
-                               const LmheadArgs& args, int num_ctas, cudaStream_t stream) {
-    lmhead_kernel<MODE><<<num_ctas, kThreads, kSmemBytes, stream>>>(tmA, tmB, tmSA, tmSB, args);
+static cudaError_t launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, const LmheadArgs& args, int num_ctas,
+                               cudaStream_t stream) {
+    lmhead_kernel<MODE><<<num_ctas, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
     return cudaGetLastError();
 }
 
 cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
                           const CUtensorMap& tmSB, const LmheadArgs& args, int num_ctas, cudaStream_t stream) {
     switch (mode) {
-        case kFwdBf16: return launch_mode<kFwdBf16>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
-        case kFwdFp8:  return launch_mode<kFwdFp8>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
-        case kBwdP:    return launch_mode<kBwdP>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
-        case kBwdDh:   return launch_mode<kBwdDh>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
-        case kFwdFp8T: return launch_mode<kFwdFp8T>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
-        case kBwdDw:   return launch_mode<kBwdDw>(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
+        case kFwdBf16: return launch_mode<kFwdBf16>(tmA, tmB, args, num_ctas, stream);
+        case kFwdFp8:  return launch_lmhead_fp8_block(tmA, tmB, tmSA, tmSB, args, num_ctas, stream);
+        case kBwdP:    return launch_mode<kBwdP>(tmA, tmB, args, num_ctas, stream);
+        case kBwdDh:   return launch_mode<kBwdDh>(tmA, tmB, args, num_ctas, stream);
+        case kFwdFp8T: return launch_mode<kFwdFp8T>(tmA, tmB, args, num_ctas, stream);
+        case kBwdDw:   return launch_mode<kBwdDw>(tmA, tmB, args, num_ctas, stream);
     }
     return cudaErrorInvalidValue;
 }
@@ -659,7 +414,7 @@ cudaError_t lmhead_prepare() {
     cudaError_t e;
     e = cudaFuncSetAttribute(lmhead_kernel<kFwdBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(lmhead_kernel<kFwdFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = lmhead_fp8_block_prepare();
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lmhead_kernel<kBwdP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;

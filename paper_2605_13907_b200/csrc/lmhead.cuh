@@ -28,13 +28,10 @@ constexpr int kDhRows = 2 * kBM;
 constexpr int kDhStageBytes = 2 * kAStageBytes + kBStageBytes;
 constexpr int kDhStages = 3;
 static_assert(kDhStages * kDhStageBytes <= kStages * kStageBytes, "the dH stage ring must fit the same shared memory");
-constexpr int kScaleSlots = 4;
-constexpr int kScaleSlotBytes = 4 * (kBM + kBN) * 4;   // up to 4 scale blocks per stage
-constexpr int kScaleBOffset = 4 * kBM * 4;
-constexpr int kNumBarriers = 2 * kStages + 4 + 2 * kScaleSlots + 1;
+constexpr int kNumBarriers = 2 * kStages + 4 + 1;
 constexpr int kThreads = 384;            // warp 0 TMA, warp 1 MMA, warps 2..3 idle, warps 4..11 epilogue
 constexpr int kEpiWarps = 8;
-constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kScaleSlots * kScaleSlotBytes + kNumBarriers * 8 + 64;
+constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kNumBarriers * 8 + 64;
 
 struct LmheadArgs {
     int64_t rows;          // valid rows handled by this launch
@@ -70,5 +67,11 @@ struct LmheadArgs {
 cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
                           const CUtensorMap& tmSB, const LmheadArgs& args, int num_ctas, cudaStream_t stream);
 cudaError_t lmhead_prepare();   // sets the dynamic shared-memory attribute of every instantiation
+
+// The rollout pass with per-block scales (mode kFwdFp8; args.sgroups = 128 / block = 1, 2 or 4).  tmSA / tmSB map the
+// block-major scale arrays with boxes of (128 rows, sgroups) and (256 rows, sgroups).
+cudaError_t launch_lmhead_fp8_block(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmSA,
+                                    const CUtensorMap& tmSB, const LmheadArgs& args, int num_ctas, cudaStream_t stream);
+cudaError_t lmhead_fp8_block_prepare();
 
 }  // namespace ais

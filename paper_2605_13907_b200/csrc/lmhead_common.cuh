@@ -1,0 +1,91 @@
+// Device helpers shared by the LM-head tensor-core kernels: stage-ring bookkeeping, warp-wide bounded waits,
+// register re-splitting, work-unit decoding and the test for row tiles without work.
+#pragma once
+
+#include "lmhead.cuh"
+#include "ptx.cuh"
+
+namespace ais {
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kNegBig = -1.0e30f;
+
+struct Pipe {
+    uint32_t idx = 0, phase = 0;
+    int n;
+    __device__ explicit Pipe(int n_) : n(n_) {}
+    __device__ __forceinline__ void advance() {
+        if (++idx == static_cast<uint32_t>(n)) { idx = 0; phase ^= 1u; }
+    }
+};
+
+// Warp-wide wait: every lane polls (so every lane observes the completed phase itself) and the outcome is
+// made uniform, because the tcgen05.ld / __syncwarp that follow need the whole warp.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    const bool r = mbar_wait(bar, parity, abort_flag);
+    return __all_sync(0xffffffffu, r);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int N>
+__device__ __forceinline__ void reg_alloc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void reg_dealloc() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Which row tile and which column tiles a work unit covers.
+struct Unit {
+    int rt, t0, t1, part;
+};
+template <int MODE>
+__device__ __forceinline__ Unit decode_unit(const LmheadArgs& a, int u) {
+    Unit w;
+    if (MODE == kBwdDh || MODE == kBwdDw) {
+        w.rt = u / a.n_col_tiles;
+        w.t0 = u % a.n_col_tiles;
+        w.t1 = w.t0 + 1;
+        w.part = 0;
+    } else {
+        w.rt = u / a.nsplit;
+        const int c = u % a.nsplit;
+        w.t0 = static_cast<int>((static_cast<int64_t>(c) * a.n_col_tiles) / a.nsplit);
+        w.t1 = static_cast<int>((static_cast<int64_t>(c + 1) * a.n_col_tiles) / a.nsplit);
+        w.part = c;
+    }
+    return w;
+}
+
+// Row tiles in which no row needs computing (all rows masked in the forward passes, all gradient factors zero in
+// the backward passes) are skipped by all three roles alike; the epilogue writes the neutral output where one is
+// needed.  The dW pass contracts over rows, so it has nothing to skip.
+template <int MODE>
+__device__ __forceinline__ bool unit_active(const LmheadArgs& a, const Unit& w) {
+    if (MODE == kBwdDw || a.tile_active == nullptr) return true;
+    const int64_t g = a.row0 / kBM;
+    if (MODE == kBwdDh) {
+        const int64_t t0 = g + 2 * static_cast<int64_t>(w.rt);
+        const bool second = (2 * static_cast<int64_t>(w.rt) + 1) * kBM < a.rows;
+        return a.tile_active[t0] != 0 || (second && a.tile_active[t0 + 1] != 0);
+    }
+    return a.tile_active[g + w.rt] != 0;
+}
+
+}  // namespace
+
+}  // namespace ais
