@@ -7,7 +7,7 @@ calls raise.
 """
 
 from .binding import (  # noqa: F401
-    AisError, Params, Diag, Shape, lib, lib_path, default_params, workspace_bytes, workspace_min_bytes,
+    AisError, Params, Diag, Shape, lib, lib_path, default_params, make_shape, workspace_bytes, workspace_min_bytes,
     quantize_fp8, logprob_fwd, diagnostics, loss_bwd, AisStep, logprob_train_static, STATIC_MAX_ROWS, diag_moments, diag_finalize, NUM_MOMENTS, RowCompaction,
     FLAG_EMPTY, FLAG_TOKEN_RANGE, FLAG_NONFINITE, FLAG_TIMEOUT,
 )

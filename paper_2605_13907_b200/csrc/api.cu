@@ -326,11 +326,10 @@ int ais_diagnostics(const ais_shape* shape, const ais_params* params, const floa
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     const int S = shape->P * shape->G;
-    if (launch_seq_stats(mask, seq_offsets, rewards, S, shape->G, params->adv_std_norm, params->eps, adv, n_valid_seq, s) !=
-        cudaSuccess)
+    if (launch_advantages(rewards, S, shape->G, params->adv_std_norm, params->eps, adv, n_valid_seq, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     if (launch_diag(lp_train, lp_roll, mask, seq_offsets, adv, shape->T, S, *params, reinterpret_cast<double*>(ws + L.off_diag),
-                    rho, w_tilde, diag, s) != cudaSuccess)
+                    n_valid_seq, rho, w_tilde, diag, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     return AIS_OK;
 }
@@ -351,11 +350,10 @@ int ais_diag_moments(const ais_shape* shape, const ais_params* params, const flo
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     const int S = shape->P * shape->G;
-    if (launch_seq_stats(mask, seq_offsets, rewards, S, shape->G, params->adv_std_norm, params->eps, adv, n_valid_seq, s) !=
-        cudaSuccess)
+    if (launch_advantages(rewards, S, shape->G, params->adv_std_norm, params->eps, adv, n_valid_seq, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     if (launch_moments(lp_train, lp_roll, mask, seq_offsets, adv, shape->T, S, *params, reinterpret_cast<double*>(ws + L.off_diag),
-                       moments, s) != cudaSuccess)
+                       n_valid_seq, moments, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     return AIS_OK;
 }
@@ -401,7 +399,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
     const int S = shape->P * shape->G;
     float* coef = reinterpret_cast<float*>(ws + L.off_coef);
     int32_t* nseq = reinterpret_cast<int32_t*>(ws + L.off_nseq);
-    if (launch_seq_stats(mask, seq_offsets, nullptr, S, shape->G, 0, 0.f, nullptr, nseq, s) != cudaSuccess) return AIS_ERR_DEVICE;
+    if (launch_seq_counts(mask, seq_offsets, S, nseq, s) != cudaSuccess) return AIS_ERR_DEVICE;
     const int P_norm = shape->P_total > 0 ? shape->P_total : shape->P;
     if (launch_loss_coef(lp_train, lp_old, lp_ref, params->beta_kl, mask, seq_offsets, adv, w_tilde, nseq, shape->T, S, P_norm * shape->G, params->clip_eps,
                          reinterpret_cast<double*>(ws + L.off_diag), coef, loss, diag, s) != cudaSuccess)

@@ -214,7 +214,6 @@ __global__ void combine_kernel(const float* __restrict__ part_m, const float* __
 
 // ------------------------------------------------------------------------------------------------
 // Segmented reductions: valid rows per sequence and group-relative advantages (Eq. grpo_adv).
-// One CTA per sequence.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
@@ -237,34 +236,50 @@ __device__ double block_sum(double v, double* scratch /*[32]*/) {
     return tot;
 }
 
-__global__ void seq_stats_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ seq_offsets,
-                                 const float* __restrict__ rewards, int G, int adv_std_norm, float eps,
-                                 float* __restrict__ adv, int32_t* __restrict__ n_valid_seq) {
-    __shared__ double scratch[32];
-    const int s = blockIdx.x;
-    const int b = seq_offsets[s], e = seq_offsets[s + 1];
-    double cnt = 0.0;
-    for (int t = b + threadIdx.x; t < e; t += blockDim.x) cnt += mask[t] ? 1.0 : 0.0;
-    const double tot = block_sum(cnt, scratch);
-    if (threadIdx.x == 0) {
-        if (n_valid_seq) n_valid_seq[s] = static_cast<int32_t>(tot);
-        if (rewards && adv) {
-            const int g0 = (s / G) * G;
-            double mean = 0.0;
-            for (int j = 0; j < G; ++j) mean += static_cast<double>(rewards[g0 + j]);
-            mean /= G;
-            double a = static_cast<double>(rewards[s]) - mean;
-            if (adv_std_norm) {
-                double var = 0.0;
-                for (int j = 0; j < G; ++j) {
-                    const double dlt = static_cast<double>(rewards[g0 + j]) - mean;
-                    var += dlt * dlt;
-                }
-                a /= (sqrt(var / G) + static_cast<double>(eps));
-            }
-            adv[s] = static_cast<float>(a);
-        }
+// Valid rows of each sequence: one warp per sequence, 4 mask bytes per lane and load where the row range allows it.
+__global__ void __launch_bounds__(256) seq_count_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ seq_offsets,
+                                                         int S, int32_t* __restrict__ n_valid_seq) {
+    const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (s >= S) return;
+    const int lane = threadIdx.x & 31;
+    const int64_t b = seq_offsets[s], e = seq_offsets[s + 1];
+    const uintptr_t base = reinterpret_cast<uintptr_t>(mask);
+    const int64_t b4 = b + static_cast<int64_t>((4 - ((base + b) & 3)) & 3);          // first row on a 4-byte boundary
+    int cnt = 0;
+    for (int64_t t = b + lane; t < (b4 < e ? b4 : e); t += 32) cnt += mask[t] != 0;
+    const int64_t nwords = b4 < e ? (e - b4) / 4 : 0;
+    for (int64_t i = lane; i < nwords; i += 32) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(mask + b4 + 4 * i);
+        cnt += ((w & 0xFFu) != 0) + ((w & 0xFF00u) != 0) + ((w & 0xFF0000u) != 0) + ((w & 0xFF000000u) != 0);
     }
+    for (int64_t t = b4 + 4 * nwords + lane; t < e; t += 32) cnt += (t >= b4 && mask[t] != 0);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+    if (lane == 0) n_valid_seq[s] = cnt;
+}
+
+// Group-relative advantages (Eq. grpo_adv): one thread per sequence.  With `zero_counts` the per-sequence row
+// counts are cleared for the moments kernel, which adds them up.
+__global__ void adv_kernel(const float* __restrict__ rewards, int S, int G, int adv_std_norm, float eps, float* __restrict__ adv,
+                           int32_t* __restrict__ zero_counts) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= S) return;
+    if (zero_counts) zero_counts[s] = 0;
+    if (!rewards || !adv) return;
+    const int g0 = (s / G) * G;
+    double mean = 0.0;
+    for (int j = 0; j < G; ++j) mean += static_cast<double>(rewards[g0 + j]);
+    mean /= G;
+    double a = static_cast<double>(rewards[s]) - mean;
+    if (adv_std_norm) {
+        double var = 0.0;
+        for (int j = 0; j < G; ++j) {
+            const double dlt = static_cast<double>(rewards[g0 + j]) - mean;
+            var += dlt * dlt;
+        }
+        a /= (sqrt(var / G) + static_cast<double>(eps));
+    }
+    adv[s] = static_cast<float>(a);
 }
 
 // One byte per 128-row tile: does any row of the tile need computing?  (mask != 0 / gradient factor != 0)
@@ -290,34 +305,137 @@ __device__ __forceinline__ int seq_of_row(const int32_t* __restrict__ seq_offset
 //   0 N   1 sum w   2 sum w^2   3 sum |D|   4 sum A   5 sum A^2   6 sum Aw   7 sum (Aw)^2
 //   8 sum (lp_roll - lp_train)   9 sum |exp(lp_train) - exp(lp_roll)|
 // ------------------------------------------------------------------------------------------------
+// Rows are read VEC at a time (16-byte loads of the two log-prob vectors, one 4-byte load of the mask); the
+// sequence of a group's first row comes from a binary search and the following rows only step forward.  The
+// exponentials are evaluated in fp32 (the inputs are fp32 and the sums need seven digits at most), the sums
+// themselves in fp64.  Two groups are in flight per thread so that the fixed grid keeps HBM busy on long batches.
+template <int VEC>
+struct RowGroup {
+    float lt[VEC], lr[VEC];
+    uint8_t mk[VEC];
+    bool any;
+};
+template <int VEC>
+__device__ __forceinline__ RowGroup<VEC> load_group(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
+                                                    const uint8_t* __restrict__ mask, int64_t g) {
+    RowGroup<VEC> r;
+    if (VEC == 4) {
+        const float4 a = reinterpret_cast<const float4*>(lp_train)[g];
+        const float4 b = reinterpret_cast<const float4*>(lp_roll)[g];
+        const uchar4 m = reinterpret_cast<const uchar4*>(mask)[g];
+        r.lt[0] = a.x; r.lt[1 % VEC] = a.y; r.lt[2 % VEC] = a.z; r.lt[3 % VEC] = a.w;
+        r.lr[0] = b.x; r.lr[1 % VEC] = b.y; r.lr[2 % VEC] = b.z; r.lr[3 % VEC] = b.w;
+        r.mk[0] = m.x; r.mk[1 % VEC] = m.y; r.mk[2 % VEC] = m.z; r.mk[3 % VEC] = m.w;
+    } else {
+        r.lt[0] = lp_train[g]; r.lr[0] = lp_roll[g]; r.mk[0] = mask[g];
+    }
+    r.any = false;
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) r.any |= (r.mk[j] != 0);
+    return r;
+}
+
+template <int VEC>
 __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
                                                                 const uint8_t* __restrict__ mask,
                                                                 const int32_t* __restrict__ seq_offsets,
-                                                                const float* __restrict__ adv, int64_t T, int S, double logC,
-                                                                double* __restrict__ partials) {
+                                                                const float* __restrict__ adv, int64_t T, int S, float C,
+                                                                double* __restrict__ partials, int32_t* __restrict__ n_valid_seq) {
     __shared__ double scratch[32];
     double acc[kNumMoments];
 #pragma unroll
     for (int i = 0; i < kNumMoments; ++i) acc[i] = 0.0;
-    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T;
-         t += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-        if (!mask[t]) continue;
-        const double lt = lp_train[t], lr = lp_roll[t];
-        const double dl = lt - lr;
-        const double w = exp(fmin(dl, logC));
-        const double A = adv[seq_of_row(seq_offsets, S, t)];
-        const double Aw = A * w;
-        acc[0] += 1.0;
-        acc[1] += w;
-        acc[2] += w * w;
-        acc[3] += fabs(dl);
-        acc[4] += A;
-        acc[5] += A * A;
-        acc[6] += Aw;
-        acc[7] += Aw * Aw;
-        acc[8] += -dl;
-        acc[9] += fabs(exp(lt) - exp(lr));
+    // Every warp owns a contiguous range of row groups and its lanes interleave inside it, so a lane's rows only
+    // move forward: one binary search for its first group, then the sequence index steps (the next boundary is kept
+    // in a register).  Valid rows are counted per sequence on the way (integer atomics: the result does not depend
+    // on their order).  The rows of one pass of the loop (at most 2 VEC) are summed in fp32 and those short sums
+    // go into the fp64 accumulators, which keeps the fp64 pipe out of the per-row work.
+    int sq = -1, cur = -1, cnt = 0;
+    int64_t next_b = 0;                                   // first row of sequence sq + 1 (or "never" for the last one)
+    float f[kNumMoments];
+    auto flush = [&]() {
+        if (n_valid_seq && cur >= 0 && cnt > 0) atomicAdd(&n_valid_seq[cur], cnt);
+        cnt = 0;
+    };
+    auto clear = [&]() {
+#pragma unroll
+        for (int i = 0; i < 10; ++i) f[i] = 0.f;
+    };
+    auto commit = [&]() {
+#pragma unroll
+        for (int i = 0; i < 10; ++i) acc[i] += static_cast<double>(f[i]);
+    };
+    auto seek = [&](int64_t t) {
+        if (sq < 0) {
+            sq = seq_of_row(seq_offsets, S, t);
+            next_b = sq + 1 < S ? static_cast<int64_t>(seq_offsets[sq + 1]) : (int64_t(1) << 62);
+        }
+        while (t >= next_b) {
+            ++sq;
+            next_b = sq + 1 < S ? static_cast<int64_t>(seq_offsets[sq + 1]) : (int64_t(1) << 62);
+        }
+    };
+    auto add_row = [&](float lt, float lr, float A) {
+        // two fast exponentials per row (relative error about 1e-6, far inside what the sums need):
+        // rho = e^dl, truncated weight min(rho, C), and |e^lt - e^lr| = e^lr |rho - 1|
+        const float dl = lt - lr;
+        const float rho = __expf(dl);
+        const float w = fminf(rho, C);
+        const float Aw = A * w;
+        f[0] += 1.0f;
+        f[1] += w;
+        f[2] = fmaf(w, w, f[2]);
+        f[3] += fabsf(dl);
+        f[4] += A;
+        f[5] = fmaf(A, A, f[5]);
+        f[6] += Aw;
+        f[7] = fmaf(Aw, Aw, f[7]);
+        f[8] -= dl;
+        f[9] = fmaf(__expf(lr), fabsf(rho - 1.0f), f[9]);
+        if (sq != cur) { flush(); cur = sq; }
+        ++cnt;
+    };
+    auto add_group = [&](const RowGroup<VEC>& r, int64_t g) {
+        if (!r.any) return;
+        const int64_t t0 = g * VEC;
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+            if (r.mk[j]) {
+                seek(t0 + j);
+                add_row(r.lt[j], r.lr[j], adv[sq]);
+            }
+        }
+    };
+    const int lane = threadIdx.x & 31;
+    const int64_t ngroups = T / VEC;
+    const int64_t nwarps = static_cast<int64_t>(gridDim.x) * (blockDim.x >> 5);
+    const int64_t gw = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t per = ((ngroups + nwarps - 1) / nwarps + 63) / 64 * 64;             // groups per warp
+    const int64_t g_end = (gw + 1) * per < ngroups ? (gw + 1) * per : ngroups;
+    int64_t g = gw * per + lane;
+    for (; g + 32 < g_end; g += 64) {                                                  // two groups in flight per lane
+        const RowGroup<VEC> r0 = load_group<VEC>(lp_train, lp_roll, mask, g);
+        const RowGroup<VEC> r1 = load_group<VEC>(lp_train, lp_roll, mask, g + 32);
+        clear();
+        add_group(r0, g);
+        add_group(r1, g + 32);
+        commit();
     }
+    clear();
+    if (g < g_end) add_group(load_group<VEC>(lp_train, lp_roll, mask, g), g);
+    flush();
+    // rows after the last whole group: the first threads of the grid, one row each
+    {
+        const int64_t t = ngroups * VEC + static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+        if (t < T && mask[t]) {
+            sq = -1;
+            cur = -1;
+            seek(t);
+            add_row(lp_train[t], lp_roll[t], adv[sq]);
+            flush();
+        }
+    }
+    commit();
     for (int i = 0; i < kNumMoments; ++i) {
         const double tot = block_sum(acc[i], scratch);
         if (threadIdx.x == 0) partials[blockIdx.x * kNumMoments + i] = tot;
@@ -378,26 +496,48 @@ __global__ void moments_reduce_kernel(const double* __restrict__ partials, int n
     moments[threadIdx.x] = m;
 }
 
-__global__ void rectify_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
-                               const uint8_t* __restrict__ mask, int64_t T, double logC, const ais_diag* __restrict__ diag,
-                               float* __restrict__ rho, float* __restrict__ w_tilde) {
-    const double alpha = diag->alpha;
-    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T;
-         t += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-        double r = 1.0, wt = 1.0;
-        if (mask[t]) {
-            const double dl = static_cast<double>(lp_train[t]) - static_cast<double>(lp_roll[t]);
-            r = exp(dl);
-            wt = 1.0 + alpha * (exp(fmin(dl, logC)) - 1.0);
+template <int VEC>
+__global__ void __launch_bounds__(256) rectify_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
+                                                      const uint8_t* __restrict__ mask, int64_t T, float C,
+                                                      const ais_diag* __restrict__ diag, float* __restrict__ rho,
+                                                      float* __restrict__ w_tilde) {
+    const float alpha = static_cast<float>(diag->alpha);
+    auto one = [&](float lt, float lr, uint8_t mk, float& r, float& wt) {
+        r = 1.0f;
+        wt = 1.0f;
+        if (mk) {
+            const float dl = lt - lr;
+            r = __expf(dl);
+            wt = fmaf(alpha, fminf(r, C) - 1.0f, 1.0f);
         }
-        if (rho) rho[t] = static_cast<float>(r);
-        w_tilde[t] = static_cast<float>(wt);
+    };
+    const int64_t ngroups = T / VEC;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
+        const RowGroup<VEC> in = load_group<VEC>(lp_train, lp_roll, mask, g);
+        float r[VEC], wt[VEC];
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) one(in.lt[j], in.lr[j], in.mk[j], r[j], wt[j]);
+        if (VEC == 4) {
+            if (rho) reinterpret_cast<float4*>(rho)[g] = make_float4(r[0], r[1 % VEC], r[2 % VEC], r[3 % VEC]);
+            reinterpret_cast<float4*>(w_tilde)[g] = make_float4(wt[0], wt[1 % VEC], wt[2 % VEC], wt[3 % VEC]);
+        } else {
+            if (rho) rho[g] = r[0];
+            w_tilde[g] = wt[0];
+        }
+    }
+    for (int64_t t = ngroups * VEC + static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
+        float r, wt;
+        one(lp_train[t], lp_roll[t], mask[t], r, wt);
+        if (rho) rho[t] = r;
+        w_tilde[t] = wt;
     }
 }
 
 // ------------------------------------------------------------------------------------------------
 // Per-token gradient factor c_t and the surrogate loss (Eq. ais-grpo without the KL term).
 // ------------------------------------------------------------------------------------------------
+template <int VEC>
 __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_old,
                                                                   const float* __restrict__ lp_ref, double beta_kl,
                                                                   const uint8_t* __restrict__ mask,
@@ -408,30 +548,58 @@ __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __
                                                                   float* __restrict__ coef) {
     __shared__ double scratch[32];
     double J = 0.0, KL = 0.0;
-    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T;
-         t += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    // one valid row of sequence sq: its share of the objective, of the KL estimate, and its gradient factor
+    auto one = [&](int64_t t, int sq, float wtf) -> float {
+        const double A = adv[sq];
+        const int n = n_valid_seq[sq] > 0 ? n_valid_seq[sq] : 1;
+        const double norm = 1.0 / (static_cast<double>(S_norm) * static_cast<double>(n));
+        const double rho_on = lp_old ? exp(static_cast<double>(lp_train[t]) - static_cast<double>(lp_old[t])) : 1.0;
+        const double un = rho_on * A;
+        const double cl = fmin(fmax(rho_on, 1.0 - clip_eps), 1.0 + clip_eps) * A;
+        const double wt = wtf;
         double c = 0.0;
-        if (mask[t]) {
-            const int s = seq_of_row(seq_offsets, S, t);
-            const double A = adv[s];
-            const int n = n_valid_seq[s] > 0 ? n_valid_seq[s] : 1;
-            const double norm = 1.0 / (static_cast<double>(S_norm) * static_cast<double>(n));
-            const double rho_on = lp_old ? exp(static_cast<double>(lp_train[t]) - static_cast<double>(lp_old[t])) : 1.0;
-            const double un = rho_on * A;
-            const double cl = fmin(fmax(rho_on, 1.0 - clip_eps), 1.0 + clip_eps) * A;
-            const double wt = w_tilde[t];
-            J += wt * fmin(un, cl) * norm;
-            if (un <= cl) c = wt * A * rho_on * norm;
-            if (lp_ref) {
-                // KL(pi_theta || pi_ref) estimate r - log r - 1, r = pi_ref / pi_theta; its slope in lp_theta is 1 - r
-                const double log_r = static_cast<double>(lp_ref[t]) - static_cast<double>(lp_train[t]);
-                const double r = exp(log_r);
-                KL += (r - log_r - 1.0) * norm;
-                c -= beta_kl * (1.0 - r) * norm;
+        J += wt * fmin(un, cl) * norm;
+        if (un <= cl) c = wt * A * rho_on * norm;
+        if (lp_ref) {
+            // KL(pi_theta || pi_ref) estimate r - log r - 1, r = pi_ref / pi_theta; its slope in lp_theta is 1 - r
+            const double log_r = static_cast<double>(lp_ref[t]) - static_cast<double>(lp_train[t]);
+            const double r = exp(log_r);
+            KL += (r - log_r - 1.0) * norm;
+            c -= beta_kl * (1.0 - r) * norm;
+        }
+        return static_cast<float>(c);
+    };
+    const int64_t ngroups = T / VEC;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; g < ngroups; g += stride) {
+        float c[VEC], wt[VEC];
+        uint8_t mk[VEC];
+        bool any = false;
+        if (VEC == 4) {
+            const uchar4 m = reinterpret_cast<const uchar4*>(mask)[g];
+            const float4 w4 = reinterpret_cast<const float4*>(w_tilde)[g];
+            mk[0] = m.x; mk[1 % VEC] = m.y; mk[2 % VEC] = m.z; mk[3 % VEC] = m.w;
+            wt[0] = w4.x; wt[1 % VEC] = w4.y; wt[2 % VEC] = w4.z; wt[3 % VEC] = w4.w;
+        } else {
+            mk[0] = mask[g];
+            wt[0] = w_tilde[g];
+        }
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) { c[j] = 0.f; any |= (mk[j] != 0); }
+        if (any) {
+            const int64_t t0 = g * VEC;
+            int sq = seq_of_row(seq_offsets, S, t0);
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) {
+                while (sq + 1 < S && static_cast<int64_t>(seq_offsets[sq + 1]) <= t0 + j) ++sq;
+                if (mk[j]) c[j] = one(t0 + j, sq, wt[j]);
             }
         }
-        coef[t] = static_cast<float>(c);
+        if (VEC == 4) reinterpret_cast<float4*>(coef)[g] = make_float4(c[0], c[1 % VEC], c[2 % VEC], c[3 % VEC]);
+        else coef[g] = c[0];
     }
+    for (int64_t t = ngroups * VEC + static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride)
+        coef[t] = mask[t] ? one(t, seq_of_row(seq_offsets, S, t), w_tilde[t]) : 0.f;
     const double tot = block_sum(J, scratch);
     const double tot_kl = block_sum(KL, scratch);
     if (threadIdx.x == 0) {
@@ -454,6 +622,34 @@ __global__ void loss_finalize_kernel(const double* __restrict__ partials, int nb
         diag->loss = total;
         diag->kl_ref = KL;
     }
+}
+
+// 16-byte loads need every per-row vector on a 16-byte boundary (the mask on a 4-byte one).
+inline bool vec4_ok(const void* a, const void* b, const void* c, const void* d, const void* m) {
+    const uintptr_t f = reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c) |
+                        reinterpret_cast<uintptr_t>(d);
+    return (f % 16 == 0) && (reinterpret_cast<uintptr_t>(m) % 4 == 0);
+}
+
+void launch_moments_kernel(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
+                           const float* adv, int64_t T, int S, float C, double* partials, int32_t* n_valid_seq,
+                           cudaStream_t stream) {
+    if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask))
+        moments_kernel<4><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials,
+                                                                      n_valid_seq);
+    else
+        moments_kernel<1><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials,
+                                                                      n_valid_seq);
+}
+
+void launch_rectify_kernel(const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T, float C,
+                           const ais_diag* diag, float* rho, float* w_tilde, cudaStream_t stream) {
+    const int64_t groups = (T + 3) / 4;
+    const int blocks = static_cast<int>(((groups + 255) / 256) < 2368 ? ((groups + 255) / 256) : 2368);
+    if (vec4_ok(lp_train, lp_roll, rho, w_tilde, mask))
+        rectify_kernel<4><<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde);
+    else
+        rectify_kernel<1><<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde);
 }
 
 }  // namespace
@@ -506,43 +702,41 @@ cudaError_t launch_tile_flags_coef(const float* coef, int64_t T, uint8_t* flags,
     return cudaGetLastError();
 }
 
-cudaError_t launch_seq_stats(const uint8_t* mask, const int32_t* seq_offsets, const float* rewards, int S, int G,
-                             int adv_std_norm, float eps, float* adv, int32_t* n_valid_seq, cudaStream_t stream) {
+cudaError_t launch_seq_counts(const uint8_t* mask, const int32_t* seq_offsets, int S, int32_t* n_valid_seq, cudaStream_t stream) {
     if (S == 0) return cudaSuccess;
-    seq_stats_kernel<<<S, 256, 0, stream>>>(mask, seq_offsets, rewards, G, adv_std_norm, eps, adv, n_valid_seq);
+    seq_count_kernel<<<(S + 7) / 8, 256, 0, stream>>>(mask, seq_offsets, S, n_valid_seq);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_advantages(const float* rewards, int S, int G, int adv_std_norm, float eps, float* adv, int32_t* zero_counts,
+                              cudaStream_t stream) {
+    if (S == 0) return cudaSuccess;
+    adv_kernel<<<(S + 255) / 256, 256, 0, stream>>>(rewards, S, G, adv_std_norm, eps, adv, zero_counts);
     return cudaGetLastError();
 }
 
 cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
-                        const float* adv, int64_t T, int S, const ais_params& p, double* partials, float* rho,
-                        float* w_tilde, ais_diag* diag, cudaStream_t stream) {
-    const double logC = log(static_cast<double>(p.C));
-    moments_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, logC, partials);
+                        const float* adv, int64_t T, int S, const ais_params& p, double* partials, int32_t* n_valid_seq,
+                        float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream) {
+    const float C = p.C;
+    launch_moments_kernel(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials, n_valid_seq, stream);
     diag_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, p, diag);
-    if (T > 0) {
-        const int blocks = static_cast<int>(((T + 255) / 256) < 1184 ? ((T + 255) / 256) : 1184);
-        rectify_kernel<<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, logC, diag, rho, w_tilde);
-    }
+    if (T > 0) launch_rectify_kernel(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde, stream);
     return cudaGetLastError();
 }
 
 cudaError_t launch_moments(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
-                           const float* adv, int64_t T, int S, const ais_params& p, double* partials, double* moments,
-                           cudaStream_t stream) {
-    const double logC = log(static_cast<double>(p.C));
-    moments_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, logC, partials);
+                           const float* adv, int64_t T, int S, const ais_params& p, double* partials, int32_t* n_valid_seq,
+                           double* moments, cudaStream_t stream) {
+    launch_moments_kernel(lp_train, lp_roll, mask, seq_offsets, adv, T, S, p.C, partials, n_valid_seq, stream);
     moments_reduce_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, moments);
     return cudaGetLastError();
 }
 
 cudaError_t launch_finalize(const double* moments, const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T,
                             const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream) {
-    const double logC = log(static_cast<double>(p.C));
     diag_finalize_kernel<<<1, 32, 0, stream>>>(moments, 1, p, diag);
-    if (T > 0) {
-        const int blocks = static_cast<int>(((T + 255) / 256) < 1184 ? ((T + 255) / 256) : 1184);
-        rectify_kernel<<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, logC, diag, rho, w_tilde);
-    }
+    if (T > 0) launch_rectify_kernel(lp_train, lp_roll, mask, T, p.C, diag, rho, w_tilde, stream);
     return cudaGetLastError();
 }
 
@@ -551,9 +745,14 @@ cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const f
                              const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S, int S_norm,
                              float clip_eps, double* partials, float* coef, float* loss, ais_diag* diag, cudaStream_t stream) {
     const float* ref = (beta_kl != 0.f) ? lp_ref : nullptr;
-    loss_coef_kernel<<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, ref, static_cast<double>(beta_kl), mask, seq_offsets,
-                                                                 adv, w_tilde, n_valid_seq, T, S, S_norm,
-                                                                 static_cast<double>(clip_eps), partials, coef);
+    if (vec4_ok(w_tilde, coef, nullptr, nullptr, mask))
+        loss_coef_kernel<4><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, ref, static_cast<double>(beta_kl), mask,
+                                                                        seq_offsets, adv, w_tilde, n_valid_seq, T, S, S_norm,
+                                                                        static_cast<double>(clip_eps), partials, coef);
+    else
+        loss_coef_kernel<1><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, ref, static_cast<double>(beta_kl), mask,
+                                                                        seq_offsets, adv, w_tilde, n_valid_seq, T, S, S_norm,
+                                                                        static_cast<double>(clip_eps), partials, coef);
     loss_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, ref ? static_cast<double>(beta_kl) : 0.0, loss, diag);
     return cudaGetLastError();
 }

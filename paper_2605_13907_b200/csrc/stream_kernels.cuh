@@ -9,7 +9,7 @@
 
 namespace ais {
 
-constexpr int kDiagBlocks = 296;      // fixed grid of the batch reductions (keeps the summation order fixed)
+constexpr int kDiagBlocks = 592;      // fixed grid of the batch reductions (keeps the summation order fixed)
 constexpr int kDiagThreads = 256;
 constexpr int kNumMoments = 12;
 
@@ -28,19 +28,22 @@ cudaError_t launch_combine(const float* part_m, const float* part_s, const float
 cudaError_t launch_tile_flags_mask(const uint8_t* mask, int64_t T, uint8_t* flags, cudaStream_t stream);
 cudaError_t launch_tile_flags_coef(const float* coef, int64_t T, uint8_t* flags, cudaStream_t stream);
 
-// n_valid_seq[s] and (when rewards != nullptr) adv[s].
-cudaError_t launch_seq_stats(const uint8_t* mask, const int32_t* seq_offsets, const float* rewards, int S, int G,
-                             int adv_std_norm, float eps, float* adv, int32_t* n_valid_seq, cudaStream_t stream);
+// n_valid_seq[s] = valid rows of sequence s.
+cudaError_t launch_seq_counts(const uint8_t* mask, const int32_t* seq_offsets, int S, int32_t* n_valid_seq, cudaStream_t stream);
+// adv[s] (group-relative advantages); zero_counts [S] (may be NULL) is cleared for the moments kernel to count into.
+cudaError_t launch_advantages(const float* rewards, int S, int G, int adv_std_norm, float eps, float* adv, int32_t* zero_counts,
+                              cudaStream_t stream);
 
+// n_valid_seq (may be NULL) must have been cleared: the moments kernel adds every sequence's valid rows to it.
 cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
                         const float* adv, int64_t T, int S, const ais_params& p, double* partials /*[kDiagBlocks][kNumMoments]*/,
-                        float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
+                        int32_t* n_valid_seq, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
 
 // The two halves of launch_diag: partial moments summed into `moments` [kNumMoments], and everything that follows
 // from a (possibly all-reduced) moment vector.
 cudaError_t launch_moments(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
-                           const float* adv, int64_t T, int S, const ais_params& p, double* partials, double* moments,
-                           cudaStream_t stream);
+                           const float* adv, int64_t T, int S, const ais_params& p, double* partials, int32_t* n_valid_seq,
+                           double* moments, cudaStream_t stream);
 cudaError_t launch_finalize(const double* moments, const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T,
                             const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
 
