@@ -1,0 +1,113 @@
+"""Layouts of the same batch must not change the result: sequences packed back to back against the same sequences
+padded to a common length with masked rows, and the batch reductions on vectors that do not start on a 16-byte
+boundary (the kernels then read row by row instead of four rows per load) and whose length is not a multiple of 4."""
+
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle import ais as oais
+
+pytestmark = pytest.mark.gpu
+
+
+def test_padded_sequences_equal_packed_sequences():
+    import paper_2605_13907_b200 as ais
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], d=256, V=1280, P=3, G=4, lengths="uniform:30:200", seed=71)
+    b = workloads.make_batch(w, device="cpu")
+    offs = b.seq_offsets.numpy().astype(np.int64)
+    S, lens = w.P * w.G, np.diff(offs)
+    L = int(lens.max()) + 7                                   # padded length, not a multiple of anything
+    g = torch.Generator().manual_seed(3)
+    Hp = torch.randn(S * L, w.d, generator=g).to(torch.bfloat16)        # padding rows hold arbitrary hidden states
+    tokp = torch.randint(0, w.V, (S * L,), generator=g, dtype=torch.int32)
+    mskp = torch.zeros(S * L, dtype=torch.uint8)
+    rows = np.concatenate([s * L + np.arange(lens[s]) for s in range(S)])   # where the packed rows sit in the padded batch
+    Hp[rows] = b.H
+    tokp[rows] = b.tokens
+    mskp[rows] = b.mask
+    offp = torch.arange(0, S * L + 1, L, dtype=torch.int32)
+
+    W = b.W.cuda()
+    rew = b.rewards.cuda()
+    packed = ais.AisStep(b.T, w.d, w.V, w.P, w.G, w.block)
+    packed.step(b.H.cuda(), W, b.tokens.cuda(), b.mask.cuda(), b.seq_offsets.cuda(), rew)
+    padded = ais.AisStep(S * L, w.d, w.V, w.P, w.G, w.block)
+    padded.step(Hp.cuda(), W, tokp.cuda(), mskp.cuda(), offp.cuda(), rew)
+    torch.cuda.synchronize()
+    assert int(packed.status.item()) == 0 and int(padded.status.item()) == 0
+
+    r = torch.as_tensor(rows)
+    # a row's logits do not depend on its neighbours: the per-row results are the same bits
+    for name in ("lp_train", "lse_train", "lp_roll", "rho"):
+        assert torch.equal(getattr(packed, name)[:b.T].cpu(), getattr(padded, name).cpu()[r]), name
+    dp, dq = packed.read_diag(), padded.read_diag()
+    assert dp["n_valid"] == dq["n_valid"] == float(b.mask.sum())
+    for k in ("alpha", "d_bar", "cv2", "ess", "delta_sigma", "loss"):
+        assert abs(dp[k] - dq[k]) <= 1e-6 * max(1.0, abs(dp[k])), k
+    assert torch.equal(packed.n_valid_seq.cpu(), padded.n_valid_seq.cpu())
+    dH_packed = packed.dH[:b.T].float().cpu()
+    dH_padded = padded.dH.float().cpu()
+    assert float((dH_packed - dH_padded[r]).norm()) <= 1e-3 * float(dH_packed.norm())      # alpha differs in the last bits
+    pad = torch.ones(S * L, dtype=torch.bool)
+    pad[r] = False
+    assert torch.all(dH_padded[pad] == 0) and torch.all(padded.lp_train.cpu()[pad] == 0) and torch.all(padded.rho.cpu()[pad] == 1)
+    # and both agree with the oracle on the packed batch
+    a = workloads.to_numpy(b)
+    ref = oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, w.block)
+    assert abs(dq["alpha"] - ref["diag"]["alpha"]) <= 1e-3
+    assert np.linalg.norm(dH_padded[r].numpy().astype(np.float64) - ref["dH"]) <= 1e-2 * np.linalg.norm(ref["dH"])
+
+
+@pytest.mark.parametrize("T,shift", [(1, 0), (3, 1), (1027, 0), (1027, 1), (4101, 3)])
+def test_batch_reductions_on_unaligned_and_ragged_vectors(T, shift):
+    import paper_2605_13907_b200 as ais
+    rng = np.random.default_rng(100 + T + shift)
+    P, G = 3, 2
+    S = P * G
+    # sequence boundaries anywhere, two of the sequences empty
+    cuts = np.sort(rng.integers(0, T + 1, S - 1))
+    cuts[1] = cuts[0]
+    cuts[-1] = T
+    offs = np.concatenate([[0], cuts, [T]]).astype(np.int32)
+    lp_t = -rng.uniform(0.1, 6.0, T).astype(np.float32)
+    lp_r = (lp_t + rng.normal(0, 0.3, T)).astype(np.float32)
+    mask = (rng.random(T) < 0.7).astype(np.uint8)
+    rew = (rng.random(S) < 0.5).astype(np.float32)
+    params = ais.default_params()
+    op = oais.Params()
+    ref_adv = oais.advantages(rew.astype(np.float64), G)
+    ref_diag = oais.diagnostics(lp_t, lp_r, mask, ref_adv[oais.seq_ids(offs, T)], op)
+    _, ref_rho, ref_wbar = oais.ratios(lp_t, lp_r, mask, op.C)
+    ref_wt = oais.rectify(ref_wbar, ref_diag["alpha"], mask)
+
+    def shifted(x):                                          # same values, storage starting `shift` elements later
+        buf = torch.empty(x.size + 8, dtype=torch.from_numpy(x).dtype, device="cuda")
+        v = buf[shift:shift + x.size]
+        v.copy_(torch.from_numpy(x))
+        return v
+
+    shape = ais.make_shape(T, 128, 1024, P, G, 128)
+    ws = torch.empty(ais.workspace_min_bytes(shape, params), dtype=torch.uint8, device="cuda")
+    d_lp_t, d_lp_r, d_mask = shifted(lp_t), shifted(lp_r), shifted(mask)
+    adv = torch.empty(S, device="cuda")
+    nseq = torch.full((S,), -1, dtype=torch.int32, device="cuda")
+    rho, wt = shifted(np.zeros(T, np.float32)), shifted(np.zeros(T, np.float32))
+    diag = torch.zeros(32, dtype=torch.float64, device="cuda")
+    ais.diagnostics(shape, params, d_lp_t, d_lp_r, d_mask, torch.from_numpy(offs).cuda(), torch.from_numpy(rew).cuda(), adv, nseq,
+                    rho, wt, diag, ws)
+    torch.cuda.synchronize()
+    d = ais.Diag.from_buffer_copy(diag.cpu().numpy().tobytes()[:ctypes.sizeof(ais.Diag)]).as_dict()
+    valid = mask.astype(bool)
+    counts = np.array([mask[offs[s]:offs[s + 1]].sum() for s in range(S)], np.int32)
+    assert np.array_equal(nseq.cpu().numpy(), counts)
+    assert d["n_valid"] == float(valid.sum())
+    for k in ("alpha", "alpha_ess", "alpha_mis", "alpha_var", "d_bar", "cv2", "delta_sigma", "mean_abs_dp", "kl_k1"):
+        assert abs(d[k] - ref_diag[k]) <= 1e-4 * max(1.0, abs(ref_diag[k])), (k, d[k], ref_diag[k])
+    assert np.allclose(adv.cpu().numpy(), ref_adv, atol=1e-6)
+    got_rho, got_wt = rho.cpu().numpy(), wt.cpu().numpy()
+    assert np.allclose(got_rho[valid], ref_rho[valid], rtol=1e-5) and np.all(got_rho[~valid] == 1)
+    assert np.allclose(got_wt[valid], ref_wt[valid], rtol=1e-4, atol=1e-5) and np.all(got_wt[~valid] == 1)
