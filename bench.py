@@ -197,8 +197,8 @@ def run_ours(args) -> None:
     # the HBM-bound kernels timed alone, before the long power-capped loop (burst conditions, like the copy that
     # measured the bandwidth they are compared with); inside the step they are bound by launch latency
     streaming = None
-    if rank == 0 and world == 1 and w.block and not args.prompts:
-        streaming = streaming_scale(dev, batch.W, w.block)
+    if rank == 0 and world == 1 and w.block and not args.prompts and not args.no_streaming:
+        streaming = streaming_scale(dev, batch.W, w.block, args.streaming_rows)
     for _ in range(args.warmup):
         one_step()
     barrier()
@@ -401,6 +401,10 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workspace-gb", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-streaming", action="store_true", help="skip the HBM-bound kernels timed alone at 2^26 rows")
+    ap.add_argument("--streaming-only", action="store_true",
+                    help="only time the HBM-bound kernels alone (batch reductions at --streaming-rows rows, quantiser on W)")
+    ap.add_argument("--streaming-rows", type=int, default=1 << 26)
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (small profiling case)")
     ap.add_argument("--compact", action="store_true",
                     help="pack the valid rows first (for workloads with scattered masks, e.g. llada_8b)")
@@ -410,6 +414,14 @@ def main() -> None:
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.streaming_only:
+        w = workloads.WORKLOADS[args.workload]
+        dev = torch.device("cuda:0")
+        torch.cuda.set_device(dev)
+        W = (torch.randn(w.V, w.d, device=dev) * w.w_std).to(torch.bfloat16)
+        out = streaming_scale(dev, W, w.block or 128, args.streaming_rows)
+        out["peak_gbs"] = _peaks()["hbm_gbs"]
+        print(json.dumps({"streaming": out}), flush=True)
     else:
         args.warmup = max(args.warmup, 3)
         run_ours(args)
