@@ -67,12 +67,21 @@ def logprob_train(H, W, tokens, mask):
     return log_softmax_gather(logits(H, W), tokens, mask)
 
 
+MX32 = -32        # `block` value selecting microscaling FP8 (E8M0 scale per 32 elements)
+
+
 def logprob_rollout(H, W, tokens, mask, block: int):
     """Rollout pass: weights and activations quantised to E4M3 per block along d
     (Section 2.1: 'we quantize both the weights and activations of the rollout model'),
     then the same log-softmax.  block = 0 selects one scale per tensor (Appendix 'FP8 rollout': per-tensor
-    dynamic scaling).  Returns (lp, lse, (qH, sH, qW, sW))."""
-    if block == 0:
+    dynamic scaling); block = MX32 selects power-of-two scales per 32 elements (the microscaling format named as
+    future work in the paper's limitations).  Returns (lp, lse, (qH, sH, qW, sW))."""
+    if block == MX32:
+        qH, sH = e4m3.quantize_mx(H)
+        qW, sW = e4m3.quantize_mx(W)
+        Hq = e4m3.dequantize_mx(qH, sH)
+        Wq = e4m3.dequantize_mx(qW, sW)
+    elif block == 0:
         qH, sH = e4m3.quantize_tensor(H)
         qW, sW = e4m3.quantize_tensor(W)
         Hq = e4m3.decode(qH) * np.float64(sH)

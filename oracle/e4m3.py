@@ -145,3 +145,64 @@ def dequantize_blocks(codes, scales, block: int) -> np.ndarray:
     vals = decode(codes).reshape(R, K // block, block)
     out = vals * np.asarray(scales, dtype=np.float64)[:, :, None]
     return out.reshape(R, K)
+
+
+# --------------------------------------------------------------------------- microscaling (power-of-two scales)
+MX_BLOCK = 32
+_MX_EMAX = 8              # exponent of the largest E4M3 binade: 448 = 1.75 * 2^8
+
+
+def quantize_mx(x):
+    """Microscaling FP8: blocks of 32 consecutive elements along the last axis share one power-of-two scale
+    stored as an 8-bit biased exponent (E8M0, bias 127) -- the format the paper's limitations section points to
+    for lower-precision rollouts.  Rule of the published OCP microscaling specification: the shared exponent is
+    floor(log2(max|x|)) minus the exponent of the element format's largest binade, X = floor(log2 amax) - 8, and
+    the elements are x / 2^X rounded to nearest-even onto the E4M3 grid, saturating (scaled magnitudes in
+    (448, 512) become 448).  The specification leaves an all-zero block open: scale code 127 (2^0) here.  Codes
+    are clamped to 0..254 (255 is the format's NaN).
+
+    Returns (codes uint8 [R, K], scale codes uint8 [R, K // 32]).
+    """
+    x64 = np.asarray(x, dtype=np.float64)
+    R, K = x64.shape
+    if K % MX_BLOCK:
+        raise ValueError("the last dimension must be a multiple of 32")
+    slab = max(1, (1 << 22) // max(K, 1))
+    if R > slab:
+        parts = [quantize_mx(x64[r0:r0 + slab]) for r0 in range(0, R, slab)]
+        return np.concatenate([p[0] for p in parts], axis=0), np.concatenate([p[1] for p in parts], axis=0)
+    xb = x64.reshape(R, K // MX_BLOCK, MX_BLOCK)
+    amax = np.max(np.abs(xb), axis=2)
+    _, e = np.frexp(amax)                                   # amax = m * 2^e, m in [0.5, 1): floor(log2 amax) = e - 1
+    X = np.where(amax > 0, e - 1 - _MX_EMAX, 0)
+    sc = np.clip(X + 127, 0, 254).astype(np.int64)
+    sc = np.where(amax > 0, sc, 127)
+    scaled = np.ldexp(xb, -(sc[:, :, None] - 127))          # exact: a power of two
+    scaled = np.clip(scaled, -3.0e38, 3.0e38).astype(np.float32)   # binary32 holds every scaled bf16 value exactly or saturates
+    codes = encode(scaled).reshape(R, K)
+    return codes, sc.astype(np.uint8)
+
+
+def dequantize_mx(codes, scale_codes) -> np.ndarray:
+    """codes [R, K], E8M0 scale codes [R, K // 32] -> float64 [R, K] = decode(q) * 2^(code - 127), exactly."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    R, K = codes.shape
+    vals = decode(codes).reshape(R, K // MX_BLOCK, MX_BLOCK)
+    out = np.ldexp(vals, np.asarray(scale_codes, dtype=np.int64)[:, :, None] - 127)
+    return out.reshape(R, K)
+
+
+def pack_mx_scales(scale_codes, row_pad: int = 128) -> np.ndarray:
+    """Layout of the scale codes that the GPU kernels exchange: chunks of 128 rows x 4 blocks (512 bytes), byte
+    (r % 32) * 16 + ((r % 128) // 32) * 4 + (kb % 4) of chunk (r // 128, kb // 4); rows are padded to a multiple
+    of `row_pad` with code 127.  This is the order in which the block-scaled tensor-core instruction wants one
+    stage's scales in tensor memory; it only permutes bytes."""
+    sc = np.asarray(scale_codes, dtype=np.uint8)
+    R, NB = sc.shape
+    if NB % 4:
+        raise ValueError("the number of blocks per row must be a multiple of 4")
+    Rp = (R + row_pad - 1) // row_pad * row_pad
+    full = np.full((Rp, NB), 127, np.uint8)
+    full[:R] = sc
+    v = full.reshape(Rp // 128, 4, 32, NB // 4, 4)          # [chunk row, r1, r0, chunk col, kb]
+    return np.ascontiguousarray(v.transpose(0, 3, 2, 1, 4)).reshape(Rp // 128, NB // 4, 512)

@@ -445,3 +445,28 @@ def test_full_path_runs_on_tiny_workload():
     assert out["dH"].shape == a["H"].shape
     assert 0 <= out["diag"]["alpha"] <= 1
     assert 1e-3 < out["diag"]["d_bar"] < 0.3
+
+
+def test_microscaling_rollout_equals_trainer_when_lossless():
+    """Every block on the E4M3 grid times a power of two: the microscaling rollout pass sees the same operands as
+    the trainer pass (zero divergence), and otherwise it differs by a small, non-zero amount."""
+    rng = np.random.default_rng(31)
+    T, d, V = 6, 64, 24
+    def lossless(rows):
+        codes = rng.integers(0, 256, size=(rows, d)).astype(np.uint8)
+        codes[(codes & 0x7F) == 0x7F] = 0x28
+        codes[(codes & 0x78) == 0x78] &= 0xBF                      # keep |values| <= 120 so that bf16 holds them exactly
+        codes[:, ::32] = 0x7E
+        k = rng.integers(-12, -6, size=(rows, d // 32))
+        return np.ldexp(e4m3.decode(codes).reshape(rows, d // 32, 32), k[:, :, None]).reshape(rows, d)
+    H, W = lossless(T), lossless(V)
+    tok = rng.integers(0, V, T)
+    mask = np.ones(T, np.uint8)
+    lp_t, _ = ais.logprob_train(H, W, tok, mask)
+    lp_r, _, _ = ais.logprob_rollout(H, W, tok, mask, ais.MX32)
+    assert np.array_equal(lp_t, lp_r)
+    H2 = np.asarray(rng.normal(size=(T, d)), np.float32).astype(np.float64)
+    lp_t2, _ = ais.logprob_train(H2, W, tok, mask)
+    lp_r2, _, _ = ais.logprob_rollout(H2, W, tok, mask, ais.MX32)
+    dlt = np.abs(lp_t2 - lp_r2)
+    assert 0 < dlt.max() < 0.5

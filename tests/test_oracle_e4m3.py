@@ -203,3 +203,80 @@ def test_per_tensor_quantisation():
     assert codes[i] & 0x7F == 0x7E
     z, sz = e4m3.quantize_tensor(np.zeros((3, 8), np.float32))
     assert sz == 1.0 and not z.any()
+
+
+# --------------------------------------------------------------------------- microscaling (E8M0 scale per 32 elements)
+def test_mx_shared_exponent_rule_and_saturation_band():
+    """Hand-worked blocks: the scale code is floor(log2 amax) - 8 + 127; a zero block gets 127; scaled magnitudes
+    between 448 and 512 saturate to 448 (the known clipping band of the microscaling rule)."""
+    def one(amax, fill=0.0):
+        x = np.full((1, 32), fill, np.float32)
+        x[0, 5] = amax
+        c, s = e4m3.quantize_mx(x)
+        return int(s[0, 0]), float(e4m3.dequantize_mx(c, s)[0, 5])
+    assert one(1.0) == (119, 1.0)                  # 1 = 256 * 2^-8
+    assert one(448.0) == (127, 448.0)
+    assert one(256.0) == (127, 256.0)
+    assert one(255.0) == (126, 224.0)              # floor(log2 255) = 7: 255 / 2^-1 = 510 saturates to 448, times 2^-1
+    assert one(0.0) == (127, 0.0)
+    assert one(-3.5) == (120, -3.5)                # 3.5 = 448 * 2^-7
+    assert one(480.0) == (127, 448.0)              # inside (448, 512): saturates
+    assert one(2.0 ** -140) == (0, 0.0)            # below the smallest scale: the code clamps at 0, the element underflows
+
+
+def test_mx_values_on_the_scaled_grid_round_trip_exactly():
+    rng = np.random.default_rng(21)
+    codes = rng.integers(0, 256, size=(8, 128)).astype(np.uint8)
+    codes[(codes & 0x7F) == 0x7F] = 0x30
+    codes[:, ::32] = 0x7E                                   # every block holds the largest magnitude 448
+    k = rng.integers(-20, 20, size=(8, 4))
+    x = np.ldexp(e4m3.decode(codes).reshape(8, 4, 32), k[:, :, None]).reshape(8, 128)
+    c, s = e4m3.quantize_mx(x)
+    assert np.array_equal(s.astype(np.int64), k + 127)
+    assert np.array_equal(e4m3.dequantize_mx(c, s), x)
+
+
+def test_mx_against_nearest_value_search():
+    """Independent restatement: exponent from math.frexp, element by exhaustive search for the nearest grid value
+    (ties to the even code), saturating."""
+    import math
+    rng = np.random.default_rng(22)
+    x = _bf16_round(rng.normal(size=(3, 64)) * np.exp(rng.normal(size=(3, 1)) * 4))
+    c, s = e4m3.quantize_mx(x)
+    grid = e4m3.decode(np.arange(127, dtype=np.uint8))                  # non-negative finite values, ascending
+    for r in range(3):
+        for b in range(2):
+            blk = x[r, 32 * b:32 * b + 32].astype(np.float64)
+            amax = float(np.abs(blk).max())
+            X = math.frexp(amax)[1] - 1 - 8
+            assert int(s[r, b]) == X + 127
+            for j, v in enumerate(blk):
+                t = min(abs(float(v)) / 2.0 ** X, 448.0)
+                d = np.abs(grid - t)
+                best = np.flatnonzero(d == d.min())
+                code = int(best[0]) if len(best) == 1 else int([q for q in best if q % 2 == 0][0])
+                assert int(c[r, 32 * b + j]) & 0x7F == code, (r, b, j, v)
+                assert (int(c[r, 32 * b + j]) >> 7) == int(np.signbit(v))
+
+
+def test_mx_error_bound():
+    rng = np.random.default_rng(23)
+    x = _bf16_round(rng.normal(size=(16, 256)))
+    c, s = e4m3.quantize_mx(x)
+    deq = e4m3.dequantize_mx(c, s)
+    scale = np.repeat(np.ldexp(1.0, s.astype(np.int64) - 127), 32, axis=1)
+    q = np.abs(x.astype(np.float64)) / scale
+    ok = (q >= 2.0 ** -6) & (q <= 448)
+    assert np.all(np.abs(deq - x)[ok] <= 2.0 ** -4 * np.abs(x)[ok])
+    assert np.all(q < 512)                                   # the shared exponent never lets an element reach 512
+
+
+def test_mx_scale_packing_positions():
+    """Byte (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4 of chunk (r // 128, kb // 4); padding rows hold 127."""
+    R, NB = 200, 8
+    sc = (np.arange(R)[:, None] * 7 + np.arange(NB)[None, :] * 3) % 250
+    p = e4m3.pack_mx_scales(sc.astype(np.uint8))
+    assert p.shape == (2, 2, 512)
+    for r, kb in [(0, 0), (31, 3), (32, 0), (127, 7), (128, 4), (199, 5)]:
+        assert p[r // 128, kb // 4, (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4] == sc[r, kb]
+    assert p[1, 0, (210 % 32) * 16 + ((210 % 128) // 32) * 4] == 127
