@@ -146,6 +146,8 @@ def run_ours(args) -> None:
         w = workloads.scaled(w, P=args.prompts)                       # reduced case for profiler captures
     if args.fp8_per_tensor:
         w = workloads.scaled(w, block=0)                              # variant: one FP8 scale per tensor
+    if args.fp8_mx:
+        w = workloads.scaled(w, block=ais.FP8_MX32)                   # variant: microscaling, E8M0 scale per 32 elements
     batch = workloads.make_batch(w, device=dev)
     if args.compact:
         # scattered masks: pack the valid rows once per batch (inside the step for the end-to-end figure) and run on those
@@ -197,7 +199,7 @@ def run_ours(args) -> None:
     # the HBM-bound kernels timed alone, before the long power-capped loop (burst conditions, like the copy that
     # measured the bandwidth they are compared with); inside the step they are bound by launch latency
     streaming = None
-    if rank == 0 and world == 1 and w.block and not args.prompts and not args.no_streaming:
+    if rank == 0 and world == 1 and w.block > 0 and not args.prompts and not args.no_streaming:
         streaming = streaming_scale(dev, batch.W, w.block, args.streaming_rows)
     for _ in range(args.warmup):
         one_step()
@@ -286,7 +288,7 @@ def run_ours(args) -> None:
         blk_rows = (step.workspace.numel() - fixed) // (_ld_u(w.V) * 2) // 128 * 128
         blk_rows = max(128, min(blk_rows, (T + 127) // 128 * 128))
         chunks = -(-T // blk_rows)
-        launches = (2 if w.block else 6) + 3 + 3 + (4 if world == 1 else 5) + 4 + (3 if args.with_dw else 2) * chunks
+        launches = (6 if w.block == 0 else 4 if w.block < 0 else 2) + 3 + 3 + (4 if world == 1 else 5) + 4 + (3 if args.with_dw else 2) * chunks
         out = {
             "metric": METRIC, "value": tokens_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -302,7 +304,7 @@ def run_ours(args) -> None:
                          "peak_source": peaks["source"] + " bf16 sustained (kernel timed inside a long step)",
                          "passes": {"fwd_roll_fp8_tflops": flops_pass / (seg["fwd_roll_fp8"] * 1e-3) / 1e12,
                                     "bwd_two_passes_tflops": (3 if args.with_dw else 2) * flops_pass / (seg["loss_bwd"] * 1e-3) / 1e12,
-                                    "quantize_gbs": (T + w.V) * w.d * (3.03 if w.block else 5.0) / (seg["quantize"] * 1e-3) / 1e9}},
+                                    "quantize_gbs": (T + w.V) * w.d * (3.0 + 4.0 / w.block if w.block > 0 else 3.03 if w.block < 0 else 5.0) / (seg["quantize"] * 1e-3) / 1e9}},
             "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches * args.steps,
             "clocks": clocks,
@@ -409,6 +411,8 @@ def main() -> None:
     ap.add_argument("--compact", action="store_true",
                     help="pack the valid rows first (for workloads with scattered masks, e.g. llada_8b)")
     ap.add_argument("--with-dw", action="store_true", help="variant: ais_loss_bwd also writes dW (a fifth tensor-core pass)")
+    ap.add_argument("--fp8-mx", action="store_true",
+                    help="variant (not the headline workload): microscaling FP8, power-of-two scale per 32 elements")
     ap.add_argument("--fp8-per-tensor", action="store_true",
                     help="variant (not the headline workload): per-tensor dynamic FP8 scaling instead of per-block scales")
     args = ap.parse_args()
@@ -419,7 +423,7 @@ def main() -> None:
         dev = torch.device("cuda:0")
         torch.cuda.set_device(dev)
         W = (torch.randn(w.V, w.d, device=dev) * w.w_std).to(torch.bfloat16)
-        out = streaming_scale(dev, W, w.block or 128, args.streaming_rows)
+        out = streaming_scale(dev, W, w.block if w.block > 0 else 128, args.streaming_rows)
         out["peak_gbs"] = _peaks()["hbm_gbs"]
         print(json.dumps({"streaming": out}), flush=True)
     else:

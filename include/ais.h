@@ -58,6 +58,8 @@ extern "C" {
 #define AIS_FLAG_NONFINITE    4u   /* a log-prob of a valid row is not finite               */
 #define AIS_FLAG_TIMEOUT      8u   /* a bounded device-side wait ran out; outputs undefined */
 
+#define AIS_FP8_MX32 (-32)        /* ais_shape.fp8_block: microscaling FP8, E8M0 scale per 32 elements */
+
 typedef struct ais_shape {
     int64_t T;            /* token rows                                                      */
     int32_t d;            /* hidden size                                                     */
@@ -65,7 +67,8 @@ typedef struct ais_shape {
     int32_t P;            /* prompts in the batch                                            */
     int32_t G;            /* responses per prompt; sequence s belongs to prompt s / G        */
     int32_t fp8_block;    /* elements along d sharing one FP8 scale: 32, 64 or 128;
-                             0 = one scale per tensor (ais_quantize_fp8_tensor)              */
+                             0 = one scale per tensor (ais_quantize_fp8_tensor);
+                             AIS_FP8_MX32 = power-of-two scale per 32 (ais_quantize_mxfp8)   */
     int32_t P_total;      /* prompts over all data-parallel ranks (loss normaliser); 0 = P    */
     int64_t ldh;          /* row stride of H (and of its codes) in elements                  */
     int64_t ldw;          /* row stride of W (and of its codes) in elements                  */
@@ -152,6 +155,25 @@ int ais_quantize_fp8_tensor(const void* x, int64_t rows, int64_t cols, int64_t l
                             uint8_t* codes, int64_t ldq, float* scale, void* stream);
 
 /*
+ * Microscaling FP8 (the lower-precision block-scaled formats that the paper's Limitations section names for future
+ * rollouts; format rule from the published OCP microscaling specification): every 32 consecutive elements of a row
+ * share the power-of-two scale 2^X, X = floor(log2 max|x|) - 8, stored as the byte X + 127 (clamped to 0..254; 127
+ * for an all-zero block), and the elements are E4M3_rne_saturating(x / 2^X).
+ * x       [rows, ld]  bf16, row-major; cols a multiple of 128
+ * codes   [rows, ldq] uint8                                   (written)
+ * scales  ais_mx_scale_bytes(rows, cols) bytes, 16-byte aligned (written): chunks of 128 rows x 4 blocks, chunk
+ *         (r / 128, kb / 4) at ((r / 128) * (cols / 128) + kb / 4) * 512, byte (r % 32) * 16 + ((r % 128) / 32) * 4
+ *         + kb % 4 inside it -- the order in which the block-scaled tensor-core instruction reads one K-step's
+ *         scales; rows are padded to a multiple of 256 with the neutral byte 127.
+ * With shape->fp8_block == AIS_FP8_MX32, ais_logprob_fwd takes such codes, reads sH / sW as these packed arrays
+ * (ldsH / ldsW are ignored) and lets tcgen05's block-scaled MMA apply the scales, so the whole contraction stays in
+ * tensor memory.
+ */
+size_t ais_mx_scale_bytes(int64_t rows, int64_t cols);
+int ais_quantize_mxfp8(const void* x, int64_t rows, int64_t cols, int64_t ld,
+                       uint8_t* codes, int64_t ldq, uint8_t* scales, void* stream);
+
+/*
  * Trainer and rollout log-probabilities (Algorithm 1: "full-precision log-probs" and the sampler's
  * log-probs entering rho_rt; Eq. logit-mismatch).  For every row t with mask[t] = 1:
  *     lse_train[t] = log sum_v exp(z[t,v]),  z = H W^T  (bf16 operands, fp32 accumulation)
@@ -159,13 +181,14 @@ int ais_quantize_fp8_tensor(const void* x, int64_t rows, int64_t cols, int64_t l
  *     lp_roll[t], lse_roll[t]: the same with z^[t,v] = sum_kb sH[kb,t] sW[kb,v] sum_{k in kb} qH[t,k] qW[v,k]
  * The train pass is skipped when lp_train is NULL; the rollout pass when lp_roll is NULL.
  * lse_train / lse_roll may be NULL when not wanted (lse_train is needed later by ais_loss_bwd).
- * sH is [d/B, ldsH] and sW is [d/B, ldsW] (block-major, as ais_quantize_fp8 writes them).
+ * sH is [d/B, ldsH] and sW is [d/B, ldsW] floats (block-major, as ais_quantize_fp8 writes them); one float each with
+ * fp8_block == 0; packed scale bytes with fp8_block == AIS_FP8_MX32.
  * tokens [T] int32, mask [T] uint8, dev_status: one uint32 on the device (OR-ed into; may be NULL).
  */
 int ais_logprob_fwd(const ais_shape* shape, const ais_params* params,
                     const void* H, const void* W,
-                    const uint8_t* qH, const float* sH, int64_t ldsH,
-                    const uint8_t* qW, const float* sW, int64_t ldsW,
+                    const uint8_t* qH, const void* sH, int64_t ldsH,
+                    const uint8_t* qW, const void* sW, int64_t ldsW,
                     const int32_t* tokens, const uint8_t* mask,
                     float* lp_train, float* lse_train, float* lp_roll, float* lse_roll,
                     uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream);

@@ -66,6 +66,10 @@ def lib() -> C.CDLL:
         L.ais_quantize_fp8.argtypes = [vp, i64, i64, i64, C.c_int, vp, i64, vp, i64, vp]
         L.ais_quantize_fp8_tensor.restype = C.c_int
         L.ais_quantize_fp8_tensor.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp]
+        L.ais_mx_scale_bytes.restype = sz
+        L.ais_mx_scale_bytes.argtypes = [i64, i64]
+        L.ais_quantize_mxfp8.restype = C.c_int
+        L.ais_quantize_mxfp8.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp]
         L.ais_logprob_fwd.restype = C.c_int
         L.ais_logprob_fwd.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, i64, vp, vp, i64, vp, vp,
                                       vp, vp, vp, vp, vp, vp, sz, vp]
@@ -135,12 +139,26 @@ def _require_cuda(*tensors):
             raise AisError("all tensors must live on a CUDA device; this library has no CPU path")
 
 
+FP8_MX32 = -32          # fp8_block value: microscaling FP8 (E8M0 scale per 32 elements, hardware block-scaled MMA)
+
+
+def mx_scale_bytes(rows: int, cols: int) -> int:
+    return int(lib().ais_mx_scale_bytes(rows, cols))
+
+
 def quantize_fp8(x: torch.Tensor, block: int, codes: torch.Tensor | None = None, scales: torch.Tensor | None = None):
-    """x [rows, cols] bf16 -> (codes [rows, cols] uint8, scales [cols/block, lds] float32, block-major)."""
+    """x [rows, cols] bf16 -> (codes [rows, cols] uint8, scales [cols/block, lds] float32, block-major);
+    block = 0: one scale per tensor; block = FP8_MX32: packed E8M0 scale bytes (see include/ais.h)."""
     _require_cuda(x, codes, scales)
     rows, cols = x.shape
     if codes is None:
         codes = torch.empty(rows, cols, dtype=torch.uint8, device=x.device)
+    if block == FP8_MX32:                            # power-of-two scale per 32 elements, packed scale bytes
+        if scales is None:
+            scales = torch.empty(mx_scale_bytes(rows, cols), dtype=torch.uint8, device=x.device)
+        _check(lib().ais_quantize_mxfp8(_ptr(x), rows, cols, x.stride(0), _ptr(codes), codes.stride(0), _ptr(scales),
+                                        _stream(x)), "ais_quantize_mxfp8")
+        return codes, scales
     if block == 0:                                   # one scale per tensor; scales holds it in its first element
         if scales is None:
             scales = torch.empty(1, 4, dtype=torch.float32, device=x.device)
@@ -159,8 +177,8 @@ def logprob_fwd(shape: Shape, params: Params, H, W, qH, sH, qW, sW, tokens, mask
                 dev_status, workspace):
     _require_cuda(H, W, qH, sH, qW, sW, tokens, mask, lp_train, lse_train, lp_roll, lse_roll, dev_status, workspace)
     _check(lib().ais_logprob_fwd(C.byref(shape), C.byref(params), _ptr(H), _ptr(W), _ptr(qH), _ptr(sH),
-                                 sH.stride(0) if sH is not None else 0, _ptr(qW), _ptr(sW),
-                                 sW.stride(0) if sW is not None else 0, _ptr(tokens), _ptr(mask), _ptr(lp_train),
+                                 sH.stride(0) if sH is not None and sH.dim() == 2 else 0, _ptr(qW), _ptr(sW),
+                                 sW.stride(0) if sW is not None and sW.dim() == 2 else 0, _ptr(tokens), _ptr(mask), _ptr(lp_train),
                                  _ptr(lse_train), _ptr(lp_roll), _ptr(lse_roll), _ptr(dev_status), _ptr(workspace),
                                  workspace.numel() * workspace.element_size(), _stream(workspace)), "ais_logprob_fwd")
 
@@ -280,7 +298,7 @@ class AisStep:
         self.params = params or default_params()
         S = P * G
         dev = self.device
-        nkb = d // fp8_block if fp8_block else 1
+        nkb = d // fp8_block if fp8_block > 0 else 1
         ws = workspace_bytes(self.shape, self.params)
         if ws == 0:
             raise AisError("invalid shape or parameters")
@@ -292,9 +310,13 @@ class AisStep:
             ws = max(ws_min, min(ws_all, workspace_bytes_cap))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
         self.qH = torch.empty(max(T, 1), ldh, dtype=torch.uint8, device=dev)[:, :d]
-        self.sH = torch.empty(nkb, max((T + 3) // 4 * 4, 4), dtype=torch.float32, device=dev)
         self.qW = torch.empty(V, ldw, dtype=torch.uint8, device=dev)[:, :d]
-        self.sW = torch.empty(nkb, (V + 3) // 4 * 4, dtype=torch.float32, device=dev)
+        if fp8_block == FP8_MX32:
+            self.sH = torch.empty(mx_scale_bytes(T, d), dtype=torch.uint8, device=dev)
+            self.sW = torch.empty(mx_scale_bytes(V, d), dtype=torch.uint8, device=dev)
+        else:
+            self.sH = torch.empty(nkb, max((T + 3) // 4 * 4, 4), dtype=torch.float32, device=dev)
+            self.sW = torch.empty(nkb, (V + 3) // 4 * 4, dtype=torch.float32, device=dev)
         f32 = dict(dtype=torch.float32, device=dev)
         self.lp_train = torch.empty(max(T, 1), **f32)
         self.lse_train = torch.empty(max(T, 1), **f32)

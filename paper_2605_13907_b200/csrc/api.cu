@@ -77,8 +77,9 @@ int check_shape(const ais_shape* s) {
     if (s->T < 0 || s->T > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
     if (s->d <= 0 || s->V <= 0 || s->P <= 0 || s->G <= 0) return AIS_ERR_SHAPE;
     if (s->d % 128 != 0 || s->V % 8 != 0) return AIS_ERR_SHAPE;
-    if (s->fp8_block != 0 && s->fp8_block != 32 && s->fp8_block != 64 && s->fp8_block != 128) return AIS_ERR_SHAPE;
-    if (s->fp8_block != 0 && s->d % s->fp8_block != 0) return AIS_ERR_SHAPE;
+    if (s->fp8_block != 0 && s->fp8_block != 32 && s->fp8_block != 64 && s->fp8_block != 128 && s->fp8_block != AIS_FP8_MX32)
+        return AIS_ERR_SHAPE;
+    if (s->fp8_block > 0 && s->d % s->fp8_block != 0) return AIS_ERR_SHAPE;
     if (s->ldh < s->d || s->ldw < s->d) return AIS_ERR_SHAPE;
     if (s->ldh % 16 != 0 || s->ldw % 16 != 0) return AIS_ERR_ALIGN;
     if (static_cast<int64_t>(s->P) * s->G > (1 << 24)) return AIS_ERR_SHAPE;
@@ -217,8 +218,28 @@ int ais_quantize_fp8_tensor(const void* x, int64_t rows, int64_t cols, int64_t l
                : AIS_ERR_DEVICE;
 }
 
+size_t ais_mx_scale_bytes(int64_t rows, int64_t cols) {
+    if (rows < 0 || cols <= 0 || cols % 128 != 0) return 0;
+    const int64_t chunks = (rows + 255) / 256 * 2;          // 128-row chunks, an even number of them
+    return static_cast<size_t>(chunks > 0 ? chunks : 2) * static_cast<size_t>(cols / 128) * 512;
+}
+
+int ais_quantize_mxfp8(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq, uint8_t* scales,
+                       void* stream) {
+    if (!x || !codes || !scales) return AIS_ERR_NULL;
+    if (rows < 0 || cols <= 0 || cols % 128 != 0 || ld < cols || ldq < cols) return AIS_ERR_SHAPE;
+    if (ld % 8 != 0 || ldq % 8 != 0 || !aligned(x, 16) || !aligned(codes, 8) || !aligned(scales, 16)) return AIS_ERR_ALIGN;
+    if (rows > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
+    int st = device_setup(nullptr);
+    if (st != AIS_OK) return st;
+    return launch_quantize_mx(x, rows, cols, ld, codes, ldq, scales, ais_mx_scale_bytes(rows, cols),
+                              static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? AIS_OK
+               : AIS_ERR_DEVICE;
+}
+
 int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void* H, const void* W, const uint8_t* qH,
-                    const float* sH, int64_t ldsH, const uint8_t* qW, const float* sW, int64_t ldsW, const int32_t* tokens,
+                    const void* sH_, int64_t ldsH, const uint8_t* qW, const void* sW_, int64_t ldsW, const int32_t* tokens,
                     const uint8_t* mask, float* lp_train, float* lse_train, float* lp_roll, float* lse_roll,
                     uint32_t* dev_status, void* workspace, size_t workspace_bytes, void* stream) {
     int st = check_shape(shape);
@@ -226,14 +247,18 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     st = check_params(params);
     if (st != AIS_OK) return st;
     if (!tokens || !mask) return AIS_ERR_NULL;
+    const float* sH = static_cast<const float*>(sH_);
+    const float* sW = static_cast<const float*>(sW_);
     const bool do_train = lp_train != nullptr, do_roll = lp_roll != nullptr;
     if (do_train && (!H || !W)) return AIS_ERR_NULL;
     if (do_roll && (!qH || !sH || !qW || !sW)) return AIS_ERR_NULL;
     if (do_train && (!aligned(H, 16) || !aligned(W, 16))) return AIS_ERR_ALIGN;
     const bool per_tensor = shape->fp8_block == 0;
+    const bool mx = shape->fp8_block == AIS_FP8_MX32;
     if (do_roll) {
         if (!aligned(qH, 16) || !aligned(qW, 16) || !aligned(sH, 4) || !aligned(sW, 4)) return AIS_ERR_ALIGN;
-        if (!per_tensor) {
+        if (mx && (!aligned(sH, 16) || !aligned(sW, 16))) return AIS_ERR_ALIGN;
+        if (!per_tensor && !mx) {
             if (!aligned(sH, 16) || !aligned(sW, 16)) return AIS_ERR_ALIGN;
             if (ldsH < shape->T || ldsW < shape->V) return AIS_ERR_SHAPE;
             if (ldsH % 4 != 0 || ldsW % 4 != 0) return AIS_ERR_ALIGN;
@@ -256,7 +281,7 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     a.ncols = shape->V;
     a.n_col_tiles = (shape->V + kBN - 1) / kBN;
     a.nsplit = L.nsplit;
-    a.sgroups = per_tensor ? 1 : 128 / shape->fp8_block;
+    a.sgroups = (per_tensor || mx) ? 1 : 128 / shape->fp8_block;
     a.tokens = tokens;
     a.mask = mask;
     a.part_m = reinterpret_cast<float*>(ws + L.off_part_m);
@@ -282,7 +307,20 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
             cudaSuccess)
             return AIS_ERR_DEVICE;
     }
-    if (do_roll && per_tensor) {
+    if (do_roll && mx) {
+        // power-of-two scales per 32 elements: the block-scaled MMA applies them, the contraction stays in tensor memory
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
+            return AIS_ERR_DEVICE;
+        a.ksteps = shape->d / 128;
+        a.sf_a = static_cast<const uint8_t*>(sH_);
+        a.sf_b = static_cast<const uint8_t*>(sW_);
+        a.nk4 = shape->d / 128;
+        if (launch_lmhead(kFwdMx, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
+        if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_roll, lse_roll, dev_status, s) !=
+            cudaSuccess)
+            return AIS_ERR_DEVICE;
+    } else if (do_roll && per_tensor) {
         // one scale per tensor: the whole contraction accumulates in tensor memory, the scales meet in the epilogue
         if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
             !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B))

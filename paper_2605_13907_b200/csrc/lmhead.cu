@@ -23,7 +23,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* stage_base = smem;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+    uint8_t* mx_scale_base = smem + kStages * kStageBytes;      // microscaling pass: one scale triple per stage
+    uint64_t* bars = reinterpret_cast<uint64_t*>(mx_scale_base + kStages * kMxStageScaleBytes);
     uint64_t* full = bars;                       // [kStages]   TMA -> MMA
     uint64_t* empty = full + kStages;            // [kStages]   MMA -> TMA
     uint64_t* tfull = empty + kStages;           // [2]         MMA -> epilogue
@@ -36,7 +37,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     constexpr int STG = TWO_ACC ? kDhStages : kStages;                          // depth of the stage ring
     constexpr int STG_BYTES = TWO_ACC ? kDhStageBytes : kStageBytes;
     constexpr int A_BYTES = TWO_ACC ? 2 * kAStageBytes : kAStageBytes;
-    constexpr int NBUF = TWO_ACC ? 1 : 2;                                       // accumulator sets that alternate
+    constexpr bool MX = (MODE == kFwdMx);                                       // block scales live in tensor memory
+    constexpr int NBUF = (TWO_ACC || MX) ? 1 : 2;                               // accumulator sets that alternate
+    constexpr uint32_t kMxScaleCol = 256;                                       // MX: scale columns after the accumulator
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int num_units = TWO_ACC ? a.n_row_tiles * a.n_col_tiles : a.n_row_tiles * a.nsplit;
@@ -73,8 +76,19 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag)) { ok = false; break; }
                         uint8_t* sA = stage_base + st.idx * STG_BYTES;
                         uint8_t* sB = sA + A_BYTES;
-                        mbar_expect_tx(&full[st.idx], STG_BYTES);
-                        const int kelem = (MODE == kFwdFp8T) ? ks * 128 : ks * 64;
+                        mbar_expect_tx(&full[st.idx], MX ? STG_BYTES + kMxStageScaleBytes : STG_BYTES);
+                        const int kelem = (MODE == kFwdFp8T || MX) ? ks * 128 : ks * 64;
+                        if (MX) {
+                            // the stage's scales: one chunk for the 128 rows of A, two for the 256 rows of B
+                            uint8_t* sS = mx_scale_base + st.idx * kMxStageScaleBytes;
+                            bulk_load(sS, a.sf_a + (static_cast<int64_t>(w.rt) * a.nk4 + ks) * kMxChunkBytes, kMxChunkBytes,
+                                      &full[st.idx]);
+                            bulk_load(sS + kMxChunkBytes, a.sf_b + (static_cast<int64_t>(2 * t) * a.nk4 + ks) * kMxChunkBytes,
+                                      kMxChunkBytes, &full[st.idx]);
+                            bulk_load(sS + 2 * kMxChunkBytes,
+                                      a.sf_b + (static_cast<int64_t>(2 * t + 1) * a.nk4 + ks) * kMxChunkBytes, kMxChunkBytes,
+                                      &full[st.idx]);
+                        }
                         if (MODE == kBwdDh) {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kDhRows);
                             tma_load_2d(sA + kAStageBytes, &tmA, &full[st.idx], kelem, w.rt * kDhRows + kBM);
@@ -113,7 +127,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc =
-                (MODE == kFwdFp8T) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
+                (MODE == kFwdFp8T || MX) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
                                   : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, MODE == kBwdDw ? 1 : 0, TWO_ACC ? 1 : 0);
             Pipe st(STG), tb(NBUF);
             bool ok = true;
@@ -147,6 +161,22 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                 mma_f16(tmem_base, smem_desc_sw128(sA + j * 2048, kAStageBytes / 2, 1024), bdesc, idesc, accum);
                                 mma_f16(tmem_base + kBN, smem_desc_sw128(sA + kAStageBytes + j * 2048, kAStageBytes / 2, 1024), bdesc,
                                         idesc, accum);
+                            }
+                        } else if (MX) {
+                            // scales of this stage: shared memory -> tensor memory (two column sets alternate between
+                            // stages), then one block-scaled instruction per 32-element block with its scale id
+                            const uint32_t sS = smem_u32(mx_scale_base + st.idx * kMxStageScaleBytes);
+                            const uint32_t tsf = tmem_base + kMxScaleCol + (st.idx & 1) * 16;
+#pragma unroll
+                            for (int c = 0; c < 3; ++c)
+                                tmem_cp_32x128b_warpx4(tsf + 4 * c, smem_desc_noswizzle(sS + c * kMxChunkBytes, 16, 128));
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const uint64_t adesc = smem_desc_sw128(sA + j * 32, 16, 1024);
+                                const uint64_t bdesc = smem_desc_sw128(sB + j * 32, 16, 1024);
+                                const uint32_t sel = static_cast<uint32_t>(j) << 30;      // byte of the scale columns
+                                mma_mxf8(tmem_base, adesc, bdesc, make_idesc_mx(kBM, kBN, j), tsf | sel, (tsf + 4) | sel,
+                                         (ks > 0 || j > 0) ? 1u : 0u);
                             }
                         } else {
                             const uint32_t dcol = tmem_base + tb.idx * kBN;
@@ -323,7 +353,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             for (int i = 0; i < 32; ++i) x[i] *= tscale;
                         }
                     }
-                    if (MODE == kFwdBf16 || MODE == kFwdFp8T) {
+                    if (MODE == kFwdBf16 || MODE == kFwdFp8T || MX) {
                         if (y >= col0 && y < col0 + 32) {
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
@@ -366,7 +396,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (lane == 0) mbar_arrive(&tempty[tb.idx]);
                 tb.advance();
             }
-            if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8T)) {
+            if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8T || MX)) {
                 const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow;
                 a.part_m[o] = m2 * kLn2;
                 a.part_s[o] = s;
@@ -406,6 +436,7 @@ cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& t
         case kBwdDh:   return launch_mode<kBwdDh>(tmA, tmB, args, num_ctas, stream);
         case kFwdFp8T: return launch_mode<kFwdFp8T>(tmA, tmB, args, num_ctas, stream);
         case kBwdDw:   return launch_mode<kBwdDw>(tmA, tmB, args, num_ctas, stream);
+        case kFwdMx:   return launch_mode<kFwdMx>(tmA, tmB, args, num_ctas, stream);
     }
     return cudaErrorInvalidValue;
 }
@@ -422,7 +453,9 @@ cudaError_t lmhead_prepare() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lmhead_kernel<kFwdFp8T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(lmhead_kernel<kBwdDw>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(lmhead_kernel<kBwdDw>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(lmhead_kernel<kFwdMx>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
 }  // namespace ais

@@ -13,7 +13,8 @@ enum LmheadMode : int {
     kBwdP    = 2,   // recompute z (bf16), write u = softmax - onehot as bf16 scratch
     kBwdDh   = 3,   // dH = c (.) (U W), contraction over the vocabulary
     kFwdFp8T = 4,   // E4M3 codes with one scale per tensor: whole contraction in tensor memory, one multiply after
-    kBwdDw   = 5    // dW += U^T H, contraction over the rows (both operands read with the contraction axis as rows)
+    kBwdDw   = 5,   // dW += U^T H, contraction over the rows (both operands read with the contraction axis as rows)
+    kFwdMx   = 6    // E4M3 codes with one power-of-two (E8M0) scale per 32 elements: hardware block-scaled MMA
 };
 
 constexpr int kBM = 128;                 // rows per tile (TMEM lanes)
@@ -29,9 +30,12 @@ constexpr int kDhStageBytes = 2 * kAStageBytes + kBStageBytes;
 constexpr int kDhStages = 3;
 static_assert(kDhStages * kDhStageBytes <= kStages * kStageBytes, "the dH stage ring must fit the same shared memory");
 constexpr int kNumBarriers = 2 * kStages + 4 + 1;
+// microscaling pass: per stage one 512-byte scale chunk for the 128 rows of A and two for the 256 rows of B
+constexpr int kMxChunkBytes = 512;
+constexpr int kMxStageScaleBytes = 3 * kMxChunkBytes;
 constexpr int kThreads = 384;            // warp 0 TMA, warp 1 MMA, warps 2..3 idle, warps 4..11 epilogue
 constexpr int kEpiWarps = 8;
-constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kNumBarriers * 8 + 64;
+constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kStages * kMxStageScaleBytes + kNumBarriers * 8 + 64;
 
 struct LmheadArgs {
     int64_t rows;          // valid rows handled by this launch
@@ -55,6 +59,9 @@ struct LmheadArgs {
     const float* scale_a;  // per-tensor FP8: the two scales (one float each, on the device)
     const float* scale_b;
     const float* coef;     // recompute: per-row factor c_t folded into the scratch
+    const uint8_t* sf_a;   // microscaling: packed scale chunks of A [row chunks of 128][d/128][512 bytes]
+    const uint8_t* sf_b;   // and of B
+    int32_t nk4;           // d / 128: scale chunks per 128 rows
     float* dW;             // dW pass: [V, lddw] fp32
     int64_t lddw;
     int32_t dw_accumulate; // dW pass: add to what dW holds instead of overwriting it

@@ -125,6 +125,58 @@ __global__ void __launch_bounds__(kQThreads) quantize_kernel(const __nv_bfloat16
 }
 
 // ------------------------------------------------------------------------------------------------
+// Microscaling FP8: 32 consecutive elements share a power-of-two scale 2^X, X = floor(log2 amax) - 8, stored as the
+// biased exponent X + 127 (clamped to 0..254; 127 for an all-zero block); the elements are x / 2^X on the E4M3 grid
+// (round to nearest even, saturating).  With bf16 inputs everything is exact integer work on exponent fields: the
+// block's amax pattern gives the scale code, and the multiplier 2^-X is a float built from its exponent field.
+// Four lanes (8 elements each) form a block.  The scale codes leave in the order the block-scaled MMA wants them:
+// chunks of 128 rows x 4 blocks, byte (r % 32) * 16 + ((r % 128) / 32) * 4 + kb % 4 of chunk (r / 128, kb / 4).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kQThreads) quantize_mx_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols,
+                                                                int64_t ld, uint8_t* __restrict__ codes, int64_t ldq,
+                                                                uint8_t* __restrict__ scales) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kQRows;
+    const int64_t col0 = static_cast<int64_t>(blockIdx.x) * kQCols;
+    const int64_t nk4 = cols / 128;
+#pragma unroll 1
+    for (int rr = 0; rr < 4; ++rr) {
+        const int64_t row = row0 + warp * 4 + rr;
+        if (row >= rows) break;
+#pragma unroll
+        for (int it = 0; it < kQIters; ++it) {
+            const int64_t col = col0 + it * 256 + lane * 8;
+            const bool in = col < cols;                     // cols is a multiple of 128: a block is wholly in or out
+            const uint4 raw = in ? __ldg(reinterpret_cast<const uint4*>(x + row * ld + col)) : make_uint4(0, 0, 0, 0);
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+            uint32_t m = __vmaxu2(__vmaxu2(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu), __vmaxu2(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu));
+            m = max(m & 0xFFFFu, m >> 16);
+            m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
+            m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
+            const int e = static_cast<int>(m >> 7);         // biased exponent of amax (0 for zero and subnormals)
+            const int code = m == 0u ? 127 : max(e - 8, 0);
+            const float mult = __uint_as_float(static_cast<uint32_t>(254 - code) << 23);      // 2^(127 - code), exact
+            if (!in) continue;
+            float q[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                q[2 * i] = __uint_as_float(w[i] << 16) * mult;
+                q[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u) * mult;
+            }
+            uint2 out;
+            out.x = static_cast<uint32_t>(cvt_e4m3x2(q[1], q[0])) | (static_cast<uint32_t>(cvt_e4m3x2(q[3], q[2])) << 16);
+            out.y = static_cast<uint32_t>(cvt_e4m3x2(q[5], q[4])) | (static_cast<uint32_t>(cvt_e4m3x2(q[7], q[6])) << 16);
+            *reinterpret_cast<uint2*>(codes + row * ldq + col) = out;
+            if ((lane & 3) == 0) {
+                const int64_t kb = col / 32;
+                scales[((row >> 7) * nk4 + (kb >> 2)) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4 + (kb & 3)] =
+                    static_cast<uint8_t>(code);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Per-tensor dynamic scaling: one scale for the whole matrix.  Pass 1 folds max|x| (as a bf16 bit pattern; the
 // patterns of non-negative values order like the values, so an integer atomicMax is exact and order-free)
 // into the word that will hold the scale, pass 2 turns it into s = amax / 448, pass 3 quantises.
@@ -666,6 +718,17 @@ cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t l
         case 128: quantize_kernel<128><<<grid, kQThreads, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scales, lds); break;
         default: return cudaErrorInvalidValue;
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_mx(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,
+                               uint8_t* scales, size_t scale_bytes, cudaStream_t stream) {
+    // rows that pad the last chunks carry the neutral scale
+    cudaError_t e = cudaMemsetAsync(scales, 127, scale_bytes, stream);
+    if (e != cudaSuccess) return e;
+    if (rows == 0 || cols == 0) return cudaSuccess;
+    dim3 grid(static_cast<unsigned>((cols + kQCols - 1) / kQCols), static_cast<unsigned>((rows + kQRows - 1) / kQRows));
+    quantize_mx_kernel<<<grid, kQThreads, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), rows, cols, ld, codes, ldq, scales);
     return cudaGetLastError();
 }
 

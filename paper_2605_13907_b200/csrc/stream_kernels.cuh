@@ -16,6 +16,11 @@ constexpr int kNumMoments = 12;
 cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes,
                             int64_t ldq, float* scales, int64_t lds, cudaStream_t stream);
 
+// Microscaling: E8M0 scale per 32 elements, packed in 512-byte chunks of 128 rows x 4 blocks; `scale_bytes` is the
+// size of the whole packed array (rows padded to a multiple of 256), filled with the neutral code first.
+cudaError_t launch_quantize_mx(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,
+                               uint8_t* scales, size_t scale_bytes, cudaStream_t stream);
+
 // One scale for the whole matrix (written to *scale on the device), then the codes.
 cudaError_t launch_quantize_tensor(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,
                                    float* scale, cudaStream_t stream);
