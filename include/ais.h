@@ -162,9 +162,10 @@ int ais_quantize_fp8_tensor(const void* x, int64_t rows, int64_t cols, int64_t l
  * x       [rows, ld]  bf16, row-major; cols a multiple of 128
  * codes   [rows, ldq] uint8                                   (written)
  * scales  ais_mx_scale_bytes(rows, cols) bytes, 16-byte aligned (written): chunks of 128 rows x 4 blocks, chunk
- *         (r / 128, kb / 4) at ((r / 128) * (cols / 128) + kb / 4) * 512, byte (r % 32) * 16 + ((r % 128) / 32) * 4
- *         + kb % 4 inside it -- the order in which the block-scaled tensor-core instruction reads one K-step's
- *         scales; rows are padded to a multiple of 256 with the neutral byte 127.
+ *         (r / 128, kb / 4) at ((r / 256) * (cols / 128) + kb / 4) * 1024 + ((r % 256) / 128) * 512, byte
+ *         (r % 32) * 16 + ((r % 128) / 32) * 4 + kb % 4 inside it -- the order in which the block-scaled
+ *         tensor-core instruction reads one K-step's scales; rows are padded to a multiple of 256 with the
+ *         neutral byte 127.
  * With shape->fp8_block == AIS_FP8_MX32, ais_logprob_fwd takes such codes, reads sH / sW as these packed arrays
  * (ldsH / ldsW are ignored) and lets tcgen05's block-scaled MMA apply the scales, so the whole contraction stays in
  * tensor memory.

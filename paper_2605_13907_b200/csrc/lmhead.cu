@@ -62,8 +62,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Microscaling pass: its one accumulator is read into registers in one go so that it can go back to the MMA
+    // issuer at once; the first warpgroup hands the registers for that to the epilogue (384 x 168 = 128 x 40 + 256 x 232).
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
+        if (MX) reg_dealloc<40>();
         if (lane == 0) {
             Pipe st(STG);
             uint32_t issued = 0;
@@ -79,15 +82,13 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         mbar_expect_tx(&full[st.idx], MX ? STG_BYTES + kMxStageScaleBytes : STG_BYTES);
                         const int kelem = (MODE == kFwdFp8T || MX) ? ks * 128 : ks * 64;
                         if (MX) {
-                            // the stage's scales: one chunk for the 128 rows of A, two for the 256 rows of B
+                            // the stage's scales: one 512-byte chunk for the 128 rows of A, the two adjacent chunks of B's 256 rows
                             uint8_t* sS = mx_scale_base + st.idx * kMxStageScaleBytes;
-                            bulk_load(sS, a.sf_a + (static_cast<int64_t>(w.rt) * a.nk4 + ks) * kMxChunkBytes, kMxChunkBytes,
-                                      &full[st.idx]);
-                            bulk_load(sS + kMxChunkBytes, a.sf_b + (static_cast<int64_t>(2 * t) * a.nk4 + ks) * kMxChunkBytes,
+                            bulk_load(sS, a.sf_a + (static_cast<int64_t>(w.rt >> 1) * a.nk4 + ks) * (2 * kMxChunkBytes) +
+                                              (w.rt & 1) * kMxChunkBytes,
                                       kMxChunkBytes, &full[st.idx]);
-                            bulk_load(sS + 2 * kMxChunkBytes,
-                                      a.sf_b + (static_cast<int64_t>(2 * t + 1) * a.nk4 + ks) * kMxChunkBytes, kMxChunkBytes,
-                                      &full[st.idx]);
+                            bulk_load(sS + kMxChunkBytes, a.sf_b + (static_cast<int64_t>(t) * a.nk4 + ks) * (2 * kMxChunkBytes),
+                                      2 * kMxChunkBytes, &full[st.idx]);
                         }
                         if (MODE == kBwdDh) {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kDhRows);
@@ -125,6 +126,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        if (MX) reg_dealloc<40>();
         if (lane == 0) {
             constexpr uint32_t idesc =
                 (MODE == kFwdFp8T || MX) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
@@ -200,8 +202,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             // everything issued has to finish before the tensor memory is given back
             tc_commit(done);
         }
-    } else if (warp >= 4) {
+    } else if (warp < 4) {
+        if (MX) reg_dealloc<40>();          // the idle warps of the first warpgroup give their registers away too
+    } else {
         // ------------------------------------------------------------------ epilogue warps
+        if (MX) reg_alloc<232>();
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int half = (warp - 4) >> 2;             // column half of the accumulator
         const int r_in_tile = q * 32 + lane;
@@ -338,11 +343,25 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 }
 
                 const uint32_t taddr = tmem_base + lane_addr + tb.idx * kBN + half * 128;
+                uint32_t vv[MX ? 4 : 1][32];
+                if (MX) {
+                    // the thread's 128 columns at once, then the accumulator is free for the next tile's MMAs
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld32(taddr + c * 32, vv[MX ? c : 0]);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld_wait(vv[MX ? c : 0]);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tempty[tb.idx]);
+                }
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const int col0 = col_base + c * 32;
                     float x[32];
-                    {
+                    if (MX) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(vv[MX ? c : 0][i]);
+                    } else {
                         uint32_t v[32];
                         tmem_ld32(taddr + c * 32, v);
                         tmem_ld_wait(v);
@@ -391,9 +410,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         }
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&tempty[tb.idx]);
+                if (!MX) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tempty[tb.idx]);
+                }
                 tb.advance();
             }
             if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8T || MX)) {

@@ -130,7 +130,8 @@ __global__ void __launch_bounds__(kQThreads) quantize_kernel(const __nv_bfloat16
 // (round to nearest even, saturating).  With bf16 inputs everything is exact integer work on exponent fields: the
 // block's amax pattern gives the scale code, and the multiplier 2^-X is a float built from its exponent field.
 // Four lanes (8 elements each) form a block.  The scale codes leave in the order the block-scaled MMA wants them:
-// chunks of 128 rows x 4 blocks, byte (r % 32) * 16 + ((r % 128) / 32) * 4 + kb % 4 of chunk (r / 128, kb / 4).
+// chunks of 128 rows x 4 blocks, byte (r % 32) * 16 + ((r % 128) / 32) * 4 + kb % 4 of chunk (r / 128, kb / 4); the two
+// chunks of a 256-row group are adjacent: chunk start ((r / 256) * (cols / 128) + kb / 4) * 1024 + ((r % 256) / 128) * 512.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kQThreads) quantize_mx_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols,
                                                                 int64_t ld, uint8_t* __restrict__ codes, int64_t ldq,
@@ -169,8 +170,8 @@ __global__ void __launch_bounds__(kQThreads) quantize_mx_kernel(const __nv_bfloa
             *reinterpret_cast<uint2*>(codes + row * ldq + col) = out;
             if ((lane & 3) == 0) {
                 const int64_t kb = col / 32;
-                scales[((row >> 7) * nk4 + (kb >> 2)) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4 + (kb & 3)] =
-                    static_cast<uint8_t>(code);
+                scales[((row >> 8) * nk4 + (kb >> 2)) * 1024 + ((row >> 7) & 1) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4 +
+                       (kb & 3)] = static_cast<uint8_t>(code);
             }
         }
     }

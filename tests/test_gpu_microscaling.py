@@ -36,7 +36,7 @@ def test_mx_quantiser_bit_exact():
     torch.cuda.synchronize()
     ref_c, ref_s = e4m3.quantize_mx(xb.float().numpy())
     assert np.array_equal(codes.cpu().numpy(), ref_c)
-    ref_p = e4m3.pack_mx_scales(ref_s, row_pad=256)
+    ref_p = e4m3.pack_mx_scales(ref_s)
     assert packed.numel() == ref_p.size == ais.mx_scale_bytes(rows, cols)
     assert np.array_equal(packed.cpu().numpy().reshape(ref_p.shape), ref_p)
 
@@ -56,8 +56,8 @@ def test_mx_rollout_path(case):
     T = b.T
     assert int(step.status.item()) == 0
     assert np.array_equal(step.qH.cpu().numpy()[:T], ref["qH"]) and np.array_equal(step.qW.cpu().numpy(), ref["qW"])
-    assert np.array_equal(step.sW.cpu().numpy(), e4m3.pack_mx_scales(ref["sW"], row_pad=256).reshape(-1))
-    assert np.array_equal(step.sH.cpu().numpy(), e4m3.pack_mx_scales(ref["sH"], row_pad=256).reshape(-1))
+    assert np.array_equal(step.sW.cpu().numpy(), e4m3.pack_mx_scales(ref["sW"]).reshape(-1))
+    assert np.array_equal(step.sH.cpu().numpy(), e4m3.pack_mx_scales(ref["sH"]).reshape(-1))
     err = np.abs(step.lp_roll.cpu().numpy()[:T] - ref["lp_roll"])
     assert err.max() <= LP_ATOL, err.max()
     assert err.max() <= 1e-4                                 # power-of-two scales are exact: only fp32 accumulation differs
@@ -86,21 +86,21 @@ def test_mx_fullsize_sampled_rows():
     qHs, sHs = e4m3.quantize_mx(Hs)
     assert np.array_equal(step.qH.cpu().numpy()[rows], qHs)
     Hq = e4m3.dequantize_mx(qHs, sHs)
-    sH_gpu = step.sH.cpu().numpy().reshape(-1, w.d // 128, 512)
+    sH_gpu = step.sH.cpu().numpy().reshape(-1, w.d // 128, 2, 512)
     for i, r in enumerate(rows):
         for kb in (0, 1, 63, 127):
-            assert sH_gpu[r // 128, kb // 4, (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4] == sHs[i, kb]
+            assert sH_gpu[r // 256, kb // 4, (r % 256) // 128, (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4] == sHs[i, kb]
     qW_gpu = step.qW.cpu().numpy()
-    sW_gpu = step.sW.cpu().numpy().reshape(-1, w.d // 128, 512)
+    sW_gpu = step.sW.cpu().numpy().reshape(-1, w.d // 128, 2, 512)
     z = np.empty((len(rows), w.V))
-    CH = 4096                                               # a multiple of 128: whole scale chunks per piece
+    CH = 4096                                               # a multiple of 256: whole scale groups per piece
     for v0 in range(0, w.V, CH):
         Wc = batch.W[v0:v0 + CH].float().cpu().numpy().astype(np.float64)
         qc, sc = e4m3.quantize_mx(Wc)
         assert np.array_equal(qW_gpu[v0:v0 + CH], qc), v0
         n = Wc.shape[0]
-        packed = e4m3.pack_mx_scales(sc, row_pad=128)
-        assert np.array_equal(sW_gpu[v0 // 128:v0 // 128 + packed.shape[0]], packed), v0
+        packed = e4m3.pack_mx_scales(sc)
+        assert np.array_equal(sW_gpu[v0 // 256:v0 // 256 + packed.shape[0]], packed), v0
         z[:, v0:v0 + n] = Hq @ e4m3.dequantize_mx(qc, sc).T
     tok = batch.tokens.cpu().numpy()[rows]
     msk = batch.mask.cpu().numpy()[rows]

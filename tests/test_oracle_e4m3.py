@@ -272,11 +272,12 @@ def test_mx_error_bound():
 
 
 def test_mx_scale_packing_positions():
-    """Byte (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4 of chunk (r // 128, kb // 4); padding rows hold 127."""
-    R, NB = 200, 8
+    """Chunk (r // 128, kb // 4) at [r // 256, kb // 4, (r % 256) // 128], byte (r % 32) * 16 + ((r % 128) // 32) * 4
+    + kb % 4 inside it; padding rows hold 127."""
+    R, NB = 300, 8
     sc = (np.arange(R)[:, None] * 7 + np.arange(NB)[None, :] * 3) % 250
     p = e4m3.pack_mx_scales(sc.astype(np.uint8))
-    assert p.shape == (2, 2, 512)
-    for r, kb in [(0, 0), (31, 3), (32, 0), (127, 7), (128, 4), (199, 5)]:
-        assert p[r // 128, kb // 4, (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4] == sc[r, kb]
-    assert p[1, 0, (210 % 32) * 16 + ((210 % 128) // 32) * 4] == 127
+    assert p.shape == (2, 2, 2, 512)
+    for r, kb in [(0, 0), (31, 3), (32, 0), (127, 7), (128, 4), (199, 5), (256, 1), (299, 6)]:
+        assert p[r // 256, kb // 4, (r % 256) // 128, (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4] == sc[r, kb]
+    assert p[1, 0, 0, (310 % 32) * 16 + ((310 % 128) // 32) * 4] == 127
