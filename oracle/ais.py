@@ -40,6 +40,7 @@ class Params:
     clip_eps: float = 0.2
     alpha_override: float | None = None
     adv_std_norm: bool = False
+    seq_level: bool = False          # importance weight per sequence (Eq. is-weight) instead of per token
 
 
 # --------------------------------------------------------------------------- log-probs
@@ -107,6 +108,22 @@ def ratios(lp_train, lp_roll, mask, C: float):
     return delta, rho, wbar
 
 
+def ratios_sequence(lp_train, lp_roll, mask, seq_offsets, C: float):
+    """Sequence-level importance weight of Eq. is-weight, w(x) = prod_t rho_t over the valid positions of a
+    sequence, truncated as in Eq. ais-components, w_bar(x) = min(w(x), C), and handed to every position of the
+    sequence.  Returns (log w per sequence, w_bar per row); invalid rows get 1.  The paper states this form and
+    then argues for per-token truncation; it is offered as a variant."""
+    valid = np.asarray(mask).astype(bool)
+    delta = np.where(valid, np.asarray(lp_train, np.float64) - np.asarray(lp_roll, np.float64), 0.0)
+    off = np.asarray(seq_offsets, dtype=np.int64)
+    logw = np.array([delta[off[s]:off[s + 1]].sum() for s in range(len(off) - 1)])
+    wbar_seq = np.exp(np.minimum(logw, math.log(C)))
+    wbar = np.ones(len(delta))
+    for s in range(len(off) - 1):
+        wbar[off[s]:off[s + 1]] = wbar_seq[s]
+    return logw, np.where(valid, wbar, 1.0)
+
+
 # --------------------------------------------------------------------------- advantages
 def advantages(rewards, G: int, adv_std_norm: bool = False, eps: float = 1e-6) -> np.ndarray:
     """A_i = r_i - mean_j r_j over the G responses of one prompt (Eq. grpo_adv, unnormalised form).
@@ -135,7 +152,7 @@ def valid_counts(mask, seq_offsets) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- diagnostics
-def diagnostics(lp_train, lp_roll, mask, adv_tok, p: Params) -> dict:
+def diagnostics(lp_train, lp_roll, mask, adv_tok, p: Params, wbar_rows=None) -> dict:
     """The three signals and the mixing coefficient over the valid token set
     (Eqs. alpha-ess, discrepancy, alpha-mis, variance-amplification ratio, alpha-var, alpha-final).
 
@@ -153,6 +170,8 @@ def diagnostics(lp_train, lp_roll, mask, adv_tok, p: Params) -> dict:
             out["alpha"] = float(p.alpha_override)
         return out
     delta, _, wbar = ratios(lp_train, lp_roll, mask, p.C)
+    if wbar_rows is not None:             # sequence-level variant: every valid row carries its sequence's weight
+        wbar = np.asarray(wbar_rows, np.float64)
     d = delta[valid]
     w = wbar[valid]
     A = np.asarray(adv_tok, dtype=np.float64)[valid]
@@ -287,7 +306,9 @@ def full_path(H, W, tokens, mask, seq_offsets, rewards, P: int, G: int, block: i
     sid = seq_ids(seq_offsets, T)
     adv_tok = adv[sid]
     delta, rho, wbar = ratios(lp_t, lp_r, mask, p.C)
-    diag = diagnostics(lp_t, lp_r, mask, adv_tok, p)
+    if p.seq_level:
+        _, wbar = ratios_sequence(lp_t, lp_r, mask, seq_offsets, p.C)
+    diag = diagnostics(lp_t, lp_r, mask, adv_tok, p, wbar_rows=wbar if p.seq_level else None)
     w_tilde = rectify(wbar, diag["alpha"], mask)
     old = lp_t if lp_old is None else lp_old
     loss, c = loss_and_coeff(lp_t, old, mask, seq_offsets, adv, w_tilde, P, G, p.clip_eps, lp_ref=lp_ref, beta_kl=beta_kl)

@@ -470,3 +470,39 @@ def test_microscaling_rollout_equals_trainer_when_lossless():
     lp_r2, _, _ = ais.logprob_rollout(H2, W, tok, mask, ais.MX32)
     dlt = np.abs(lp_t2 - lp_r2)
     assert 0 < dlt.max() < 0.5
+
+
+def test_sequence_level_weight_is_the_product_of_token_ratios():
+    """Eq. is-weight with hand numbers: rho = (2, 1/2, 3) gives w = 3; truncation at C; a masked position drops out;
+    sequences of one token reproduce the token-level weights; equal policies give weight 1."""
+    lp_r = np.zeros(7)
+    lp_t = np.log(np.array([2.0, 0.5, 3.0, 7.0, 1.0, 4.0, 4.0]))
+    mask = np.array([1, 1, 1, 0, 1, 1, 1], np.uint8)
+    offs = np.array([0, 4, 5, 7])
+    logw, wbar = ais.ratios_sequence(lp_t, lp_r, mask, offs, C=5.0)
+    assert np.allclose(np.exp(logw), [3.0, 1.0, 16.0])
+    assert np.allclose(wbar, [3, 3, 3, 1, 1, 5, 5])                     # row 3 is masked; 16 is truncated to C
+    _, wbar2 = ais.ratios_sequence(lp_t, lp_r, mask, offs, C=2.0)
+    assert np.allclose(wbar2, [2, 2, 2, 1, 1, 2, 2])
+    one = np.arange(8)
+    _, _, tok = ais.ratios(lp_t, lp_r, np.ones(7, np.uint8), 5.0)
+    _, seq = ais.ratios_sequence(lp_t, lp_r, np.ones(7, np.uint8), one, 5.0)
+    assert np.allclose(tok, seq)
+    _, same = ais.ratios_sequence(lp_t, lp_t, mask, offs, 5.0)
+    assert np.all(same == 1.0)
+
+
+def test_sequence_level_path_constant_drift():
+    """Delta = delta on every token of sequences of length L: w_bar = min(e^{L delta}, C) on every row, so the
+    weights are constant within the batch only if all lengths agree: CV = 0, alpha_ess = 1."""
+    T, L = 24, 6
+    offs = np.arange(0, T + 1, L)
+    lp_r = -np.ones(T)
+    lp_t = lp_r + 0.1
+    mask = np.ones(T, np.uint8)
+    _, wbar = ais.ratios_sequence(lp_t, lp_r, mask, offs, 5.0)
+    assert np.allclose(wbar, math.exp(0.6))
+    adv_tok = np.repeat([0.5, -0.5, 0.5, -0.5], L)
+    d = ais.diagnostics(lp_t, lp_r, mask, adv_tok, ais.Params(seq_level=True), wbar_rows=wbar)
+    assert abs(d["cv2"]) < 1e-20 and abs(d["alpha_ess"] - 1) < 1e-12 and abs(d["d_bar"] - 0.1) < 1e-12
+    assert abs(d["delta_sigma"] - math.exp(0.6) * 0.5 / (0.5 + 1e-6)) < 1e-9
