@@ -93,6 +93,9 @@ typedef struct ais_params {
                              (max, sum-exp, target logit) triples are merged afterwards.     */
     float beta_kl;        /* weight of the KL(pi_theta || pi_ref) term of the objective (0: no term;
                              the paper gives no value).  Used only when ais_loss_bwd gets lp_ref.  */
+    int32_t seq_level_weights; /* 0: per-token truncated ratios min(rho_t, C) (Algorithm 1).  1: every valid row of a
+                             sequence carries the sequence's weight min(prod_t rho_t, C) of Eq. is-weight /
+                             Eq. ais-components instead; d_bar and rho stay per token.                  */
 } ais_params;
 
 /* Everything the reductions produce; lives in DEVICE memory, the caller copies it back. */
@@ -224,10 +227,13 @@ int ais_diag_moments(const ais_shape* shape, const ais_params* params,
                      const float* lp_train, const float* lp_roll, const uint8_t* mask,
                      const int32_t* seq_offsets, const float* rewards,
                      float* adv, int32_t* n_valid_seq, double* moments,
+                     float* seq_logw /* [S], written when params->seq_level_weights; else may be NULL */,
                      void* workspace, size_t workspace_bytes, void* stream);
 int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const double* moments,
                       const float* lp_train, const float* lp_roll, const uint8_t* mask,
-                      float* rho, float* w_tilde, ais_diag* diag, void* stream);
+                      float* rho, float* w_tilde, ais_diag* diag,
+                      const int32_t* seq_offsets, const float* seq_logw /* both read only with seq_level_weights */,
+                      void* stream);
 
 /*
  * AIS-GRPO loss and its gradient with respect to H (Eq. ais-grpo; the objective is maximised, so

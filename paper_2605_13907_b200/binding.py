@@ -28,7 +28,8 @@ class Shape(C.Structure):
 class Params(C.Structure):
     _fields_ = [("C", C.c_float), ("delta", C.c_float), ("gamma", C.c_float), ("eps", C.c_float),
                 ("beta_var", C.c_float), ("clip_eps", C.c_float), ("alpha_override", C.c_float),
-                ("adv_std_norm", C.c_int32), ("vocab_chunk", C.c_int32), ("beta_kl", C.c_float)]
+                ("adv_std_norm", C.c_int32), ("vocab_chunk", C.c_int32), ("beta_kl", C.c_float),
+                ("seq_level_weights", C.c_int32)]
 
 
 class Diag(C.Structure):
@@ -78,9 +79,9 @@ def lib() -> C.CDLL:
         L.ais_loss_bwd.restype = C.c_int
         L.ais_loss_bwd.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 15 + [i64, C.c_int] + [vp, vp, sz, vp]
         L.ais_diag_moments.restype = C.c_int
-        L.ais_diag_moments.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 8 + [vp, sz, vp]
+        L.ais_diag_moments.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 9 + [vp, sz, vp]
         L.ais_diag_finalize.restype = C.c_int
-        L.ais_diag_finalize.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 8
+        L.ais_diag_finalize.argtypes = [C.POINTER(Shape), C.POINTER(Params)] + [vp] * 10
         L.ais_compact_index.restype = C.c_int
         L.ais_compact_index.argtypes = [vp, vp, C.c_int32, vp, vp, vp, vp]
         L.ais_gather_rows.restype = C.c_int
@@ -192,17 +193,20 @@ def diagnostics(shape: Shape, params: Params, lp_train, lp_roll, mask, seq_offse
            "ais_diagnostics")
 
 
-def diag_moments(shape: Shape, params: Params, lp_train, lp_roll, mask, seq_offsets, rewards, adv, n_valid_seq, moments, workspace):
-    _require_cuda(lp_train, lp_roll, mask, seq_offsets, rewards, adv, n_valid_seq, moments, workspace)
+def diag_moments(shape: Shape, params: Params, lp_train, lp_roll, mask, seq_offsets, rewards, adv, n_valid_seq, moments, workspace,
+                 seq_logw=None):
+    _require_cuda(lp_train, lp_roll, mask, seq_offsets, rewards, adv, n_valid_seq, moments, workspace, seq_logw)
     _check(lib().ais_diag_moments(C.byref(shape), C.byref(params), _ptr(lp_train), _ptr(lp_roll), _ptr(mask), _ptr(seq_offsets),
-                                  _ptr(rewards), _ptr(adv), _ptr(n_valid_seq), _ptr(moments), _ptr(workspace),
+                                  _ptr(rewards), _ptr(adv), _ptr(n_valid_seq), _ptr(moments), _ptr(seq_logw), _ptr(workspace),
                                   workspace.numel() * workspace.element_size(), _stream(workspace)), "ais_diag_moments")
 
 
-def diag_finalize(shape: Shape, params: Params, moments, lp_train, lp_roll, mask, rho, w_tilde, diag):
-    _require_cuda(moments, lp_train, lp_roll, mask, rho, w_tilde, diag)
+def diag_finalize(shape: Shape, params: Params, moments, lp_train, lp_roll, mask, rho, w_tilde, diag, seq_offsets=None,
+                  seq_logw=None):
+    _require_cuda(moments, lp_train, lp_roll, mask, rho, w_tilde, diag, seq_offsets, seq_logw)
     _check(lib().ais_diag_finalize(C.byref(shape), C.byref(params), _ptr(moments), _ptr(lp_train), _ptr(lp_roll), _ptr(mask),
-                                   _ptr(rho), _ptr(w_tilde), _ptr(diag), _stream(moments)), "ais_diag_finalize")
+                                   _ptr(rho), _ptr(w_tilde), _ptr(diag), _ptr(seq_offsets), _ptr(seq_logw), _stream(moments)),
+           "ais_diag_finalize")
 
 
 def loss_bwd(shape: Shape, params: Params, H, W, tokens, mask, seq_offsets, lse_train, lp_train, lp_old, adv, w_tilde, dH, loss,
@@ -330,6 +334,7 @@ class AisStep:
         self.diag = torch.zeros((C.sizeof(Diag) + 7) // 8, dtype=torch.float64, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.moments = torch.zeros(NUM_MOMENTS, dtype=torch.float64, device=dev)
+        self.seq_logw = torch.zeros(max(S, 1), **f32)        # sequence-level variant: log weight per sequence
         self.dH = torch.empty(max(T, 1), ldh, dtype=torch.bfloat16, device=dev)[:, :d] if want_grad else None
         self.w_quantized = False
 
@@ -353,9 +358,10 @@ class AisStep:
         # data parallel: this rank's masked sums, one all-reduce of 12 doubles, then alpha / w_tilde from the global sums
         from . import dist as _dist
         diag_moments(self.shape, self.params, self.lp_train, self.lp_roll, mask, seq_offsets, rewards, self.adv,
-                     self.n_valid_seq, self.moments, self.workspace)
+                     self.n_valid_seq, self.moments, self.workspace, seq_logw=self.seq_logw)
         _dist.allreduce_moments(self.moments, self.group)
-        diag_finalize(self.shape, self.params, self.moments, self.lp_train, self.lp_roll, mask, self.rho, self.w_tilde, self.diag)
+        diag_finalize(self.shape, self.params, self.moments, self.lp_train, self.lp_roll, mask, self.rho, self.w_tilde, self.diag,
+                      seq_offsets=seq_offsets, seq_logw=self.seq_logw)
 
     def backward(self, H, W, tokens, mask, seq_offsets, lp_old=None, lp_ref=None, dW=None, dw_accumulate: bool = False) -> None:
         loss_bwd(self.shape, self.params, H, W, tokens, mask, seq_offsets, self.lse_train, self.lp_train, lp_old, self.adv,

@@ -114,6 +114,7 @@ struct Layout {
     size_t off_diag;                              // reduction partials (doubles)
     size_t off_flags;                             // one byte per 128-row tile: anything to compute there?
     size_t off_coef, off_nseq;                    // backward: c_t, valid rows per sequence
+    size_t off_seqw;                              // sequence-level variant: log weight per sequence
     size_t off_u;                                 // backward scratch
     int64_t ldU;
     size_t fixed_bytes;                           // everything but the scratch rows
@@ -134,6 +135,7 @@ Layout make_layout(const ais_shape* s, const ais_params* p) {
     L.off_diag = off;   off += align_up(static_cast<size_t>(kDiagBlocks) * kNumMoments * sizeof(double), 256);
     L.off_coef = off;   off += align_up(static_cast<size_t>(L.t_ld) * sizeof(float), 256);
     L.off_nseq = off;   off += align_up(static_cast<size_t>(s->P) * s->G * sizeof(int32_t), 256);
+    L.off_seqw = off;   off += align_up(static_cast<size_t>(s->P) * s->G * sizeof(float), 256);
     L.off_u = off;
     L.ldU = static_cast<int64_t>(align_up(static_cast<size_t>(s->V), 64));
     L.fixed_bytes = off;
@@ -175,6 +177,7 @@ void ais_default_params(ais_params* p) {
     p->adv_std_norm = 0;
     p->vocab_chunk = 0;
     p->beta_kl = 0.0f;
+    p->seq_level_weights = 0;
 }
 
 size_t ais_workspace_min_bytes(const ais_shape* shape, const ais_params* params) {
@@ -358,7 +361,8 @@ int ais_diagnostics(const ais_shape* shape, const ais_params* params, const floa
     if (!lp_train || !lp_roll || !mask || !seq_offsets || !rewards || !adv || !w_tilde || !diag) return AIS_ERR_NULL;
     if (!aligned(diag, 8)) return AIS_ERR_ALIGN;
     const Layout L = make_layout(shape, params);
-    if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.off_coef) return AIS_ERR_WORKSPACE;
+    const bool seq_level = params->seq_level_weights != 0;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < (seq_level ? L.off_u : L.off_coef)) return AIS_ERR_WORKSPACE;
     st = device_setup(nullptr);
     if (st != AIS_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -367,19 +371,21 @@ int ais_diagnostics(const ais_shape* shape, const ais_params* params, const floa
     if (launch_advantages(rewards, S, shape->G, params->adv_std_norm, params->eps, adv, n_valid_seq, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     if (launch_diag(lp_train, lp_roll, mask, seq_offsets, adv, shape->T, S, *params, reinterpret_cast<double*>(ws + L.off_diag),
-                    n_valid_seq, rho, w_tilde, diag, s) != cudaSuccess)
+                    n_valid_seq, seq_level ? reinterpret_cast<float*>(ws + L.off_seqw) : nullptr, rho, w_tilde, diag, s) !=
+        cudaSuccess)
         return AIS_ERR_DEVICE;
     return AIS_OK;
 }
 
 int ais_diag_moments(const ais_shape* shape, const ais_params* params, const float* lp_train, const float* lp_roll,
                      const uint8_t* mask, const int32_t* seq_offsets, const float* rewards, float* adv, int32_t* n_valid_seq,
-                     double* moments, void* workspace, size_t workspace_bytes, void* stream) {
+                     double* moments, float* seq_logw, void* workspace, size_t workspace_bytes, void* stream) {
     int st = check_shape(shape);
     if (st != AIS_OK) return st;
     st = check_params(params);
     if (st != AIS_OK) return st;
     if (!lp_train || !lp_roll || !mask || !seq_offsets || !rewards || !adv || !moments) return AIS_ERR_NULL;
+    if (params->seq_level_weights != 0 && !seq_logw) return AIS_ERR_NULL;
     if (!aligned(moments, 8)) return AIS_ERR_ALIGN;
     const Layout L = make_layout(shape, params);
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.off_coef) return AIS_ERR_WORKSPACE;
@@ -391,23 +397,26 @@ int ais_diag_moments(const ais_shape* shape, const ais_params* params, const flo
     if (launch_advantages(rewards, S, shape->G, params->adv_std_norm, params->eps, adv, n_valid_seq, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     if (launch_moments(lp_train, lp_roll, mask, seq_offsets, adv, shape->T, S, *params, reinterpret_cast<double*>(ws + L.off_diag),
-                       n_valid_seq, moments, s) != cudaSuccess)
+                       n_valid_seq, params->seq_level_weights != 0 ? seq_logw : nullptr, moments, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     return AIS_OK;
 }
 
 int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const double* moments, const float* lp_train,
-                      const float* lp_roll, const uint8_t* mask, float* rho, float* w_tilde, ais_diag* diag, void* stream) {
+                      const float* lp_roll, const uint8_t* mask, float* rho, float* w_tilde, ais_diag* diag,
+                      const int32_t* seq_offsets, const float* seq_logw, void* stream) {
     int st = check_shape(shape);
     if (st != AIS_OK) return st;
     st = check_params(params);
     if (st != AIS_OK) return st;
     if (!moments || !lp_train || !lp_roll || !mask || !w_tilde || !diag) return AIS_ERR_NULL;
+    const bool seq_level = params->seq_level_weights != 0;
+    if (seq_level && (!seq_offsets || !seq_logw)) return AIS_ERR_NULL;
     if (!aligned(moments, 8) || !aligned(diag, 8)) return AIS_ERR_ALIGN;
     st = device_setup(nullptr);
     if (st != AIS_OK) return st;
-    if (launch_finalize(moments, lp_train, lp_roll, mask, shape->T, *params, rho, w_tilde, diag,
-                        static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    if (launch_finalize(moments, lp_train, lp_roll, mask, shape->T, *params, rho, w_tilde, diag, seq_offsets,
+                        shape->P * shape->G, seq_level ? seq_logw : nullptr, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return AIS_ERR_DEVICE;
     return AIS_OK;
 }

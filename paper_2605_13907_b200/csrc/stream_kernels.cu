@@ -335,6 +335,21 @@ __global__ void adv_kernel(const float* __restrict__ rewards, int S, int G, int 
     adv[s] = static_cast<float>(a);
 }
 
+// Sequence-level importance weight (Eq. is-weight): log w(x) = sum over the valid rows of a sequence of
+// lp_train - lp_roll.  One warp per sequence, double accumulation in a fixed order.
+__global__ void __launch_bounds__(256) seq_logw_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
+                                                        const uint8_t* __restrict__ mask, const int32_t* __restrict__ seq_offsets,
+                                                        int S, float* __restrict__ seq_logw) {
+    const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (s >= S) return;
+    const int lane = threadIdx.x & 31;
+    double acc = 0.0;
+    for (int64_t t = static_cast<int64_t>(seq_offsets[s]) + lane; t < seq_offsets[s + 1]; t += 32)
+        if (mask[t]) acc += static_cast<double>(lp_train[t]) - static_cast<double>(lp_roll[t]);
+    acc = warp_sum(acc);
+    if (lane == 0) seq_logw[s] = static_cast<float>(acc);
+}
+
 // One byte per 128-row tile: does any row of the tile need computing?  (mask != 0 / gradient factor != 0)
 template <typename T>
 __global__ void tile_flags_kernel(const T* __restrict__ pred, int64_t n, uint8_t* __restrict__ flags) {
@@ -393,7 +408,8 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
                                                                 const uint8_t* __restrict__ mask,
                                                                 const int32_t* __restrict__ seq_offsets,
                                                                 const float* __restrict__ adv, int64_t T, int S, float C,
-                                                                double* __restrict__ partials, int32_t* __restrict__ n_valid_seq) {
+                                                                double* __restrict__ partials, int32_t* __restrict__ n_valid_seq,
+                                                                const float* __restrict__ seq_logw) {
     __shared__ double scratch[32];
     double acc[kNumMoments];
 #pragma unroll
@@ -433,7 +449,8 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
         // rho = e^dl, truncated weight min(rho, C), and |e^lt - e^lr| = e^lr |rho - 1|
         const float dl = lt - lr;
         const float rho = __expf(dl);
-        const float w = fminf(rho, C);
+        // sequence-level variant: every row carries its sequence's truncated weight instead of its own
+        const float w = fminf(seq_logw ? __expf(seq_logw[sq]) : rho, C);
         const float Aw = A * w;
         f[0] += 1.0f;
         f[1] += w;
@@ -553,15 +570,17 @@ template <int VEC>
 __global__ void __launch_bounds__(256) rectify_kernel(const float* __restrict__ lp_train, const float* __restrict__ lp_roll,
                                                       const uint8_t* __restrict__ mask, int64_t T, float C,
                                                       const ais_diag* __restrict__ diag, float* __restrict__ rho,
-                                                      float* __restrict__ w_tilde) {
+                                                      float* __restrict__ w_tilde, const int32_t* __restrict__ seq_offsets,
+                                                      int S, const float* __restrict__ seq_logw) {
     const float alpha = static_cast<float>(diag->alpha);
-    auto one = [&](float lt, float lr, uint8_t mk, float& r, float& wt) {
+    auto one = [&](float lt, float lr, uint8_t mk, float& r, float& wt, int64_t t) {
         r = 1.0f;
         wt = 1.0f;
         if (mk) {
             const float dl = lt - lr;
             r = __expf(dl);
-            wt = fmaf(alpha, fminf(r, C) - 1.0f, 1.0f);
+            const float w = seq_logw ? __expf(seq_logw[seq_of_row(seq_offsets, S, t)]) : r;      // sequence-level variant
+            wt = fmaf(alpha, fminf(w, C) - 1.0f, 1.0f);
         }
     };
     const int64_t ngroups = T / VEC;
@@ -570,7 +589,7 @@ __global__ void __launch_bounds__(256) rectify_kernel(const float* __restrict__ 
         const RowGroup<VEC> in = load_group<VEC>(lp_train, lp_roll, mask, g);
         float r[VEC], wt[VEC];
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) one(in.lt[j], in.lr[j], in.mk[j], r[j], wt[j]);
+        for (int j = 0; j < VEC; ++j) one(in.lt[j], in.lr[j], in.mk[j], r[j], wt[j], g * VEC + j);
         if (VEC == 4) {
             if (rho) reinterpret_cast<float4*>(rho)[g] = make_float4(r[0], r[1 % VEC], r[2 % VEC], r[3 % VEC]);
             reinterpret_cast<float4*>(w_tilde)[g] = make_float4(wt[0], wt[1 % VEC], wt[2 % VEC], wt[3 % VEC]);
@@ -581,7 +600,7 @@ __global__ void __launch_bounds__(256) rectify_kernel(const float* __restrict__ 
     }
     for (int64_t t = ngroups * VEC + static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
         float r, wt;
-        one(lp_train[t], lp_roll[t], mask[t], r, wt);
+        one(lp_train[t], lp_roll[t], mask[t], r, wt, t);
         if (rho) rho[t] = r;
         w_tilde[t] = wt;
     }
@@ -686,23 +705,25 @@ inline bool vec4_ok(const void* a, const void* b, const void* c, const void* d, 
 
 void launch_moments_kernel(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
                            const float* adv, int64_t T, int S, float C, double* partials, int32_t* n_valid_seq,
-                           cudaStream_t stream) {
+                           float* seq_logw, cudaStream_t stream) {
+    if (seq_logw && S > 0) seq_logw_kernel<<<(S + 7) / 8, 256, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, S, seq_logw);
     if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask))
         moments_kernel<4><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials,
-                                                                      n_valid_seq);
+                                                                      n_valid_seq, seq_logw);
     else
         moments_kernel<1><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials,
-                                                                      n_valid_seq);
+                                                                      n_valid_seq, seq_logw);
 }
 
 void launch_rectify_kernel(const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T, float C,
-                           const ais_diag* diag, float* rho, float* w_tilde, cudaStream_t stream) {
+                           const ais_diag* diag, float* rho, float* w_tilde, const int32_t* seq_offsets, int S,
+                           const float* seq_logw, cudaStream_t stream) {
     const int64_t groups = (T + 3) / 4;
     const int blocks = static_cast<int>(((groups + 255) / 256) < 2368 ? ((groups + 255) / 256) : 2368);
     if (vec4_ok(lp_train, lp_roll, rho, w_tilde, mask))
-        rectify_kernel<4><<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde);
+        rectify_kernel<4><<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde, seq_offsets, S, seq_logw);
     else
-        rectify_kernel<1><<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde);
+        rectify_kernel<1><<<blocks, 256, 0, stream>>>(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde, seq_offsets, S, seq_logw);
 }
 
 }  // namespace
@@ -781,26 +802,27 @@ cudaError_t launch_advantages(const float* rewards, int S, int G, int adv_std_no
 
 cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
                         const float* adv, int64_t T, int S, const ais_params& p, double* partials, int32_t* n_valid_seq,
-                        float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream) {
+                        float* seq_logw, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream) {
     const float C = p.C;
-    launch_moments_kernel(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials, n_valid_seq, stream);
+    launch_moments_kernel(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials, n_valid_seq, seq_logw, stream);
     diag_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, p, diag);
-    if (T > 0) launch_rectify_kernel(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde, stream);
+    if (T > 0) launch_rectify_kernel(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde, seq_offsets, S, seq_logw, stream);
     return cudaGetLastError();
 }
 
 cudaError_t launch_moments(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
                            const float* adv, int64_t T, int S, const ais_params& p, double* partials, int32_t* n_valid_seq,
-                           double* moments, cudaStream_t stream) {
-    launch_moments_kernel(lp_train, lp_roll, mask, seq_offsets, adv, T, S, p.C, partials, n_valid_seq, stream);
+                           float* seq_logw, double* moments, cudaStream_t stream) {
+    launch_moments_kernel(lp_train, lp_roll, mask, seq_offsets, adv, T, S, p.C, partials, n_valid_seq, seq_logw, stream);
     moments_reduce_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, moments);
     return cudaGetLastError();
 }
 
 cudaError_t launch_finalize(const double* moments, const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T,
-                            const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream) {
+                            const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, const int32_t* seq_offsets, int S,
+                            const float* seq_logw, cudaStream_t stream) {
     diag_finalize_kernel<<<1, 32, 0, stream>>>(moments, 1, p, diag);
-    if (T > 0) launch_rectify_kernel(lp_train, lp_roll, mask, T, p.C, diag, rho, w_tilde, stream);
+    if (T > 0) launch_rectify_kernel(lp_train, lp_roll, mask, T, p.C, diag, rho, w_tilde, seq_offsets, S, seq_logw, stream);
     return cudaGetLastError();
 }
 

@@ -42,15 +42,17 @@ cudaError_t launch_advantages(const float* rewards, int S, int G, int adv_std_no
 // n_valid_seq (may be NULL) must have been cleared: the moments kernel adds every sequence's valid rows to it.
 cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
                         const float* adv, int64_t T, int S, const ais_params& p, double* partials /*[kDiagBlocks][kNumMoments]*/,
-                        int32_t* n_valid_seq, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
+                        int32_t* n_valid_seq, float* seq_logw /* [S] scratch: non-NULL selects sequence-level weights */,
+                        float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
 
 // The two halves of launch_diag: partial moments summed into `moments` [kNumMoments], and everything that follows
 // from a (possibly all-reduced) moment vector.
 cudaError_t launch_moments(const float* lp_train, const float* lp_roll, const uint8_t* mask, const int32_t* seq_offsets,
                            const float* adv, int64_t T, int S, const ais_params& p, double* partials, int32_t* n_valid_seq,
-                           double* moments, cudaStream_t stream);
+                           float* seq_logw, double* moments, cudaStream_t stream);
 cudaError_t launch_finalize(const double* moments, const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T,
-                            const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream);
+                            const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, const int32_t* seq_offsets, int S,
+                            const float* seq_logw, cudaStream_t stream);
 
 // coef[t] and the loss; n_valid_seq must already hold the valid counts.  S_norm is the number of sequences the
 // objective averages over (all data-parallel ranks together).

@@ -111,3 +111,43 @@ def test_batch_reductions_on_unaligned_and_ragged_vectors(T, shift):
     got_rho, got_wt = rho.cpu().numpy(), wt.cpu().numpy()
     assert np.allclose(got_rho[valid], ref_rho[valid], rtol=1e-5) and np.all(got_rho[~valid] == 1)
     assert np.allclose(got_wt[valid], ref_wt[valid], rtol=1e-4, atol=1e-5) and np.all(got_wt[~valid] == 1)
+
+
+def test_sequence_level_weights_on_gpu():
+    """params.seq_level_weights: every valid row carries min(prod_t rho_t, C) of its sequence (Eq. is-weight).  The
+    fused call and the split pair agree with the oracle's sequence-level variant; d_bar and rho stay per token."""
+    import paper_2605_13907_b200 as ais
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], d=256, V=1280, P=3, G=4, lengths="uniform:3:70", seed=77)
+    b = workloads.make_batch(w, device="cpu")
+    a = workloads.to_numpy(b)
+    ref = oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, w.block,
+                         params=oais.Params(seq_level=True))
+    tok = oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, w.block,
+                         want_grad=False)
+    assert abs(ref["diag"]["cv2"] - tok["diag"]["cv2"]) > 1e-4          # the two variants really differ on this batch
+    params = ais.default_params(seq_level_weights=1)
+    step = ais.AisStep(b.T, w.d, w.V, w.P, w.G, w.block, params=params)
+    offs, rew = b.seq_offsets.cuda(), b.rewards.cuda()
+    H, W, tokens, mask = b.H.cuda(), b.W.cuda(), b.tokens.cuda(), b.mask.cuda()
+    step.step(H, W, tokens, mask, offs, rew)
+    torch.cuda.synchronize()
+    d = step.read_diag()
+    T = b.T
+    for k in ("alpha", "alpha_ess", "alpha_var", "cv2", "d_bar", "delta_sigma"):
+        assert abs(d[k] - ref["diag"][k]) <= 1e-3 * max(1.0, abs(ref["diag"][k])), (k, d[k], ref["diag"][k])
+    assert np.max(np.abs(step.w_tilde.cpu().numpy()[:T] - ref["w_tilde"])) <= 2e-2 * np.max(ref["w_tilde"])
+    assert np.max(np.abs(step.rho.cpu().numpy()[:T] - ref["rho"]) / ref["rho"]) <= 2e-2
+    dH = step.dH.float().cpu().numpy()[:T].astype(np.float64)
+    assert np.linalg.norm(dH - ref["dH"]) <= 1e-2 * np.linalg.norm(ref["dH"])
+    fused = (d, step.w_tilde.clone())
+    # the split pair gives the same bits
+    step.w_tilde.zero_(); step.diag.zero_()
+    ais.diag_moments(step.shape, step.params, step.lp_train, step.lp_roll, mask, offs, rew, step.adv, step.n_valid_seq,
+                     step.moments, step.workspace, seq_logw=step.seq_logw)
+    ais.diag_finalize(step.shape, step.params, step.moments, step.lp_train, step.lp_roll, mask, step.rho, step.w_tilde, step.diag,
+                      seq_offsets=offs, seq_logw=step.seq_logw)
+    torch.cuda.synchronize()
+    d2 = step.read_diag()
+    for k in ("alpha", "cv2", "d_bar", "delta_sigma", "n_valid"):
+        assert d2[k] == fused[0][k], k
+    assert torch.equal(step.w_tilde, fused[1])
