@@ -69,6 +69,7 @@ def logprob_train(H, W, tokens, mask):
 
 
 MX32 = -32        # `block` value selecting microscaling FP8 (E8M0 scale per 32 elements)
+MXFP4 = -4        # `block` value selecting microscaling FP4 (E2M1 elements, E8M0 scale per 32 elements)
 
 
 def logprob_rollout(H, W, tokens, mask, block: int):
@@ -77,7 +78,12 @@ def logprob_rollout(H, W, tokens, mask, block: int):
     then the same log-softmax.  block = 0 selects one scale per tensor (Appendix 'FP8 rollout': per-tensor
     dynamic scaling); block = MX32 selects power-of-two scales per 32 elements (the microscaling format named as
     future work in the paper's limitations).  Returns (lp, lse, (qH, sH, qW, sW))."""
-    if block == MX32:
+    if block == MXFP4:
+        qH, sH = e4m3.quantize_mxfp4(H)
+        qW, sW = e4m3.quantize_mxfp4(W)
+        Hq = e4m3.dequantize_mxfp4(qH, sH)
+        Wq = e4m3.dequantize_mxfp4(qW, sW)
+    elif block == MX32:
         qH, sH = e4m3.quantize_mx(H)
         qW, sW = e4m3.quantize_mx(W)
         Hq = e4m3.dequantize_mx(qH, sH)

@@ -208,3 +208,63 @@ def pack_mx_scales(scale_codes, row_pad: int = 256) -> np.ndarray:
     full[:R] = sc
     v = full.reshape(Rp // 256, 2, 4, 32, NB // 4, 4)       # [group, half, r1, r0, chunk col, kb]
     return np.ascontiguousarray(v.transpose(0, 4, 1, 3, 2, 5)).reshape(Rp // 256, NB // 4, 2, 512)
+
+
+# --------------------------------------------------------------------------- microscaling FP4 (E2M1 elements)
+_E2M1_VALUES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+_FP4_EMAX = 2             # 6 = 1.5 * 2^2
+
+
+def encode_e2m1(x) -> np.ndarray:
+    """Value -> 4-bit E2M1 code (1 sign, 2 exponent, 1 mantissa bit; magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6; no
+    infinities or NaNs), round to nearest with ties to the code whose mantissa bit is 0, saturating at +-6.  The
+    sign bit is copied from the input.  Written as a nearest-value search: the grid has eight magnitudes."""
+    v = np.asarray(x, dtype=np.float64)
+    if not np.all(np.isfinite(v)):
+        raise ValueError("E2M1 has no encoding for infinities or NaNs")
+    mag = np.minimum(np.abs(v), 6.0)
+    d = np.abs(mag[..., None] - _E2M1_VALUES)
+    lo = np.argmin(d, axis=-1)                               # first (smaller) of two equally near codes
+    nxt = np.minimum(lo + 1, 7)
+    tie = (nxt != lo) & (np.take_along_axis(d, nxt[..., None], axis=-1)[..., 0] == np.take_along_axis(d, lo[..., None], axis=-1)[..., 0])
+    code = np.where(tie & (lo % 2 == 1), lo + 1, lo)         # on a tie take the even code
+    return (code | (np.signbit(v).astype(np.int64) << 3)).astype(np.uint8)
+
+
+def decode_e2m1(codes) -> np.ndarray:
+    c = np.asarray(codes, dtype=np.uint8)
+    return np.where(c & 8, -1.0, 1.0) * _E2M1_VALUES[c & 7]
+
+
+def quantize_mxfp4(x):
+    """Microscaling FP4: blocks of 32 elements share 2^X, X = floor(log2 amax) - 2, stored as X + 127 (clamped to
+    0..254; 127 for a zero block); elements are x / 2^X on the E2M1 grid (scaled magnitudes in (6, 8) saturate to 6).
+    Same published rule as quantize_mx with the FP4 element format -- the FP4 rollouts the paper names as future work.
+
+    Returns (codes uint8 [R, K], one 4-bit code per entry, and scale codes uint8 [R, K // 32])."""
+    x64 = np.asarray(x, dtype=np.float64)
+    R, K = x64.shape
+    if K % MX_BLOCK:
+        raise ValueError("the last dimension must be a multiple of 32")
+    xb = x64.reshape(R, K // MX_BLOCK, MX_BLOCK)
+    amax = np.max(np.abs(xb), axis=2)
+    _, e = np.frexp(amax)
+    X = np.where(amax > 0, e - 1 - _FP4_EMAX, 0)
+    sc = np.clip(X + 127, 0, 254).astype(np.int64)
+    sc = np.where(amax > 0, sc, 127)
+    scaled = np.ldexp(xb, -(sc[:, :, None] - 127))
+    codes = encode_e2m1(np.clip(scaled, -1e30, 1e30)).reshape(R, K)
+    return codes, sc.astype(np.uint8)
+
+
+def dequantize_mxfp4(codes, scale_codes) -> np.ndarray:
+    codes = np.asarray(codes, dtype=np.uint8)
+    R, K = codes.shape
+    vals = decode_e2m1(codes).reshape(R, K // MX_BLOCK, MX_BLOCK)
+    return np.ldexp(vals, np.asarray(scale_codes, dtype=np.int64)[:, :, None] - 127).reshape(R, K)
+
+
+def pack_fp4_pairs(codes) -> np.ndarray:
+    """Two 4-bit codes per byte, the element with the lower index in the low nibble."""
+    c = np.asarray(codes, dtype=np.uint8)
+    return (c[..., 0::2] | (c[..., 1::2] << 4)).astype(np.uint8)

@@ -281,3 +281,50 @@ def test_mx_scale_packing_positions():
     for r, kb in [(0, 0), (31, 3), (32, 0), (127, 7), (128, 4), (199, 5), (256, 1), (299, 6)]:
         assert p[r // 256, kb // 4, (r % 256) // 128, (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4] == sc[r, kb]
     assert p[1, 0, 0, (310 % 32) * 16 + ((310 % 128) // 32) * 4] == 127
+
+
+# --------------------------------------------------------------------------- microscaling FP4 (E2M1)
+def test_e2m1_grid_ties_saturation_and_black_box():
+    """The eight magnitudes; every midpoint goes to the code with mantissa bit 0; beyond 6 saturates; the sign is
+    copied (also for zero); a third-party 4-bit float type agrees on random in-range values."""
+    assert np.array_equal(e4m3.decode_e2m1(np.arange(8, dtype=np.uint8)), [0, 0.5, 1, 1.5, 2, 3, 4, 6])
+    grid = [0, 0.5, 1, 1.5, 2, 3, 4, 6]
+    mids = {0.25: 0.0, 0.75: 1.0, 1.25: 1.0, 1.75: 2.0, 2.5: 2.0, 3.5: 4.0, 5.0: 4.0}       # midpoint -> even neighbour
+    for i, (m, want) in enumerate(mids.items()):
+        assert e4m3.decode_e2m1(e4m3.encode_e2m1(np.array([m])))[0] == want
+        assert e4m3.decode_e2m1(e4m3.encode_e2m1(np.array([np.nextafter(m, 10)])))[0] == grid[i + 1]
+        assert e4m3.decode_e2m1(e4m3.encode_e2m1(np.array([np.nextafter(m, -10)])))[0] == grid[i]
+        assert e4m3.decode_e2m1(e4m3.encode_e2m1(np.array([-m])))[0] == -want
+    assert e4m3.decode_e2m1(e4m3.encode_e2m1(np.array([6.5, 1e9, -7.0]))).tolist() == [6, 6, -6]
+    assert e4m3.encode_e2m1(np.array([-0.0, -0.1]))[0] == 8 and e4m3.encode_e2m1(np.array([-0.0, -0.1]))[1] == 8
+    for c in range(16):
+        assert e4m3.encode_e2m1(e4m3.decode_e2m1(np.array([c], np.uint8)))[0] == c
+    ml_dtypes = pytest.importorskip("ml_dtypes")
+    if not hasattr(ml_dtypes, "float4_e2m1fn"):
+        pytest.skip("this ml_dtypes has no 4-bit float")
+    r = np.clip(np.random.default_rng(3).normal(size=200000) * 3, -6, 6).astype(np.float32)
+    ref = r.astype(ml_dtypes.float4_e2m1fn).astype(np.float64)
+    assert np.array_equal(e4m3.decode_e2m1(e4m3.encode_e2m1(r)), ref)
+
+
+def test_mxfp4_shared_exponent_and_round_trip():
+    """X = floor(log2 amax) - 2: hand cases; values on the scaled grid round-trip; the (6, 8) band saturates."""
+    def one(amax):
+        x = np.zeros((1, 32))
+        x[0, 3] = amax
+        c, s = e4m3.quantize_mxfp4(x)
+        return int(s[0, 0]), float(e4m3.dequantize_mxfp4(c, s)[0, 3])
+    assert one(6.0) == (127, 6.0)
+    assert one(4.0) == (127, 4.0)
+    assert one(1.0) == (125, 1.0)
+    assert one(7.0) == (127, 6.0)                  # floor(log2 7) = 2: 7 is in the clipping band
+    assert one(3.0) == (126, 3.0)
+    assert one(0.0) == (127, 0.0)
+    rng = np.random.default_rng(4)
+    codes = rng.integers(0, 16, size=(6, 96)).astype(np.uint8)
+    codes[:, ::32] = 7                                      # every block holds the largest magnitude
+    k = rng.integers(-10, 10, size=(6, 3))
+    x = np.ldexp(e4m3.decode_e2m1(codes).reshape(6, 3, 32), k[:, :, None]).reshape(6, 96)
+    c, s = e4m3.quantize_mxfp4(x)
+    assert np.array_equal(s.astype(np.int64), k + 127) and np.array_equal(e4m3.dequantize_mxfp4(c, s), x)
+    assert np.array_equal(e4m3.pack_fp4_pairs(np.array([[1, 2, 15, 0]], np.uint8)), [[0x21, 0x0F]])
