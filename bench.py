@@ -148,6 +148,8 @@ def run_ours(args) -> None:
         w = workloads.scaled(w, block=0)                              # variant: one FP8 scale per tensor
     if args.fp8_mx:
         w = workloads.scaled(w, block=ais.FP8_MX32)                   # variant: microscaling, E8M0 scale per 32 elements
+    if args.fp4_mx:
+        w = workloads.scaled(w, block=ais.FP4_MX32)                   # variant: microscaling FP4 (E2M1) rollout pass
     batch = workloads.make_batch(w, device=dev)
     if args.compact:
         # scattered masks: pack the valid rows once per batch (inside the step for the end-to-end figure) and run on those
@@ -304,7 +306,7 @@ def run_ours(args) -> None:
                          "peak_source": peaks["source"] + " bf16 sustained (kernel timed inside a long step)",
                          "passes": {"fwd_roll_fp8_tflops": flops_pass / (seg["fwd_roll_fp8"] * 1e-3) / 1e12,
                                     "bwd_two_passes_tflops": (3 if args.with_dw else 2) * flops_pass / (seg["loss_bwd"] * 1e-3) / 1e12,
-                                    "quantize_gbs": (T + w.V) * w.d * (3.0 + 4.0 / w.block if w.block > 0 else 3.03 if w.block < 0 else 5.0) / (seg["quantize"] * 1e-3) / 1e9}},
+                                    "quantize_gbs": (T + w.V) * w.d * (3.0 + 4.0 / w.block if w.block > 0 else 2.53 if w.block == -4 else 3.03 if w.block < 0 else 5.0) / (seg["quantize"] * 1e-3) / 1e9}},
             "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches * args.steps,
             "clocks": clocks,
@@ -411,6 +413,8 @@ def main() -> None:
     ap.add_argument("--compact", action="store_true",
                     help="pack the valid rows first (for workloads with scattered masks, e.g. llada_8b)")
     ap.add_argument("--with-dw", action="store_true", help="variant: ais_loss_bwd also writes dW (a fifth tensor-core pass)")
+    ap.add_argument("--fp4-mx", action="store_true",
+                    help="variant (not the headline workload): microscaling FP4 rollout pass (E2M1, scale per 32 elements)")
     ap.add_argument("--fp8-mx", action="store_true",
                     help="variant (not the headline workload): microscaling FP8, power-of-two scale per 32 elements")
     ap.add_argument("--fp8-per-tensor", action="store_true",

@@ -59,6 +59,7 @@ extern "C" {
 #define AIS_FLAG_TIMEOUT      8u   /* a bounded device-side wait ran out; outputs undefined */
 
 #define AIS_FP8_MX32 (-32)        /* ais_shape.fp8_block: microscaling FP8, E8M0 scale per 32 elements */
+#define AIS_FP4_MX32 (-4)         /* ais_shape.fp8_block: microscaling FP4 (E2M1 elements), E8M0 scale per 32    */
 
 typedef struct ais_shape {
     int64_t T;            /* token rows                                                      */
@@ -68,7 +69,8 @@ typedef struct ais_shape {
     int32_t G;            /* responses per prompt; sequence s belongs to prompt s / G        */
     int32_t fp8_block;    /* elements along d sharing one FP8 scale: 32, 64 or 128;
                              0 = one scale per tensor (ais_quantize_fp8_tensor);
-                             AIS_FP8_MX32 = power-of-two scale per 32 (ais_quantize_mxfp8)   */
+                             AIS_FP8_MX32 = power-of-two scale per 32 (ais_quantize_mxfp8);
+                             AIS_FP4_MX32 = the same with 4-bit elements (ais_quantize_mxfp4)*/
     int32_t P_total;      /* prompts over all data-parallel ranks (loss normaliser); 0 = P    */
     int64_t ldh;          /* row stride of H (and of its codes) in elements                  */
     int64_t ldw;          /* row stride of W (and of its codes) in elements                  */
@@ -175,6 +177,17 @@ int ais_quantize_fp8_tensor(const void* x, int64_t rows, int64_t cols, int64_t l
  */
 size_t ais_mx_scale_bytes(int64_t rows, int64_t cols);
 int ais_quantize_mxfp8(const void* x, int64_t rows, int64_t cols, int64_t ld,
+                       uint8_t* codes, int64_t ldq, uint8_t* scales, void* stream);
+
+/*
+ * Microscaling FP4, the FP4 rollouts the paper names as future work (Introduction, Limitations): the same rule with
+ * E2M1 elements (magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6; X = floor(log2 max|x|) - 2; scaled magnitudes in (6, 8)
+ * saturate).  codes [rows, ldq] bytes hold two 4-bit codes each, the element with the lower index in the low nibble
+ * (ldq >= cols / 2, a multiple of 4); scales as for ais_quantize_mxfp8.  With shape->fp8_block == AIS_FP4_MX32
+ * (d a multiple of 256, ldh and ldw multiples of 32; the codes' row strides are ldh / 2 and ldw / 2 bytes)
+ * ais_logprob_fwd runs the rollout pass on tcgen05's packed-FP4 block-scaled MMA.
+ */
+int ais_quantize_mxfp4(const void* x, int64_t rows, int64_t cols, int64_t ld,
                        uint8_t* codes, int64_t ldq, uint8_t* scales, void* stream);
 
 /*

@@ -71,6 +71,8 @@ def lib() -> C.CDLL:
         L.ais_mx_scale_bytes.argtypes = [i64, i64]
         L.ais_quantize_mxfp8.restype = C.c_int
         L.ais_quantize_mxfp8.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp]
+        L.ais_quantize_mxfp4.restype = C.c_int
+        L.ais_quantize_mxfp4.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp]
         L.ais_logprob_fwd.restype = C.c_int
         L.ais_logprob_fwd.argtypes = [C.POINTER(Shape), C.POINTER(Params), vp, vp, vp, vp, i64, vp, vp, i64, vp, vp,
                                       vp, vp, vp, vp, vp, vp, sz, vp]
@@ -141,6 +143,7 @@ def _require_cuda(*tensors):
 
 
 FP8_MX32 = -32          # fp8_block value: microscaling FP8 (E8M0 scale per 32 elements, hardware block-scaled MMA)
+FP4_MX32 = -4           # fp8_block value: microscaling FP4 (E2M1 elements, two per byte)
 
 
 def mx_scale_bytes(rows: int, cols: int) -> int:
@@ -152,6 +155,14 @@ def quantize_fp8(x: torch.Tensor, block: int, codes: torch.Tensor | None = None,
     block = 0: one scale per tensor; block = FP8_MX32: packed E8M0 scale bytes (see include/ais.h)."""
     _require_cuda(x, codes, scales)
     rows, cols = x.shape
+    if block == FP4_MX32:                            # 4-bit elements, two per byte, packed scale bytes
+        if codes is None:
+            codes = torch.empty(rows, cols // 2, dtype=torch.uint8, device=x.device)
+        if scales is None:
+            scales = torch.empty(mx_scale_bytes(rows, cols), dtype=torch.uint8, device=x.device)
+        _check(lib().ais_quantize_mxfp4(_ptr(x), rows, cols, x.stride(0), _ptr(codes), codes.stride(0), _ptr(scales),
+                                        _stream(x)), "ais_quantize_mxfp4")
+        return codes, scales
     if codes is None:
         codes = torch.empty(rows, cols, dtype=torch.uint8, device=x.device)
     if block == FP8_MX32:                            # power-of-two scale per 32 elements, packed scale bytes
@@ -313,9 +324,13 @@ class AisStep:
             ws_all = ws_min + max(0, (T + 127) // 128 * 128 - 128) * ld_u * 2
             ws = max(ws_min, min(ws_all, workspace_bytes_cap))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
-        self.qH = torch.empty(max(T, 1), ldh, dtype=torch.uint8, device=dev)[:, :d]
-        self.qW = torch.empty(V, ldw, dtype=torch.uint8, device=dev)[:, :d]
-        if fp8_block == FP8_MX32:
+        if fp8_block == FP4_MX32:
+            self.qH = torch.empty(max(T, 1), ldh // 2, dtype=torch.uint8, device=dev)[:, :d // 2]
+            self.qW = torch.empty(V, ldw // 2, dtype=torch.uint8, device=dev)[:, :d // 2]
+        else:
+            self.qH = torch.empty(max(T, 1), ldh, dtype=torch.uint8, device=dev)[:, :d]
+            self.qW = torch.empty(V, ldw, dtype=torch.uint8, device=dev)[:, :d]
+        if fp8_block in (FP8_MX32, FP4_MX32):
             self.sH = torch.empty(mx_scale_bytes(T, d), dtype=torch.uint8, device=dev)
             self.sW = torch.empty(mx_scale_bytes(V, d), dtype=torch.uint8, device=dev)
         else:

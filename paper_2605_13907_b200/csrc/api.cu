@@ -77,8 +77,10 @@ int check_shape(const ais_shape* s) {
     if (s->T < 0 || s->T > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
     if (s->d <= 0 || s->V <= 0 || s->P <= 0 || s->G <= 0) return AIS_ERR_SHAPE;
     if (s->d % 128 != 0 || s->V % 8 != 0) return AIS_ERR_SHAPE;
-    if (s->fp8_block != 0 && s->fp8_block != 32 && s->fp8_block != 64 && s->fp8_block != 128 && s->fp8_block != AIS_FP8_MX32)
+    if (s->fp8_block != 0 && s->fp8_block != 32 && s->fp8_block != 64 && s->fp8_block != 128 && s->fp8_block != AIS_FP8_MX32 &&
+        s->fp8_block != AIS_FP4_MX32)
         return AIS_ERR_SHAPE;
+    if (s->fp8_block == AIS_FP4_MX32 && (s->d % 256 != 0 || s->ldh % 32 != 0 || s->ldw % 32 != 0)) return AIS_ERR_SHAPE;
     if (s->fp8_block > 0 && s->d % s->fp8_block != 0) return AIS_ERR_SHAPE;
     if (s->ldh < s->d || s->ldw < s->d) return AIS_ERR_SHAPE;
     if (s->ldh % 16 != 0 || s->ldw % 16 != 0) return AIS_ERR_ALIGN;
@@ -235,7 +237,21 @@ int ais_quantize_mxfp8(const void* x, int64_t rows, int64_t cols, int64_t ld, ui
     if (rows > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
     int st = device_setup(nullptr);
     if (st != AIS_OK) return st;
-    return launch_quantize_mx(x, rows, cols, ld, codes, ldq, scales, ais_mx_scale_bytes(rows, cols),
+    return launch_quantize_mx(x, rows, cols, ld, codes, ldq, scales, ais_mx_scale_bytes(rows, cols), false,
+                              static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? AIS_OK
+               : AIS_ERR_DEVICE;
+}
+
+int ais_quantize_mxfp4(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq, uint8_t* scales,
+                       void* stream) {
+    if (!x || !codes || !scales) return AIS_ERR_NULL;
+    if (rows < 0 || cols <= 0 || cols % 128 != 0 || ld < cols || ldq < cols / 2) return AIS_ERR_SHAPE;
+    if (ld % 8 != 0 || ldq % 4 != 0 || !aligned(x, 16) || !aligned(codes, 4) || !aligned(scales, 16)) return AIS_ERR_ALIGN;
+    if (rows > (int64_t(1) << 31) - 1024) return AIS_ERR_SHAPE;
+    int st = device_setup(nullptr);
+    if (st != AIS_OK) return st;
+    return launch_quantize_mx(x, rows, cols, ld, codes, ldq, scales, ais_mx_scale_bytes(rows, cols), true,
                               static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? AIS_OK
                : AIS_ERR_DEVICE;
@@ -257,7 +273,8 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     if (do_roll && (!qH || !sH || !qW || !sW)) return AIS_ERR_NULL;
     if (do_train && (!aligned(H, 16) || !aligned(W, 16))) return AIS_ERR_ALIGN;
     const bool per_tensor = shape->fp8_block == 0;
-    const bool mx = shape->fp8_block == AIS_FP8_MX32;
+    const bool fp4 = shape->fp8_block == AIS_FP4_MX32;
+    const bool mx = shape->fp8_block == AIS_FP8_MX32 || fp4;
     if (do_roll) {
         if (!aligned(qH, 16) || !aligned(qW, 16) || !aligned(sH, 4) || !aligned(sW, 4)) return AIS_ERR_ALIGN;
         if (mx && (!aligned(sH, 16) || !aligned(sW, 16))) return AIS_ERR_ALIGN;
@@ -312,14 +329,18 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     }
     if (do_roll && mx) {
         // power-of-two scales per 32 elements: the block-scaled MMA applies them, the contraction stays in tensor memory
-        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
+        // FP4 codes are two per byte: the maps see d / 2 bytes per row with half the row stride
+        const uint64_t kb = fp4 ? d / 2 : d;
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, kb, T, fp4 ? shape->ldh / 2 : shape->ldh, 128, kBM,
+                       CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, kb, V, fp4 ? shape->ldw / 2 : shape->ldw, 128, kBN,
+                       CU_TENSOR_MAP_SWIZZLE_128B))
             return AIS_ERR_DEVICE;
-        a.ksteps = shape->d / 128;
+        a.ksteps = static_cast<int32_t>(kb / 128);
         a.sf_a = static_cast<const uint8_t*>(sH_);
         a.sf_b = static_cast<const uint8_t*>(sW_);
         a.nk4 = shape->d / 128;
-        if (launch_lmhead(kFwdMx, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
+        if (launch_lmhead(fp4 ? kFwdMx4 : kFwdMx, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_roll, lse_roll, dev_status, s) !=
             cudaSuccess)
             return AIS_ERR_DEVICE;

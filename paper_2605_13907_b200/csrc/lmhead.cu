@@ -37,7 +37,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     constexpr int STG = TWO_ACC ? kDhStages : kStages;                          // depth of the stage ring
     constexpr int STG_BYTES = TWO_ACC ? kDhStageBytes : kStageBytes;
     constexpr int A_BYTES = TWO_ACC ? 2 * kAStageBytes : kAStageBytes;
-    constexpr bool MX = (MODE == kFwdMx);                                       // block scales live in tensor memory
+    constexpr bool MX = (MODE == kFwdMx || MODE == kFwdMx4);                    // block scales live in tensor memory
+    constexpr bool FP4 = (MODE == kFwdMx4);                                     // 256 packed 4-bit elements per stage
+    constexpr int MX_SCALE_BYTES = FP4 ? 6 * kMxChunkBytes : 3 * kMxChunkBytes;
     constexpr int NBUF = (TWO_ACC || MX) ? 1 : 2;                               // accumulator sets that alternate
     constexpr uint32_t kMxScaleCol = 256;                                       // MX: scale columns after the accumulator
     const int warp = threadIdx.x >> 5;
@@ -79,16 +81,22 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag)) { ok = false; break; }
                         uint8_t* sA = stage_base + st.idx * STG_BYTES;
                         uint8_t* sB = sA + A_BYTES;
-                        mbar_expect_tx(&full[st.idx], MX ? STG_BYTES + kMxStageScaleBytes : STG_BYTES);
+                        mbar_expect_tx(&full[st.idx], MX ? STG_BYTES + MX_SCALE_BYTES : STG_BYTES);
                         const int kelem = (MODE == kFwdFp8T || MX) ? ks * 128 : ks * 64;
                         if (MX) {
-                            // the stage's scales: one 512-byte chunk for the 128 rows of A, the two adjacent chunks of B's 256 rows
+                            // the stage's scales (see the layout at ais_quantize_mxfp8): A's chunk(s) of this row tile, then the
+                            // adjacent chunk pair(s) of B's 256 rows; with FP4 a stage spans two chunk columns
                             uint8_t* sS = mx_scale_base + st.idx * kMxStageScaleBytes;
-                            bulk_load(sS, a.sf_a + (static_cast<int64_t>(w.rt >> 1) * a.nk4 + ks) * (2 * kMxChunkBytes) +
+                            constexpr int KC = FP4 ? 2 : 1;                    // chunk columns per stage
+                            const int64_t k4 = static_cast<int64_t>(ks) * KC;
+#pragma unroll
+                            for (int c = 0; c < KC; ++c)
+                                bulk_load(sS + c * kMxChunkBytes,
+                                          a.sf_a + (static_cast<int64_t>(w.rt >> 1) * a.nk4 + k4 + c) * (2 * kMxChunkBytes) +
                                               (w.rt & 1) * kMxChunkBytes,
-                                      kMxChunkBytes, &full[st.idx]);
-                            bulk_load(sS + kMxChunkBytes, a.sf_b + (static_cast<int64_t>(t) * a.nk4 + ks) * (2 * kMxChunkBytes),
-                                      2 * kMxChunkBytes, &full[st.idx]);
+                                          kMxChunkBytes, &full[st.idx]);
+                            bulk_load(sS + KC * kMxChunkBytes, a.sf_b + (static_cast<int64_t>(t) * a.nk4 + k4) * (2 * kMxChunkBytes),
+                                      KC * 2 * kMxChunkBytes, &full[st.idx]);
                         }
                         if (MODE == kBwdDh) {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kDhRows);
@@ -166,19 +174,28 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             }
                         } else if (MX) {
                             // scales of this stage: shared memory -> tensor memory (two column sets alternate between
-                            // stages), then one block-scaled instruction per 32-element block with its scale id
+                            // stages), then one block-scaled instruction per 32 bytes of K with its scale id.  Columns of a
+                            // set: A's chunks first (4 columns each), then B's (4 columns per 128 rows and chunk).
+                            constexpr int KC = FP4 ? 2 : 1;
                             const uint32_t sS = smem_u32(mx_scale_base + st.idx * kMxStageScaleBytes);
-                            const uint32_t tsf = tmem_base + kMxScaleCol + (st.idx & 1) * 16;
+                            const uint32_t tsf = tmem_base + kMxScaleCol + (st.idx & 1) * 32;
 #pragma unroll
-                            for (int c = 0; c < 3; ++c)
+                            for (int c = 0; c < 3 * KC; ++c)
                                 tmem_cp_32x128b_warpx4(tsf + 4 * c, smem_desc_noswizzle(sS + c * kMxChunkBytes, 16, 128));
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 const uint64_t adesc = smem_desc_sw128(sA + j * 32, 16, 1024);
                                 const uint64_t bdesc = smem_desc_sw128(sB + j * 32, 16, 1024);
-                                const uint32_t sel = static_cast<uint32_t>(j) << 30;      // byte of the scale columns
-                                mma_mxf8(tmem_base, adesc, bdesc, make_idesc_mx(kBM, kBN, j), tsf | sel, (tsf + 4) | sel,
-                                         (ks > 0 || j > 0) ? 1u : 0u);
+                                const uint32_t accum = (ks > 0 || j > 0) ? 1u : 0u;
+                                if (FP4) {
+                                    // instruction j covers scale blocks 2j, 2j+1: chunk j / 2, bytes 2 (j % 2) and the next
+                                    const uint32_t id = 2u * (j & 1), sel = id << 30;
+                                    mma_mxf4(tmem_base, adesc, bdesc, make_idesc_mx(kBM, kBN, id, 1u), (tsf + 4 * (j >> 1)) | sel,
+                                             (tsf + 4 * KC + 8 * (j >> 1)) | sel, accum);
+                                } else {
+                                    const uint32_t sel = static_cast<uint32_t>(j) << 30;      // byte of the scale columns
+                                    mma_mxf8(tmem_base, adesc, bdesc, make_idesc_mx(kBM, kBN, j), tsf | sel, (tsf + 4) | sel, accum);
+                                }
                             }
                         } else {
                             const uint32_t dcol = tmem_base + tb.idx * kBN;
@@ -458,6 +475,7 @@ cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& t
         case kFwdFp8T: return launch_mode<kFwdFp8T>(tmA, tmB, args, num_ctas, stream);
         case kBwdDw:   return launch_mode<kBwdDw>(tmA, tmB, args, num_ctas, stream);
         case kFwdMx:   return launch_mode<kFwdMx>(tmA, tmB, args, num_ctas, stream);
+        case kFwdMx4:  return launch_mode<kFwdMx4>(tmA, tmB, args, num_ctas, stream);
     }
     return cudaErrorInvalidValue;
 }
@@ -476,7 +494,9 @@ cudaError_t lmhead_prepare() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lmhead_kernel<kBwdDw>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(lmhead_kernel<kFwdMx>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(lmhead_kernel<kFwdMx>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(lmhead_kernel<kFwdMx4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
 }  // namespace ais

@@ -14,7 +14,8 @@ enum LmheadMode : int {
     kBwdDh   = 3,   // dH = c (.) (U W), contraction over the vocabulary
     kFwdFp8T = 4,   // E4M3 codes with one scale per tensor: whole contraction in tensor memory, one multiply after
     kBwdDw   = 5,   // dW += U^T H, contraction over the rows (both operands read with the contraction axis as rows)
-    kFwdMx   = 6    // E4M3 codes with one power-of-two (E8M0) scale per 32 elements: hardware block-scaled MMA
+    kFwdMx   = 6,   // E4M3 codes with one power-of-two (E8M0) scale per 32 elements: hardware block-scaled MMA
+    kFwdMx4  = 7    // packed E2M1 (FP4) codes with one E8M0 scale per 32 elements
 };
 
 constexpr int kBM = 128;                 // rows per tile (TMEM lanes)
@@ -30,9 +31,10 @@ constexpr int kDhStageBytes = 2 * kAStageBytes + kBStageBytes;
 constexpr int kDhStages = 3;
 static_assert(kDhStages * kDhStageBytes <= kStages * kStageBytes, "the dH stage ring must fit the same shared memory");
 constexpr int kNumBarriers = 2 * kStages + 4 + 1;
-// microscaling pass: per stage one 512-byte scale chunk for the 128 rows of A and two for the 256 rows of B
+// microscaling passes: per 128-byte K stage one 512-byte scale chunk for the 128 rows of A and two for the 256 rows of B
+// (FP8: 128 elements per stage), twice that with FP4 operands (256 elements per stage)
 constexpr int kMxChunkBytes = 512;
-constexpr int kMxStageScaleBytes = 3 * kMxChunkBytes;
+constexpr int kMxStageScaleBytes = 6 * kMxChunkBytes;
 constexpr int kThreads = 384;            // warp 0 TMA, warp 1 MMA, warps 2..3 idle, warps 4..11 epilogue
 constexpr int kEpiWarps = 8;
 constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kStages * kMxStageScaleBytes + kNumBarriers * 8 + 64;

@@ -139,6 +139,16 @@ __device__ __forceinline__ void mma_mxf8(uint32_t d_tmem, uint64_t adesc, uint64
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
         : "memory");
 }
+// The same with packed 4-bit E2M1 operands (64 elements of K per instruction, two 32-element scale blocks per row).
+__device__ __forceinline__ void mma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t tsfa,
+                                         uint32_t tsfb, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+        : "memory");
+}
 // Shared memory -> tensor memory copy of one scale chunk: 32 rows of 16 bytes go to lanes 0..31 x 4 columns and are
 // replicated to the other three lane quarters.  `sdesc` is a no-swizzle K-major matrix descriptor of the chunk.
 __device__ __forceinline__ void tmem_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc) {
@@ -219,8 +229,8 @@ __device__ __forceinline__ uint64_t smem_desc_noswizzle(uint32_t saddr, uint32_t
 //   bits 4-5 B scale id   bits 7-9 A format   bits 10-12 B format   bit 15 / 16 A / B is MN-major
 //   bits 17-22 N/8   bit 23 scale format (1 = E8M0)   bits 24-28 M/16   bits 29-30 A scale id
 // The scale id selects which byte of the 32-bit scale columns the instruction uses.
-__host__ __device__ constexpr uint32_t make_idesc_mx(uint32_t M, uint32_t N, uint32_t sf_id) {
-    return (sf_id << 4) | (0u << 7) | (0u << 10) | ((N >> 3) << 17) | (1u << 23) | ((M >> 4) << 24) | (sf_id << 29);
+__host__ __device__ constexpr uint32_t make_idesc_mx(uint32_t M, uint32_t N, uint32_t sf_id, uint32_t fmt = 0u /* E4M3; 1 = E2M1 of kind::mxf4 */) {
+    return (sf_id << 4) | (fmt << 7) | (fmt << 10) | ((N >> 3) << 17) | (1u << 23) | ((M >> 4) << 24) | (sf_id << 29);
 }
 
 // Instruction descriptor of tcgen05.mma (kind::f16 and kind::f8f6f4), dense, fp32 accumulator:

@@ -178,6 +178,57 @@ __global__ void __launch_bounds__(kQThreads) quantize_mx_kernel(const __nv_bfloa
 }
 
 // ------------------------------------------------------------------------------------------------
+// Microscaling FP4: as above with E2M1 elements (X = floor(log2 amax) - 2), two codes per byte, the element with
+// the lower index in the low nibble.  A lane turns 8 elements into 4 bytes.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cvt_e2m1x2(float hi, float lo) {
+    uint32_t r;
+    asm("{\n\t.reg .b8 t;\n\tcvt.rn.satfinite.e2m1x2.f32 t, %1, %2;\n\tcvt.u32.u8 %0, t;\n\t}" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__global__ void __launch_bounds__(kQThreads) quantize_mxfp4_kernel(const __nv_bfloat16* __restrict__ x, int64_t rows, int64_t cols,
+                                                                   int64_t ld, uint8_t* __restrict__ codes, int64_t ldq,
+                                                                   uint8_t* __restrict__ scales) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kQRows;
+    const int64_t col0 = static_cast<int64_t>(blockIdx.x) * kQCols;
+    const int64_t nk4 = cols / 128;
+#pragma unroll 1
+    for (int rr = 0; rr < 4; ++rr) {
+        const int64_t row = row0 + warp * 4 + rr;
+        if (row >= rows) break;
+#pragma unroll
+        for (int it = 0; it < kQIters; ++it) {
+            const int64_t col = col0 + it * 256 + lane * 8;
+            const bool in = col < cols;
+            const uint4 raw = in ? __ldg(reinterpret_cast<const uint4*>(x + row * ld + col)) : make_uint4(0, 0, 0, 0);
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+            uint32_t m = __vmaxu2(__vmaxu2(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu), __vmaxu2(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu));
+            m = max(m & 0xFFFFu, m >> 16);
+            m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
+            m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
+            const int e = static_cast<int>(m >> 7);
+            const int code = m == 0u ? 127 : max(e - 2, 0);
+            const float mult = __uint_as_float(static_cast<uint32_t>(254 - code) << 23);      // 2^(127 - code), exact
+            if (!in) continue;
+            uint32_t out = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float lo = __uint_as_float(w[i] << 16) * mult, hi = __uint_as_float(w[i] & 0xFFFF0000u) * mult;
+                out |= cvt_e2m1x2(hi, lo) << (8 * i);
+            }
+            *reinterpret_cast<uint32_t*>(codes + row * ldq + col / 2) = out;
+            if ((lane & 3) == 0) {
+                const int64_t kb = col / 32;
+                scales[((row >> 8) * nk4 + (kb >> 2)) * 1024 + ((row >> 7) & 1) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4 +
+                       (kb & 3)] = static_cast<uint8_t>(code);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Per-tensor dynamic scaling: one scale for the whole matrix.  Pass 1 folds max|x| (as a bf16 bit pattern; the
 // patterns of non-negative values order like the values, so an integer atomicMax is exact and order-free)
 // into the word that will hold the scale, pass 2 turns it into s = amax / 448, pass 3 quantises.
@@ -744,13 +795,16 @@ cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t l
 }
 
 cudaError_t launch_quantize_mx(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,
-                               uint8_t* scales, size_t scale_bytes, cudaStream_t stream) {
+                               uint8_t* scales, size_t scale_bytes, bool fp4, cudaStream_t stream) {
     // rows that pad the last chunks carry the neutral scale
     cudaError_t e = cudaMemsetAsync(scales, 127, scale_bytes, stream);
     if (e != cudaSuccess) return e;
     if (rows == 0 || cols == 0) return cudaSuccess;
     dim3 grid(static_cast<unsigned>((cols + kQCols - 1) / kQCols), static_cast<unsigned>((rows + kQRows - 1) / kQRows));
-    quantize_mx_kernel<<<grid, kQThreads, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), rows, cols, ld, codes, ldq, scales);
+    if (fp4)
+        quantize_mxfp4_kernel<<<grid, kQThreads, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), rows, cols, ld, codes, ldq, scales);
+    else
+        quantize_mx_kernel<<<grid, kQThreads, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), rows, cols, ld, codes, ldq, scales);
     return cudaGetLastError();
 }
 

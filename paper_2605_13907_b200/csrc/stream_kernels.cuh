@@ -19,7 +19,8 @@ cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t l
 // Microscaling: E8M0 scale per 32 elements, packed in 512-byte chunks of 128 rows x 4 blocks; `scale_bytes` is the
 // size of the whole packed array (rows padded to a multiple of 256), filled with the neutral code first.
 cudaError_t launch_quantize_mx(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,
-                               uint8_t* scales, size_t scale_bytes, cudaStream_t stream);
+                               uint8_t* scales, size_t scale_bytes, bool fp4 /* E2M1 elements, two per byte */,
+                               cudaStream_t stream);
 
 // One scale for the whole matrix (written to *scale on the device), then the codes.
 cudaError_t launch_quantize_tensor(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,

@@ -69,11 +69,17 @@ def test_mx_rollout_path(case):
     assert np.linalg.norm(dH - ref["dH"]) <= DH_REL * np.linalg.norm(ref["dH"])
 
 
-def test_mx_fullsize_sampled_rows():
-    """qwen3_8b shape in the launch configuration the benchmark's --fp8-mx variant times: all of W's codes and scale
-    bytes bit-exact, and the rollout log-probs of a seeded sample of rows against the oracle over the whole vocabulary."""
+@pytest.mark.parametrize("fmt", ["fp8", "fp4"])
+def test_mx_fullsize_sampled_rows(fmt):
+    """qwen3_8b shape in the launch configuration the benchmark's --fp8-mx / --fp4-mx variants time: all of W's codes and
+    scale bytes bit-exact, and the rollout log-probs of a seeded sample of rows against the oracle over the whole
+    vocabulary."""
     import paper_2605_13907_b200 as ais
-    w = workloads.scaled(workloads.WORKLOADS["qwen3_8b"], block=ais.FP8_MX32)
+    fp4 = fmt == "fp4"
+    quant = e4m3.quantize_mxfp4 if fp4 else e4m3.quantize_mx
+    dequant = e4m3.dequantize_mxfp4 if fp4 else e4m3.dequantize_mx
+    stored = e4m3.pack_fp4_pairs if fp4 else (lambda c: c)
+    w = workloads.scaled(workloads.WORKLOADS["qwen3_8b"], block=ais.FP4_MX32 if fp4 else ais.FP8_MX32)
     batch = workloads.make_batch(w, device="cuda")
     T = batch.T
     step = ais.AisStep(T, w.d, w.V, w.P, w.G, w.block, want_grad=False)
@@ -83,9 +89,9 @@ def test_mx_fullsize_sampled_rows():
     rng = np.random.default_rng(5)
     rows = np.unique(np.concatenate([[0, 127, 128, T - 1, (T // 128) * 128 - 1, (T // 128) * 128], rng.integers(0, T, 42)]))
     Hs = batch.H[torch.as_tensor(rows, device="cuda")].float().cpu().numpy().astype(np.float64)
-    qHs, sHs = e4m3.quantize_mx(Hs)
-    assert np.array_equal(step.qH.cpu().numpy()[rows], qHs)
-    Hq = e4m3.dequantize_mx(qHs, sHs)
+    qHs, sHs = quant(Hs)
+    assert np.array_equal(step.qH.cpu().numpy()[rows], stored(qHs))
+    Hq = dequant(qHs, sHs)
     sH_gpu = step.sH.cpu().numpy().reshape(-1, w.d // 128, 2, 512)
     for i, r in enumerate(rows):
         for kb in (0, 1, 63, 127):
@@ -96,14 +102,62 @@ def test_mx_fullsize_sampled_rows():
     CH = 4096                                               # a multiple of 256: whole scale groups per piece
     for v0 in range(0, w.V, CH):
         Wc = batch.W[v0:v0 + CH].float().cpu().numpy().astype(np.float64)
-        qc, sc = e4m3.quantize_mx(Wc)
-        assert np.array_equal(qW_gpu[v0:v0 + CH], qc), v0
+        qc, sc = quant(Wc)
+        assert np.array_equal(qW_gpu[v0:v0 + CH], stored(qc)), v0
         n = Wc.shape[0]
         packed = e4m3.pack_mx_scales(sc)
         assert np.array_equal(sW_gpu[v0 // 256:v0 // 256 + packed.shape[0]], packed), v0
-        z[:, v0:v0 + n] = Hq @ e4m3.dequantize_mx(qc, sc).T
+        z[:, v0:v0 + n] = Hq @ dequant(qc, sc).T
     tok = batch.tokens.cpu().numpy()[rows]
     msk = batch.mask.cpu().numpy()[rows]
     lp_ref, _ = oais.log_softmax_gather(z, tok, msk)
     got = step.lp_roll.cpu().numpy()[rows]
     assert np.max(np.abs(got - lp_ref)) <= 1e-3, np.max(np.abs(got - lp_ref))
+
+
+# --------------------------------------------------------------------------- FP4 elements
+def test_mxfp4_quantiser_bit_exact():
+    import paper_2605_13907_b200 as ais
+    g = torch.Generator().manual_seed(12)
+    rows, cols = 301, 512
+    x = torch.randn(rows, cols, generator=g) * torch.exp(torch.randn(rows, 1, generator=g) * 4)
+    x[5] = 0.0
+    x[6, :32] = 1e-39
+    x[7, 40] = 3.0e38
+    x[8, :64] = torch.tensor([7.0, -6.5, 5.0, 2.5, 0.25, 0.75, 1.25, 3.5] * 8)      # clipping band and every tie
+    x[9] = -0.0
+    xb = x.to(torch.bfloat16)
+    codes, packed = ais.quantize_fp8(xb.cuda(), ais.FP4_MX32)
+    torch.cuda.synchronize()
+    ref_c, ref_s = e4m3.quantize_mxfp4(xb.float().numpy())
+    assert codes.shape == (rows, cols // 2)
+    assert np.array_equal(codes.cpu().numpy(), e4m3.pack_fp4_pairs(ref_c))
+    assert np.array_equal(packed.cpu().numpy(), e4m3.pack_mx_scales(ref_s).reshape(-1))
+
+
+@pytest.mark.parametrize("case", ["tiny", "ragged"])
+def test_mxfp4_rollout_path(case):
+    """FP4 rollouts are far from the trainer (d_bar of order 1), which is the regime where the mixing coefficient
+    saturates; what is checked is parity with the oracle on the same codes."""
+    import paper_2605_13907_b200 as ais
+    base = workloads.WORKLOADS["tiny"]
+    w = workloads.scaled(base, block=ais.FP4_MX32) if case == "tiny" else \
+        workloads.scaled(base, block=ais.FP4_MX32, d=512, V=1336, P=3, G=4, lengths="uniform:5:90", seed=84)
+    b = _cuda(workloads.make_batch(w, device="cpu"))
+    step = ais.AisStep(b.T, w.d, w.V, w.P, w.G, w.block)
+    step.step(b.H, b.W, b.tokens, b.mask, b.seq_offsets.cuda(), b.rewards.cuda())
+    torch.cuda.synchronize()
+    a = workloads.to_numpy(b)
+    ref = oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, oais.MXFP4)
+    T = b.T
+    assert int(step.status.item()) == 0
+    assert np.array_equal(step.qH.cpu().numpy()[:T], e4m3.pack_fp4_pairs(ref["qH"]))
+    assert np.array_equal(step.qW.cpu().numpy(), e4m3.pack_fp4_pairs(ref["qW"]))
+    assert np.array_equal(step.sW.cpu().numpy(), e4m3.pack_mx_scales(ref["sW"]).reshape(-1))
+    err = np.abs(step.lp_roll.cpu().numpy()[:T] - ref["lp_roll"])
+    assert err.max() <= 1e-3, err.max()
+    d = step.read_diag()
+    assert abs(d["alpha"] - ref["diag"]["alpha"]) <= ALPHA_ATOL
+    assert abs(d["d_bar"] - ref["diag"]["d_bar"]) <= 1e-3 * max(1.0, ref["diag"]["d_bar"])
+    dH = step.dH.float().cpu().numpy()[:T].astype(np.float64)
+    assert np.linalg.norm(dH - ref["dH"]) <= DH_REL * np.linalg.norm(ref["dH"])
