@@ -468,8 +468,8 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
     // Every warp owns a contiguous range of row groups and its lanes interleave inside it, so a lane's rows only
     // move forward: one binary search for its first group, then the sequence index steps (the next boundary is kept
     // in a register).  Valid rows are counted per sequence on the way (integer atomics: the result does not depend
-    // on their order).  The rows of one pass of the loop (at most 2 VEC) are summed in fp32 and those short sums
-    // go into the fp64 accumulators, which keeps the fp64 pipe out of the per-row work.
+    // on their order).  Runs of at most 64 rows are summed in fp32 and those short sums go into the fp64
+    // accumulators, which keeps the fp64 pipe out of the per-row work.
     int sq = -1, cur = -1, cnt = 0;
     int64_t next_b = 0;                                   // first row of sequence sq + 1 (or "never" for the last one)
     float f[kNumMoments];
@@ -519,6 +519,37 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
     auto add_group = [&](const RowGroup<VEC>& r, int64_t g) {
         if (!r.any) return;
         const int64_t t0 = g * VEC;
+        seek(t0);
+        if (VEC > 1 && t0 + VEC <= next_b) {
+            // the usual case, all rows of the group in one sequence: one advantage and one weight source for the
+            // group, masked rows drop out by selection, and the sums that involve A follow from sum w and sum w^2
+            const float A = adv[sq];
+            const float wseq = seq_logw ? __expf(seq_logw[sq]) : 0.f;
+            float n = 0.f, sw = 0.f, sw2 = 0.f;
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) {
+                const bool on = r.mk[j] != 0;
+                const float dl = r.lt[j] - r.lr[j];
+                const float rho = __expf(dl);
+                const float w = fminf(seq_logw ? wseq : rho, C);
+                n += on ? 1.0f : 0.f;
+                sw += on ? w : 0.f;
+                sw2 += on ? w * w : 0.f;
+                f[3] += on ? fabsf(dl) : 0.f;
+                f[8] -= on ? dl : 0.f;
+                f[9] += on ? __expf(r.lr[j]) * fabsf(rho - 1.0f) : 0.f;
+            }
+            f[0] += n;
+            f[1] += sw;
+            f[2] += sw2;
+            f[4] = fmaf(A, n, f[4]);
+            f[5] = fmaf(A * A, n, f[5]);
+            f[6] = fmaf(A, sw, f[6]);
+            f[7] = fmaf(A * A, sw2, f[7]);
+            if (sq != cur) { flush(); cur = sq; }
+            cnt += static_cast<int>(n);
+            return;
+        }
 #pragma unroll
         for (int j = 0; j < VEC; ++j) {
             if (r.mk[j]) {
@@ -534,15 +565,17 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
     const int64_t per = ((ngroups + nwarps - 1) / nwarps + 63) / 64 * 64;             // groups per warp
     const int64_t g_end = (gw + 1) * per < ngroups ? (gw + 1) * per : ngroups;
     int64_t g = gw * per + lane;
-    for (; g + 32 < g_end; g += 64) {                                                  // two groups in flight per lane
+    clear();
+    for (int pass = 0; g + 32 < g_end; g += 64) {                                      // two groups in flight per lane
         const RowGroup<VEC> r0 = load_group<VEC>(lp_train, lp_roll, mask, g);
         const RowGroup<VEC> r1 = load_group<VEC>(lp_train, lp_roll, mask, g + 32);
-        clear();
         add_group(r0, g);
         add_group(r1, g + 32);
-        commit();
+        if ((++pass & 7) == 0) {                                                       // at most 64 rows per fp32 run
+            commit();
+            clear();
+        }
     }
-    clear();
     if (g < g_end) add_group(load_group<VEC>(lp_train, lp_roll, mask, g), g);
     flush();
     // rows after the last whole group: the first threads of the grid, one row each
