@@ -242,25 +242,57 @@ def run_ours(args) -> None:
     h2d = sum(t.numel() * t.element_size() for t in pin.values())
     d2h = dH_host.numel() * dH_host.element_size() + small_host.numel() * 8
 
-    def e2e_step():
-        H2.copy_(pin["H"], non_blocking=True)
+    # Every step copies its inputs in from pinned host memory and its results (dH, diagnostics, loss) out.  The copies
+    # run on two side streams so that a step's input copy and the previous step's result copy overlap the tensor-core
+    # passes: two device buffers for H alternate, and the backward waits until the previous dH has left the device.
+    in_s, out_s = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    Hbuf = [H2, torch.empty_like(batch.H)]
+    ev_in = [torch.cuda.Event(), torch.cuda.Event()]
+    ev_used = [torch.cuda.Event(), torch.cuda.Event()]      # the step that read Hbuf[i] has finished
+    ev_bwd, ev_out = torch.cuda.Event(), torch.cuda.Event()
+
+    def e2e_prefetch(i):
+        with torch.cuda.stream(in_s):
+            in_s.wait_event(ev_used[i % 2])
+            Hbuf[i % 2].copy_(pin["H"], non_blocking=True)
+            ev_in[i % 2].record(in_s)
+
+    def e2e_step(i, last):
+        stream.wait_event(ev_in[i % 2])
+        if not last:
+            e2e_prefetch(i + 1)
         tok2.copy_(pin["tokens"], non_blocking=True)
         msk2.copy_(pin["mask"], non_blocking=True)
         offs2.copy_(pin["offs"], non_blocking=True)
         rew2.copy_(pin["rew"], non_blocking=True)
-        step.step(H2, batch.W, tok2, msk2, offs2, rew2)
-        dH_host.copy_(step.dH, non_blocking=True)
-        small_host[:-1].copy_(step.diag, non_blocking=True)
-        small_host[-1:].copy_(step.loss.double(), non_blocking=True)
+        Hi = Hbuf[i % 2]
+        step.forward(Hi, batch.W, tok2, msk2)
+        step.diagnose(msk2, offs2, rew2)
+        stream.wait_event(ev_out)                           # dH and the diagnostics of the previous step are on the host
+        step.backward(Hi, batch.W, tok2, msk2, offs2)
+        ev_bwd.record(stream)
+        ev_used[i % 2].record(stream)
+        with torch.cuda.stream(out_s):
+            out_s.wait_event(ev_bwd)
+            dH_host.copy_(step.dH, non_blocking=True)
+            small_host[:-1].copy_(step.diag, non_blocking=True)
+            small_host[-1:].copy_(step.loss.double(), non_blocking=True)
+            ev_out.record(out_s)
 
     e2e_steps = max(1, min(args.steps, 5))
-    e2e_step()
+    ev_used[0].record(stream)
+    ev_used[1].record(stream)
+    ev_out.record(stream)
+    e2e_prefetch(0)
+    e2e_step(0, True)                                       # warm-up
     barrier()
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
+    e2e_prefetch(0)
+    for i in range(e2e_steps):
+        e2e_step(i, i == e2e_steps - 1)
+    stream.wait_event(ev_out)                               # the last results have reached the host
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
