@@ -46,3 +46,26 @@ def test_host_side_validation_needs_no_gpu():
     import torch
     with pytest.raises(ais.AisError):                                   # CPU tensors are refused: no CPU path
         ais.quantize_fp8(torch.zeros(4, 128, dtype=torch.bfloat16), 128)
+
+
+def test_microscaling_entry_points_validate_on_the_host():
+    """Sizes of the packed scale arrays, the shape rules of the two block-scaled variants and the argument checks that
+    come before any device call."""
+    import paper_2605_13907_b200 as ais
+    lib = ais.lib()
+    assert ais.mx_scale_bytes(1, 128) == 2 * 512                       # rows padded to 256: two chunks of 128 rows
+    assert ais.mx_scale_bytes(256, 4096) == 2 * 32 * 512
+    assert ais.mx_scale_bytes(257, 4096) == 4 * 32 * 512
+    assert ais.mx_scale_bytes(10, 100) == 0                            # columns must be a multiple of 128
+    p = ais.default_params()
+    assert p.seq_level_weights == 0
+    assert ais.workspace_bytes(ais.make_shape(1000, 4096, 151936, 8, 8, ais.FP8_MX32), p) > 0
+    assert ais.workspace_bytes(ais.make_shape(1000, 4096, 151936, 8, 8, ais.FP4_MX32), p) > 0
+    assert ais.workspace_bytes(ais.make_shape(1000, 4224, 151936, 8, 8, ais.FP4_MX32), p) == 0    # FP4 wants d % 256 == 0
+    assert ais.workspace_bytes(ais.make_shape(1000, 4096, 151936, 8, 8, -7), p) == 0
+    null = ctypes.c_void_p(None)
+    one = ctypes.c_void_p(256)                                         # never dereferenced: the checks below fail first
+    for fn in (lib.ais_quantize_mxfp8, lib.ais_quantize_mxfp4):
+        assert fn(null, 4, 128, 128, one, 128, one, null) == -1       # AIS_ERR_NULL
+        assert fn(one, 4, 100, 128, one, 128, one, null) == -2        # AIS_ERR_SHAPE: columns not a multiple of 128
+        assert fn(one, 4, 256, 128, one, 256, one, null) == -2        # row stride shorter than the row
