@@ -6,8 +6,10 @@
 // thread) and column half (w-4)/4 of the 256-column accumulator.  The dH pass gives a CTA two row tiles
 // (256 rows, both accumulators) so that every W slice it loads is used twice; its contraction over the
 // vocabulary is so long that the one epilogue per unit need not overlap anything.  Two 256-column accumulators
-// alternate so that the epilogue of one tile overlaps the MMAs of the next.  The rollout pass with per-block
-// scales has a kernel of its own (lmhead_fp8.cu).
+// alternate so that the epilogue of one tile overlaps the MMAs of the next.  The microscaling modes add a fourth
+// warpgroup (warps 12..15) that moves each stage's block scales from shared to tensor memory, where the
+// block-scaled MMA reads them; their scale columns leave room for one accumulator only.  The rollout pass with
+// fp32 per-block scales has a kernel of its own (lmhead_fp8.cu).
 #include <type_traits>
 
 #include "lmhead_common.cuh"
@@ -17,8 +19,10 @@ namespace ais {
 
 namespace {
 
+constexpr int threads_of(int mode) { return (mode == kFwdMx || mode == kFwdMx4) ? kMxThreads : kThreads; }
+
 template <int MODE>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(threads_of(MODE), 1)
 lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const LmheadArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -30,6 +34,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     uint64_t* tfull = empty + kStages;           // [2]         MMA -> epilogue
     uint64_t* tempty = tfull + 2;                // [2]         epilogue -> MMA
     uint64_t* done = tempty + 2;                 // [1]         all MMAs of this CTA have completed
+    uint64_t* sfull = done + 1;                  // [kStages]   scale warps -> MMA (microscaling passes)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBarriers);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -41,13 +46,15 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     constexpr bool FP4 = (MODE == kFwdMx4);                                     // 256 packed 4-bit elements per stage
     constexpr int MX_SCALE_BYTES = FP4 ? 6 * kMxChunkBytes : 3 * kMxChunkBytes;
     constexpr int NBUF = (TWO_ACC || MX) ? 1 : 2;                               // accumulator sets that alternate
-    constexpr uint32_t kMxScaleCol = 256;                                       // MX: scale columns after the accumulator
+    constexpr uint32_t kMxScaleCol = 256;                                       // MX: scale columns after the accumulator,
+    constexpr uint32_t kMxSetCols = 32;                                         // one set of 32 per stage of the ring
+    constexpr int kScaleWarp0 = 12;                                             // MX: first of the four scale warps
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int num_units = TWO_ACC ? a.n_row_tiles * a.n_col_tiles : a.n_row_tiles * a.nsplit;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); mbar_init(&sfull[i], 4); }
         for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
         mbar_init(done, 1);
         *abort_flag = 0;
@@ -65,10 +72,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const uint32_t tmem_base = *tmem_slot;
 
     // Microscaling pass: its one accumulator is read into registers in one go so that it can go back to the MMA
-    // issuer at once; the first warpgroup hands the registers for that to the epilogue (384 x 168 = 128 x 40 + 256 x 232).
+    // issuer at once; the other warps hand the registers for that to the epilogue (512 x 128 = 256 x 32 + 256 x 224).
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (MX) reg_dealloc<40>();
+        if (MX) reg_dealloc<32>();
         if (lane == 0) {
             Pipe st(STG);
             uint32_t issued = 0;
@@ -134,7 +141,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (MX) reg_dealloc<40>();
+        if (MX) reg_dealloc<32>();
         if (lane == 0) {
             constexpr uint32_t idesc =
                 (MODE == kFwdFp8T || MX) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
@@ -173,15 +180,13 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                         idesc, accum);
                             }
                         } else if (MX) {
-                            // scales of this stage: shared memory -> tensor memory (two column sets alternate between
-                            // stages), then one block-scaled instruction per 32 bytes of K with its scale id.  Columns of a
-                            // set: A's chunks first (4 columns each), then B's (4 columns per 128 rows and chunk).
+                            // the scale warps have put this stage's scales into its column set: A's chunks first (4 columns
+                            // each), then B's (4 columns per 128 rows and chunk).  One block-scaled instruction per 32 bytes
+                            // of K, each with its scale id.
                             constexpr int KC = FP4 ? 2 : 1;
-                            const uint32_t sS = smem_u32(mx_scale_base + st.idx * kMxStageScaleBytes);
-                            const uint32_t tsf = tmem_base + kMxScaleCol + (st.idx & 1) * 32;
-#pragma unroll
-                            for (int c = 0; c < 3 * KC; ++c)
-                                tmem_cp_32x128b_warpx4(tsf + 4 * c, smem_desc_noswizzle(sS + c * kMxChunkBytes, 16, 128));
+                            if (!mbar_wait(&sfull[st.idx], st.phase, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                            const uint32_t tsf = tmem_base + kMxScaleCol + st.idx * kMxSetCols;
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 const uint64_t adesc = smem_desc_sw128(sA + j * 32, 16, 1024);
@@ -220,10 +225,41 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             tc_commit(done);
         }
     } else if (warp < 4) {
-        if (MX) reg_dealloc<40>();          // the idle warps of the first warpgroup give their registers away too
+        if (MX) reg_dealloc<32>();          // the idle warps of the first warpgroup give their registers away too
+    } else if (MX && warp >= kScaleWarp0) {
+        // ------------------------------------------------------------------ scale warps (microscaling passes)
+        // A scale chunk in shared memory is 32 rows of 16 bytes: row l holds, for each of four 32-row groups, the
+        // four E8M0 bytes of the stage's K blocks.  The MMA reads scales from tensor memory, lane l of every lane
+        // quarter, one 32-bit column per group: warp 12 + q copies the stage's chunks to quarter q with plain stores
+        // (a tcgen05.cp from the MMA thread would queue in front of the MMAs and costs about a tenth of the pass).
+        // A stage's column set is free again once its `empty` barrier has completed, which the producer waited for
+        // before the loads that complete `full`.
+        reg_dealloc<32>();
+        constexpr int KC = FP4 ? 2 : 1;
+        const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        Pipe st(STG);
+        bool ok = true;
+        for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+            const Unit w = decode_unit<MODE>(a, u);
+            if (!unit_active<MODE>(a, w)) continue;
+            for (int t = w.t0; t < w.t1 && ok; ++t) {
+                for (int ks = 0; ks < a.ksteps; ++ks) {
+                    if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag)) { ok = false; break; }
+                    const uint4* src = reinterpret_cast<const uint4*>(mx_scale_base + st.idx * kMxStageScaleBytes) + lane;
+                    const uint32_t tsf = tmem_base + lane_addr + kMxScaleCol + st.idx * kMxSetCols;
+#pragma unroll
+                    for (int c = 0; c < 3 * KC; ++c) tmem_st_32x32b_x4(tsf + 4 * c, src[c * (kMxChunkBytes / 16)]);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sfull[st.idx]);
+                    st.advance();
+                }
+            }
+        }
     } else {
         // ------------------------------------------------------------------ epilogue warps
-        if (MX) reg_alloc<232>();
+        if (MX) reg_alloc<224>();
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int half = (warp - 4) >> 2;             // column half of the accumulator
         const int r_in_tile = q * 32 + lane;
@@ -461,7 +497,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 template <int MODE>
 static cudaError_t launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, const LmheadArgs& args, int num_ctas,
                                cudaStream_t stream) {
-    lmhead_kernel<MODE><<<num_ctas, kThreads, kSmemBytes, stream>>>(tmA, tmB, args);
+    lmhead_kernel<MODE><<<num_ctas, threads_of(MODE), kSmemBytes, stream>>>(tmA, tmB, args);
     return cudaGetLastError();
 }
 

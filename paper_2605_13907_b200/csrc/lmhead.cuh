@@ -30,13 +30,14 @@ constexpr int kDhRows = 2 * kBM;
 constexpr int kDhStageBytes = 2 * kAStageBytes + kBStageBytes;
 constexpr int kDhStages = 3;
 static_assert(kDhStages * kDhStageBytes <= kStages * kStageBytes, "the dH stage ring must fit the same shared memory");
-constexpr int kNumBarriers = 2 * kStages + 4 + 1;
+constexpr int kNumBarriers = 3 * kStages + 4 + 1;
 // microscaling passes: per 128-byte K stage one 512-byte scale chunk for the 128 rows of A and two for the 256 rows of B
 // (FP8: 128 elements per stage), twice that with FP4 operands (256 elements per stage)
 constexpr int kMxChunkBytes = 512;
 constexpr int kMxStageScaleBytes = 6 * kMxChunkBytes;
 constexpr int kThreads = 384;            // warp 0 TMA, warp 1 MMA, warps 2..3 idle, warps 4..11 epilogue
 constexpr int kEpiWarps = 8;
+constexpr int kMxThreads = 512;          // microscaling passes: warps 12..15 move the block scales into tensor memory
 constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kStages * kMxStageScaleBytes + kNumBarriers * 8 + 64;
 
 struct LmheadArgs {
