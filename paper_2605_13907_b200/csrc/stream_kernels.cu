@@ -1,5 +1,6 @@
 // Streaming kernels of the AIS path (everything that is not a dense contraction).
 #include "stream_kernels.cuh"
+#include "ptx.cuh"
 
 #include <cuda_bf16.h>
 #include <math.h>
@@ -596,14 +597,215 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
     }
 }
 
+// The same moments for 16-byte aligned inputs, fed by bulk asynchronous copies: a block walks a contiguous range of
+// 1024-row tiles; thread 0 keeps four tiles (two log-prob vectors and the mask bytes, 9 KB each) in flight into a ring
+// of shared-memory stages, completion arrives on one mbarrier per stage, and every thread takes the four rows
+// 4 tid .. 4 tid + 3 of each tile from shared memory.  Memory latency is carried by the copies in flight (36 KB per
+// block, four blocks per SM) instead of by registers, and the per-row work is kept to about twenty instructions
+// (flush-to-zero exponentials, 32-bit row indices, the group's sequence looked up before the data arrives), because
+// at 9 bytes per row the instruction issue rate is the next limit after HBM.  Rows after the last whole tile are read
+// directly.  Summation order is fixed by the grid as above.
+constexpr int kMomRows = 1024;
+constexpr int kMomStages = 4;
+constexpr int kMomStageBytes = kMomRows * 9;
+
+__device__ __forceinline__ float exp_ftz(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x * 1.4426950408889634f));
+    return y;
+}
+
+template <bool SEQ>   // SEQ: every row carries its sequence's truncated weight instead of its own
+__global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const float* __restrict__ lp_train,
+                                                                         const float* __restrict__ lp_roll,
+                                                                         const uint8_t* __restrict__ mask,
+                                                                         const int32_t* __restrict__ seq_offsets,
+                                                                         const float* __restrict__ adv, int T, int S, float C,
+                                                                         double* __restrict__ partials,
+                                                                         int32_t* __restrict__ n_valid_seq,
+                                                                         const float* __restrict__ seq_logw) {
+    static_assert(kDiagThreads * 4 == kMomRows, "one 4-row group per thread and tile");
+    __shared__ __align__(128) uint8_t stages[kMomStages * kMomStageBytes];
+    __shared__ uint64_t full[kMomStages];
+    __shared__ double scratch[32];
+    __shared__ int abort_flag;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int ntiles = T / kMomRows;
+    const int per = (ntiles + gridDim.x - 1) / gridDim.x;
+    const int tile0 = blockIdx.x * per < ntiles ? blockIdx.x * per : ntiles;
+    const int tile1 = tile0 + per < ntiles ? tile0 + per : ntiles;
+    if (tid == 0) {
+        for (int i = 0; i < kMomStages; ++i) mbar_init(&full[i], 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    auto issue = [&](int tile, int st) {               // thread 0: the three copies of one tile onto the stage's barrier
+        uint8_t* dst = stages + st * kMomStageBytes;
+        const size_t r0 = static_cast<size_t>(tile) * kMomRows;
+        mbar_expect_tx(&full[st], kMomStageBytes);
+        bulk_load(dst, lp_train + r0, kMomRows * 4, &full[st]);
+        bulk_load(dst + kMomRows * 4, lp_roll + r0, kMomRows * 4, &full[st]);
+        bulk_load(dst + kMomRows * 8, mask + r0, kMomRows, &full[st]);
+    };
+    int issued = tile0;                                 // first tile not yet requested (thread 0)
+    if (tid == 0)
+        for (; issued < tile1 && issued < tile0 + kMomStages; ++issued) issue(issued, issued - tile0);
+
+    double acc[10];
+    float f[10];
+#pragma unroll
+    for (int i = 0; i < 10; ++i) { acc[i] = 0.0; f[i] = 0.f; }
+    constexpr int kNever = 0x7fffffff;
+    int sq = -1, cur = -1;
+    int next_b = 0;                                     // first row of sequence sq + 1 (or "never" for the last one)
+    float A = 0.f, wseq = 0.f;                          // advantage and sequence-level weight of sequence `cur`
+    int wsq = -1, wcnt = 0;                             // lane 0: valid rows of the warp's strips counted for sequence wsq
+    auto seek = [&](int t) {
+        if (sq < 0) {
+            sq = seq_of_row(seq_offsets, S, t);
+            next_b = sq + 1 < S ? seq_offsets[sq + 1] : kNever;
+        }
+        while (t >= next_b) {
+            ++sq;
+            next_b = sq + 1 < S ? seq_offsets[sq + 1] : kNever;
+        }
+    };
+    auto enter = [&]() {                                // the row's sequence becomes the current one
+        if (sq != cur) {
+            cur = sq;
+            A = adv[sq];
+            if (SEQ) wseq = fminf(__expf(seq_logw[sq]), C);
+        }
+    };
+    // sums over the rows of a group whose mask byte in `mk` is set, all in sequence `cur`; returns how many they are
+    auto add_rows = [&](const float (&lt)[4], const float (&lr)[4], uint32_t mk) -> int {
+        int n = 0;
+        float sw = 0.f, sw2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const bool on = (mk & (0xFFu << (8 * j))) != 0u;
+            const float dl = on ? lt[j] - lr[j] : 0.f;             // a masked row enters with dl = 0 and weight 0
+            const float rho = exp_ftz(dl);
+            const float w = on ? (SEQ ? wseq : fminf(rho, C)) : 0.f;
+            n += on ? 1 : 0;
+            sw += w;
+            sw2 = fmaf(w, w, sw2);
+            f[3] += fabsf(dl);
+            f[8] -= dl;
+            f[9] = fmaf(exp_ftz(on ? lr[j] : 0.f), fabsf(rho - 1.0f), f[9]);     // |e^lt - e^lr| = e^lr |rho - 1|
+        }
+        const float nf = static_cast<float>(n);
+        f[0] += nf;
+        f[1] += sw;
+        f[2] += sw2;
+        f[4] = fmaf(A, nf, f[4]);
+        f[5] = fmaf(A * A, nf, f[5]);
+        f[6] = fmaf(A, sw, f[6]);
+        f[7] = fmaf(A * A, sw2, f[7]);
+        return n;
+    };
+
+    bool failed = false;
+    for (int tile = tile0; tile < tile1; ++tile) {
+        const int k = tile - tile0;
+        const int st = k % kMomStages;
+        // the group's sequence, advantage and weight source do not depend on the tile's data: fetched before the wait
+        const int t0 = tile * kMomRows + 4 * tid;
+        seek(t0);
+        const bool single = t0 + 4 <= next_b;          // the usual case: the four rows belong to one sequence
+        if (single) enter();
+        // warp-uniform outcome: the warp-wide operations below need all 32 lanes
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&full[st], static_cast<uint32_t>((k / kMomStages) & 1), &abort_flag));
+        if (ok) {
+            const uint8_t* src = stages + st * kMomStageBytes;
+            const float4 a = reinterpret_cast<const float4*>(src)[tid];
+            const float4 b = reinterpret_cast<const float4*>(src + kMomRows * 4)[tid];
+            const uint32_t mk = reinterpret_cast<const uint32_t*>(src + kMomRows * 8)[tid];
+            const float lt[4] = {a.x, a.y, a.z, a.w}, lr[4] = {b.x, b.y, b.z, b.w};
+            int n = 0;
+            if (single) {
+                if (mk != 0u) n = add_rows(lt, lr, mk);
+            } else if (mk != 0u) {
+                int j = 0;
+                while (j < 4) {                         // a boundary inside the group: one run of rows per sequence
+                    seek(t0 + j);
+                    const int left = next_b - (t0 + j);
+                    const int j1 = left < 4 - j ? j + left : 4;
+                    enter();
+                    const uint32_t run = (j1 == 4 ? 0xFFFFFFFFu : (1u << (8 * j1)) - 1u) & ~((1u << (8 * j)) - 1u);
+                    const int nr = add_rows(lt, lr, mk & run);
+                    if (n_valid_seq && nr > 0) atomicAdd(&n_valid_seq[sq], nr);
+                    j = j1;
+                }
+            }
+            if (n_valid_seq) {
+                // valid rows per sequence: a warp's 128-row strip usually lies in one sequence, whose count lane 0 keeps
+                // in a register until the strip moves on (integer atomics: the result does not depend on their order)
+                const int sq0 = __shfl_sync(0xffffffffu, sq, 0);
+                if (__all_sync(0xffffffffu, single && sq == sq0)) {
+                    const int tot = __reduce_add_sync(0xffffffffu, n);
+                    if (lane == 0) {
+                        if (sq0 != wsq) {
+                            if (wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
+                            wsq = sq0;
+                            wcnt = 0;
+                        }
+                        wcnt += tot;
+                    }
+                } else if (single && n > 0) {
+                    atomicAdd(&n_valid_seq[sq], n);
+                }
+            }
+            if ((k & 15) == 15) {                       // at most 64 rows per fp32 run
+#pragma unroll
+                for (int i = 0; i < 10; ++i) { acc[i] += static_cast<double>(f[i]); f[i] = 0.f; }
+            }
+        }
+        // everyone is done with the stage (or someone gave up): the stage can take the tile four ahead
+        if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
+        if (tid == 0 && issued < tile1) { issue(issued, st); ++issued; }
+    }
+    if (failed && tid == 0) {
+        // let the copies still in flight land before the block's shared memory is given up
+        for (int k = 0; k < issued - tile0; ++k)
+            if (issued - tile0 - k <= kMomStages) mbar_wait_drain(&full[k % kMomStages], static_cast<uint32_t>((k / kMomStages) & 1));
+    }
+    if (n_valid_seq && lane == 0 && wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
+    // rows after the last whole tile: the first threads of the grid, one row each
+    {
+        const int t = ntiles * kMomRows + static_cast<int>(blockIdx.x * blockDim.x) + tid;
+        if (t < T && mask[t]) {
+            sq = -1;
+            seek(t);
+            enter();
+            const float lt[4] = {lp_train[t], 0.f, 0.f, 0.f}, lr[4] = {lp_roll[t], 0.f, 0.f, 0.f};
+            add_rows(lt, lr, 1u);
+            if (n_valid_seq) atomicAdd(&n_valid_seq[sq], 1);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 10; ++i) acc[i] += static_cast<double>(f[i]);
+    if (failed) acc[0] = __longlong_as_double(0x7ff8000000000000LL);     // a NaN count marks the batch as not reduced
+#pragma unroll
+    for (int i = 0; i < kNumMoments; ++i) {
+        const double tot = i < 10 ? block_sum(acc[i < 10 ? i : 0], scratch) : 0.0;
+        if (tid == 0) partials[blockIdx.x * kNumMoments + i] = tot;
+    }
+}
+
 __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nblocks, ais_params p, ais_diag* __restrict__ diag) {
-    // one thread per moment sums the partials in block order; thread 0 then derives the diagnostics
+    // one warp per moment sums the partials (lane l takes blocks l, l + 32, ... in order, then a fixed shuffle tree);
+    // thread 0 then derives the diagnostics
     __shared__ double m[kNumMoments];
     if (blockIdx.x != 0) return;
-    if (threadIdx.x < kNumMoments) {
+    {
+        const int i = threadIdx.x >> 5, lane = threadIdx.x & 31;
         double acc = 0.0;
-        for (int b = 0; b < nblocks; ++b) acc += partials[b * kNumMoments + threadIdx.x];
-        m[threadIdx.x] = acc;
+        for (int b = lane; b < nblocks; b += 32) acc += partials[b * kNumMoments + i];
+        acc = warp_sum(acc);
+        if (lane == 0) m[i] = acc;
     }
     __syncthreads();
     if (threadIdx.x != 0) return;
@@ -638,16 +840,20 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
         d.kl_k1 = m[8] / N;
         d.mean_abs_dp = m[9] / N;
     }
+    if (isnan(N)) d.status_flags |= AIS_FLAG_TIMEOUT;       // a block of the moments kernel gave up on a bounded wait
     d.alpha = isnan(p.alpha_override) ? d.alpha_adaptive : static_cast<double>(p.alpha_override);
     *diag = d;
 }
 
 // Sums the per-block partial moments in block order into one vector of kNumMoments doubles.
+// One warp per moment: lane l takes blocks l, l + 32, ... in order, then a fixed shuffle tree.
 __global__ void moments_reduce_kernel(const double* __restrict__ partials, int nblocks, double* __restrict__ moments) {
-    if (blockIdx.x != 0 || threadIdx.x >= kNumMoments) return;
+    if (blockIdx.x != 0) return;
+    const int i = threadIdx.x >> 5, lane = threadIdx.x & 31;
     double m = 0.0;
-    for (int b = 0; b < nblocks; ++b) m += partials[b * kNumMoments + threadIdx.x];
-    moments[threadIdx.x] = m;
+    for (int b = lane; b < nblocks; b += 32) m += partials[b * kNumMoments + i];
+    m = warp_sum(m);
+    if (lane == 0) moments[i] = m;
 }
 
 template <int VEC>
@@ -766,12 +972,16 @@ __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __
 
 __global__ void loss_finalize_kernel(const double* __restrict__ partials, int nblocks, double beta_kl, float* loss,
                                      ais_diag* diag) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    // one warp: lane l takes blocks l, l + 32, ... in order, then a fixed shuffle tree
+    if (threadIdx.x >= 32 || blockIdx.x != 0) return;
     double J = 0.0, KL = 0.0;
-    for (int b = 0; b < nblocks; ++b) {
+    for (int b = threadIdx.x; b < nblocks; b += 32) {
         J += partials[2 * b];
         KL += partials[2 * b + 1];
     }
+    J = warp_sum(J);
+    KL = warp_sum(KL);
+    if (threadIdx.x != 0) return;
     const double total = -J + beta_kl * KL;
     if (loss) *loss = static_cast<float>(total);
     if (diag) {
@@ -791,7 +1001,14 @@ void launch_moments_kernel(const float* lp_train, const float* lp_roll, const ui
                            const float* adv, int64_t T, int S, float C, double* partials, int32_t* n_valid_seq,
                            float* seq_logw, cudaStream_t stream) {
     if (seq_logw && S > 0) seq_logw_kernel<<<(S + 7) / 8, 256, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, S, seq_logw);
-    if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask))
+    if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask) && reinterpret_cast<uintptr_t>(mask) % 16 == 0 && T < (int64_t(1) << 31)) {
+        if (seq_logw)
+            moments_staged_kernel<true><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
+                                                                                  static_cast<int>(T), S, C, partials, n_valid_seq, seq_logw);
+        else
+            moments_staged_kernel<false><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
+                                                                                   static_cast<int>(T), S, C, partials, n_valid_seq, seq_logw);
+    } else if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask))
         moments_kernel<4><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials,
                                                                       n_valid_seq, seq_logw);
     else
@@ -892,7 +1109,7 @@ cudaError_t launch_diag(const float* lp_train, const float* lp_roll, const uint8
                         float* seq_logw, float* rho, float* w_tilde, ais_diag* diag, cudaStream_t stream) {
     const float C = p.C;
     launch_moments_kernel(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials, n_valid_seq, seq_logw, stream);
-    diag_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, p, diag);
+    diag_finalize_kernel<<<1, 32 * kNumMoments, 0, stream>>>(partials, kDiagBlocks, p, diag);
     if (T > 0) launch_rectify_kernel(lp_train, lp_roll, mask, T, C, diag, rho, w_tilde, seq_offsets, S, seq_logw, stream);
     return cudaGetLastError();
 }
@@ -901,14 +1118,14 @@ cudaError_t launch_moments(const float* lp_train, const float* lp_roll, const ui
                            const float* adv, int64_t T, int S, const ais_params& p, double* partials, int32_t* n_valid_seq,
                            float* seq_logw, double* moments, cudaStream_t stream) {
     launch_moments_kernel(lp_train, lp_roll, mask, seq_offsets, adv, T, S, p.C, partials, n_valid_seq, seq_logw, stream);
-    moments_reduce_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, moments);
+    moments_reduce_kernel<<<1, 32 * kNumMoments, 0, stream>>>(partials, kDiagBlocks, moments);
     return cudaGetLastError();
 }
 
 cudaError_t launch_finalize(const double* moments, const float* lp_train, const float* lp_roll, const uint8_t* mask, int64_t T,
                             const ais_params& p, float* rho, float* w_tilde, ais_diag* diag, const int32_t* seq_offsets, int S,
                             const float* seq_logw, cudaStream_t stream) {
-    diag_finalize_kernel<<<1, 32, 0, stream>>>(moments, 1, p, diag);
+    diag_finalize_kernel<<<1, 32 * kNumMoments, 0, stream>>>(moments, 1, p, diag);
     if (T > 0) launch_rectify_kernel(lp_train, lp_roll, mask, T, p.C, diag, rho, w_tilde, seq_offsets, S, seq_logw, stream);
     return cudaGetLastError();
 }
