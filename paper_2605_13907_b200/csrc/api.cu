@@ -48,7 +48,7 @@ int device_setup(int* num_sms) {
                 return info.status;
             g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
         }
-        if (lmhead_prepare() != cudaSuccess) return info.status;
+        if (lmhead_prepare() != cudaSuccess || stream_prepare() != cudaSuccess) return info.status;
         info.num_sms = prop.multiProcessorCount;
         info.status = AIS_OK;
     }

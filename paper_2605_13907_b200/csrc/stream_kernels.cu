@@ -598,21 +598,27 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
 }
 
 // The same moments for 16-byte aligned inputs, fed by bulk asynchronous copies: a block walks a contiguous range of
-// 1024-row tiles; thread 0 keeps four tiles (two log-prob vectors and the mask bytes, 9 KB each) in flight into a ring
-// of shared-memory stages, completion arrives on one mbarrier per stage, and every thread takes the four rows
-// 4 tid .. 4 tid + 3 of each tile from shared memory.  Memory latency is carried by the copies in flight (36 KB per
-// block, four blocks per SM) instead of by registers, and the per-row work is kept to about twenty instructions
-// (flush-to-zero exponentials, 32-bit row indices, the group's sequence looked up before the data arrives), because
-// at 9 bytes per row the instruction issue rate is the next limit after HBM.  Rows after the last whole tile are read
-// directly.  Summation order is fixed by the grid as above.
-constexpr int kMomRows = 1024;
-constexpr int kMomStages = 4;
+// 2048-row tiles; thread 0 keeps three tiles (two log-prob vectors and the mask bytes, 18 KB each) in flight into a
+// ring of shared-memory stages, completion arrives on one mbarrier per stage, and every thread takes the eight rows
+// 8 tid .. 8 tid + 7 of each tile from shared memory.  Memory latency is carried by the copies in flight (54 KB per
+// block, four blocks per SM) instead of by registers, and the work per row is kept to about twenty instructions
+// (flush-to-zero exponentials, 32-bit row indices, the group's sequence looked up before the data arrives, the
+// per-tile bookkeeping shared by eight rows), because at 9 bytes per row the instruction issue rate is the next limit
+// after HBM.  Rows after the last whole tile are read directly.  Summation order is fixed by the grid as above.
+constexpr int kMomRows = 2048;
+constexpr int kMomStages = 3;
 constexpr int kMomStageBytes = kMomRows * 9;
+constexpr int kMomSmemBytes = kMomStages * kMomStageBytes + 128;
 
 __device__ __forceinline__ float exp_ftz(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x * 1.4426950408889634f));
     return y;
+}
+
+// The waiting part of a bounded mbarrier wait, kept out of line so that the loop around it stays small.
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, int* abort_flag) {
+    return mbar_wait(bar, parity, abort_flag);
 }
 
 template <bool SEQ>   // SEQ: every row carries its sequence's truncated weight instead of its own
@@ -624,9 +630,9 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
                                                                          double* __restrict__ partials,
                                                                          int32_t* __restrict__ n_valid_seq,
                                                                          const float* __restrict__ seq_logw) {
-    static_assert(kDiagThreads * 4 == kMomRows, "one 4-row group per thread and tile");
-    __shared__ __align__(128) uint8_t stages[kMomStages * kMomStageBytes];
-    __shared__ uint64_t full[kMomStages];
+    static_assert(kDiagThreads * 8 == kMomRows, "one 8-row group per thread and tile");
+    extern __shared__ __align__(128) uint8_t stages[];          // kMomStages stages, then the barriers
+    uint64_t* full = reinterpret_cast<uint64_t*>(stages + kMomStages * kMomStageBytes);
     __shared__ double scratch[32];
     __shared__ int abort_flag;
     const int tid = threadIdx.x;
@@ -679,13 +685,14 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
             if (SEQ) wseq = fminf(__expf(seq_logw[sq]), C);
         }
     };
-    // sums over the rows of a group whose mask byte in `mk` is set, all in sequence `cur`; returns how many they are
-    auto add_rows = [&](const float (&lt)[4], const float (&lr)[4], uint32_t mk) -> int {
+    // sums over the rows of a group whose mask byte (rows 0..3 in `m0`, 4..7 in `m1`) is set, all of them in sequence
+    // `cur`; returns how many they are
+    auto add_rows = [&](const float (&lt)[8], const float (&lr)[8], uint32_t m0, uint32_t m1) -> int {
         int n = 0;
         float sw = 0.f, sw2 = 0.f;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const bool on = (mk & (0xFFu << (8 * j))) != 0u;
+        for (int j = 0; j < 8; ++j) {
+            const bool on = ((j < 4 ? m0 : m1) & (0xFFu << (8 * (j & 3)))) != 0u;
             const float dl = on ? lt[j] - lr[j] : 0.f;             // a masked row enters with dl = 0 and weight 0
             const float rho = exp_ftz(dl);
             const float w = on ? (SEQ ? wseq : fminf(rho, C)) : 0.f;
@@ -709,61 +716,65 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
 
     bool failed = false;
     for (int tile = tile0; tile < tile1; ++tile) {
-        const int k = tile - tile0;
-        const int st = k % kMomStages;
+        const unsigned k = static_cast<unsigned>(tile - tile0);
+        const unsigned st = k % kMomStages;
         // the group's sequence, advantage and weight source do not depend on the tile's data: fetched before the wait
-        const int t0 = tile * kMomRows + 4 * tid;
+        const int t0 = tile * kMomRows + 8 * tid;
         seek(t0);
-        const bool single = t0 + 4 <= next_b;          // the usual case: the four rows belong to one sequence
+        const bool single = t0 + 8 <= next_b;          // the usual case: the eight rows belong to one sequence
         if (single) enter();
-        // warp-uniform outcome: the warp-wide operations below need all 32 lanes
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(&full[st], static_cast<uint32_t>((k / kMomStages) & 1), &abort_flag));
+        const uint32_t parity = (k / kMomStages) & 1u;
+        bool ok = mbar_try_wait(&full[st], parity);
+        if (!ok) ok = mbar_wait_slow(&full[st], parity, &abort_flag);
+        int n = 0;
         if (ok) {
             const uint8_t* src = stages + st * kMomStageBytes;
-            const float4 a = reinterpret_cast<const float4*>(src)[tid];
-            const float4 b = reinterpret_cast<const float4*>(src + kMomRows * 4)[tid];
-            const uint32_t mk = reinterpret_cast<const uint32_t*>(src + kMomRows * 8)[tid];
-            const float lt[4] = {a.x, a.y, a.z, a.w}, lr[4] = {b.x, b.y, b.z, b.w};
-            int n = 0;
+            const float4* pa = reinterpret_cast<const float4*>(src) + 2 * tid;
+            const float4* pb = reinterpret_cast<const float4*>(src + kMomRows * 4) + 2 * tid;
+            const float4 a0 = pa[0], a1 = pa[1], b0 = pb[0], b1 = pb[1];
+            const uint2 mk = reinterpret_cast<const uint2*>(src + kMomRows * 8)[tid];
+            const float lt[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            const float lr[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
             if (single) {
-                if (mk != 0u) n = add_rows(lt, lr, mk);
-            } else if (mk != 0u) {
+                if ((mk.x | mk.y) != 0u) n = add_rows(lt, lr, mk.x, mk.y);
+            } else if ((mk.x | mk.y) != 0u) {
+                const uint64_t m64 = (static_cast<uint64_t>(mk.y) << 32) | mk.x;
                 int j = 0;
-                while (j < 4) {                         // a boundary inside the group: one run of rows per sequence
+                while (j < 8) {                         // a boundary inside the group: one run of rows per sequence
                     seek(t0 + j);
                     const int left = next_b - (t0 + j);
-                    const int j1 = left < 4 - j ? j + left : 4;
+                    const int j1 = left < 8 - j ? j + left : 8;
                     enter();
-                    const uint32_t run = (j1 == 4 ? 0xFFFFFFFFu : (1u << (8 * j1)) - 1u) & ~((1u << (8 * j)) - 1u);
-                    const int nr = add_rows(lt, lr, mk & run);
+                    const uint64_t run = (j1 == 8 ? ~uint64_t(0) : (uint64_t(1) << (8 * j1)) - 1u) & ~((uint64_t(1) << (8 * j)) - 1u);
+                    const int nr = add_rows(lt, lr, static_cast<uint32_t>(m64 & run), static_cast<uint32_t>((m64 & run) >> 32));
                     if (n_valid_seq && nr > 0) atomicAdd(&n_valid_seq[sq], nr);
                     j = j1;
                 }
             }
-            if (n_valid_seq) {
-                // valid rows per sequence: a warp's 128-row strip usually lies in one sequence, whose count lane 0 keeps
-                // in a register until the strip moves on (integer atomics: the result does not depend on their order)
-                const int sq0 = __shfl_sync(0xffffffffu, sq, 0);
-                if (__all_sync(0xffffffffu, single && sq == sq0)) {
-                    const int tot = __reduce_add_sync(0xffffffffu, n);
-                    if (lane == 0) {
-                        if (sq0 != wsq) {
-                            if (wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
-                            wsq = sq0;
-                            wcnt = 0;
-                        }
-                        wcnt += tot;
-                    }
-                } else if (single && n > 0) {
-                    atomicAdd(&n_valid_seq[sq], n);
-                }
-            }
-            if ((k & 15) == 15) {                       // at most 64 rows per fp32 run
+            if ((k & 7u) == 7u) {                       // at most 64 rows per fp32 run
 #pragma unroll
                 for (int i = 0; i < 10; ++i) { acc[i] += static_cast<double>(f[i]); f[i] = 0.f; }
             }
         }
-        // everyone is done with the stage (or someone gave up): the stage can take the tile four ahead
+        if (n_valid_seq) {
+            // valid rows per sequence: a warp's 256-row strip usually lies in one sequence, whose count lane 0 keeps in
+            // a register until the strip moves on (integer atomics: the result does not depend on their order)
+            const int sq0 = __shfl_sync(0xffffffffu, sq, 0);
+            if (__all_sync(0xffffffffu, single && sq == sq0)) {
+                const int tot = __reduce_add_sync(0xffffffffu, n);
+                if (lane == 0) {
+                    if (sq0 != wsq) {
+                        if (wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
+                        wsq = sq0;
+                        wcnt = 0;
+                    }
+                    wcnt += tot;
+                }
+            } else if (single && n > 0) {
+                atomicAdd(&n_valid_seq[sq], n);
+            }
+        }
+        // everyone is done with the stage (or someone gave up): the stage can take the tile three ahead
         if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
         if (tid == 0 && issued < tile1) { issue(issued, st); ++issued; }
     }
@@ -774,16 +785,14 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
     }
     if (n_valid_seq && lane == 0 && wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
     // rows after the last whole tile: the first threads of the grid, one row each
-    {
-        const int t = ntiles * kMomRows + static_cast<int>(blockIdx.x * blockDim.x) + tid;
-        if (t < T && mask[t]) {
-            sq = -1;
-            seek(t);
-            enter();
-            const float lt[4] = {lp_train[t], 0.f, 0.f, 0.f}, lr[4] = {lp_roll[t], 0.f, 0.f, 0.f};
-            add_rows(lt, lr, 1u);
-            if (n_valid_seq) atomicAdd(&n_valid_seq[sq], 1);
-        }
+    for (int t = ntiles * kMomRows + static_cast<int>(blockIdx.x * blockDim.x) + tid; t < T; t += gridDim.x * blockDim.x) {
+        if (!mask[t]) continue;
+        sq = -1;
+        seek(t);
+        enter();
+        const float lt[8] = {lp_train[t], 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, lr[8] = {lp_roll[t], 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        add_rows(lt, lr, 1u, 0u);
+        if (n_valid_seq) atomicAdd(&n_valid_seq[sq], 1);
     }
 #pragma unroll
     for (int i = 0; i < 10; ++i) acc[i] += static_cast<double>(f[i]);
@@ -1003,10 +1012,10 @@ void launch_moments_kernel(const float* lp_train, const float* lp_roll, const ui
     if (seq_logw && S > 0) seq_logw_kernel<<<(S + 7) / 8, 256, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, S, seq_logw);
     if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask) && reinterpret_cast<uintptr_t>(mask) % 16 == 0 && T < (int64_t(1) << 31)) {
         if (seq_logw)
-            moments_staged_kernel<true><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
+            moments_staged_kernel<true><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
                                                                                   static_cast<int>(T), S, C, partials, n_valid_seq, seq_logw);
         else
-            moments_staged_kernel<false><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
+            moments_staged_kernel<false><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
                                                                                    static_cast<int>(T), S, C, partials, n_valid_seq, seq_logw);
     } else if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask))
         moments_kernel<4><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials,
@@ -1028,6 +1037,12 @@ void launch_rectify_kernel(const float* lp_train, const float* lp_roll, const ui
 }
 
 }  // namespace
+
+cudaError_t stream_prepare() {
+    cudaError_t e = cudaFuncSetAttribute(moments_staged_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMomSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(moments_staged_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMomSmemBytes);
+}
 
 // ------------------------------------------------------------------------------------------------ launchers
 cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes,

@@ -13,6 +13,9 @@ constexpr int kDiagBlocks = 592;      // fixed grid of the batch reductions (kee
 constexpr int kDiagThreads = 256;
 constexpr int kNumMoments = 12;
 
+// Raises the dynamic shared-memory limit of the kernels here that need it (once per device).
+cudaError_t stream_prepare();
+
 cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes,
                             int64_t ldq, float* scales, int64_t lds, cudaStream_t stream);
 
