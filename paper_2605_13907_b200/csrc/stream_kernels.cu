@@ -831,8 +831,17 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
         d.alpha_adaptive = 0.0; d.kl_k1 = 0.0; d.mean_abs_dp = 0.0;
         d.status_flags |= AIS_FLAG_EMPTY;
     } else {
+        // Population variance from a sum and a sum of squares whose terms were rounded to fp32: a result below the
+        // rounding noise of those terms and of their fp32 partial sums (2^-20 of the mean square) is zero.  Without this a batch whose valid
+        // rows all share one advantage (one row, one sequence) gets std(A w) = 1e-4 |A w| instead of 0, which the
+        // eps of Delta-sigma turns into a huge variance ratio.
+        auto variance = [&](double sum, double sumsq) {
+            const double mean = sum / N, ms = sumsq / N;
+            const double v = ms - mean * mean;
+            return v > ms * 0x1p-20 ? v : 0.0;
+        };
         const double mu = m[1] / N;
-        const double var = fmax(m[2] / N - mu * mu, 0.0);
+        const double var = variance(m[1], m[2]);
         d.mean_w = mu;
         d.cv2 = var / (mu * mu);
         d.ess = m[1] * m[1] / m[2];
@@ -840,9 +849,8 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
         d.alpha_ess = 1.0 / sqrt(1.0 + d.cv2);
         d.d_bar = m[3] / N;
         d.alpha_mis = fmin(1.0, d.d_bar / static_cast<double>(p.delta));
-        const double mA = m[4] / N, mAw = m[6] / N;
-        d.std_A = sqrt(fmax(m[5] / N - mA * mA, 0.0));
-        d.std_Aw = sqrt(fmax(m[7] / N - mAw * mAw, 0.0));
+        d.std_A = sqrt(variance(m[4], m[5]));
+        d.std_Aw = sqrt(variance(m[6], m[7]));
         d.delta_sigma = d.std_Aw / (d.std_A + static_cast<double>(p.eps));
         d.alpha_var = fmax(0.0, (d.delta_sigma - static_cast<double>(p.gamma)) / static_cast<double>(p.gamma));
         d.alpha_adaptive = fmin(1.0, fmax(0.0, d.alpha_ess - static_cast<double>(p.beta_var) * d.alpha_var)) * d.alpha_mis;

@@ -62,20 +62,31 @@ def test_padded_sequences_equal_packed_sequences():
     assert np.linalg.norm(dH_padded[r].numpy().astype(np.float64) - ref["dH"]) <= 1e-2 * np.linalg.norm(ref["dH"])
 
 
-@pytest.mark.parametrize("T,shift", [(1, 0), (3, 1), (1027, 0), (1027, 1), (4101, 3)])
-def test_batch_reductions_on_unaligned_and_ragged_vectors(T, shift):
+@pytest.mark.parametrize("T,shift,S", [(1, 0, 6), (3, 1, 6), (1027, 0, 6), (1027, 1, 6), (4101, 3, 6), (4101, 0, 6),
+                                       (5 * 2048 + 77, 0, 1600), (3 * 2048, 0, 8), (20 * 2048 + 1, 0, 400)])
+def test_batch_reductions_on_unaligned_and_ragged_vectors(T, shift, S):
+    """S = 6: a few sequences with boundaries anywhere.  Larger S on aligned storage: the kernel that stages 2048-row tiles
+    in shared memory, with sequences of a few rows (several boundaries inside one thread's eight rows), empty sequences,
+    masked stretches longer than a tile and a ragged tail."""
     import paper_2605_13907_b200 as ais
-    rng = np.random.default_rng(100 + T + shift)
-    P, G = 3, 2
-    S = P * G
-    # sequence boundaries anywhere, two of the sequences empty
+    rng = np.random.default_rng(100 + T + shift + S)
+    G = 2
+    P = S // G
+    # sequence boundaries anywhere, some of the sequences empty
     cuts = np.sort(rng.integers(0, T + 1, S - 1))
     cuts[1] = cuts[0]
     cuts[-1] = T
+    if S > 100:
+        cuts[S // 2:S // 2 + 5] = cuts[S // 2]              # a run of empty sequences in the middle
     offs = np.concatenate([[0], cuts, [T]]).astype(np.int32)
     lp_t = -rng.uniform(0.1, 6.0, T).astype(np.float32)
     lp_r = (lp_t + rng.normal(0, 0.3, T)).astype(np.float32)
     mask = (rng.random(T) < 0.7).astype(np.uint8)
+    if T > 3 * 2048:
+        mask[2048 - 100:2 * 2048 + 300] = 0                 # more than one whole tile without a valid row
+        mask[T // 2] = 7                                     # any non-zero byte counts as valid
+        lp_t[2048:2048 + 8] = np.float32(-np.inf)            # masked rows may hold anything
+        lp_r[2048 + 8:2048 + 16] = np.float32(np.nan)
     rew = (rng.random(S) < 0.5).astype(np.float32)
     params = ais.default_params()
     op = oais.Params()
@@ -102,7 +113,7 @@ def test_batch_reductions_on_unaligned_and_ragged_vectors(T, shift):
     torch.cuda.synchronize()
     d = ais.Diag.from_buffer_copy(diag.cpu().numpy().tobytes()[:ctypes.sizeof(ais.Diag)]).as_dict()
     valid = mask.astype(bool)
-    counts = np.array([mask[offs[s]:offs[s + 1]].sum() for s in range(S)], np.int32)
+    counts = np.array([(mask[offs[s]:offs[s + 1]] != 0).sum() for s in range(S)], np.int32)
     assert np.array_equal(nseq.cpu().numpy(), counts)
     assert d["n_valid"] == float(valid.sum())
     for k in ("alpha", "alpha_ess", "alpha_mis", "alpha_var", "d_bar", "cv2", "delta_sigma", "mean_abs_dp", "kl_k1"):
