@@ -41,27 +41,21 @@ __device__ __forceinline__ float exact_div(float x, float s, float y) {
 // be inlined eight times into every copy of the hot loop.
 __device__ __noinline__ float slow_div(float x, float s) { return __fdiv_rn(x, s); }
 
+// amax of the block a lane belongs to, on the bf16 bit patterns: |x| is the pattern without its sign bit, and patterns
+// of non-negative values order like the values, so packed 16-bit unsigned maxima do the work of eight float compares
 template <int BLOCK>
-__device__ __forceinline__ void quantize_lane(const uint4 raw, bool in_range, int lane, float& scale_out, uint2& out) {
+__device__ __forceinline__ uint32_t block_amax_bits(const uint4 raw) {
     constexpr int kLanesPerBlock = BLOCK / 8;
-    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-    // amax on the bf16 bit patterns: |x| is the pattern without its sign bit, and patterns of non-negative
-    // values order like the values, so packed 16-bit unsigned maxima do the work of eight float compares
-    uint32_t m = __vmaxu2(__vmaxu2(w[0] & 0x7FFF7FFFu, w[1] & 0x7FFF7FFFu), __vmaxu2(w[2] & 0x7FFF7FFFu, w[3] & 0x7FFF7FFFu));
+    uint32_t m = __vmaxu2(__vmaxu2(raw.x & 0x7FFF7FFFu, raw.y & 0x7FFF7FFFu), __vmaxu2(raw.z & 0x7FFF7FFFu, raw.w & 0x7FFF7FFFu));
     m = max(m & 0xFFFFu, m >> 16);
 #pragma unroll
     for (int off = 1; off < kLanesPerBlock; off <<= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, off));
-    // the first lane of the block derives the scale and its reciprocal once and hands both to the others
-    float s = 1.0f, y = 1.0f;
-    const int leader = lane & ~(kLanesPerBlock - 1);
-    if (lane == leader && m != 0u) {
-        s = __fdiv_rn(__uint_as_float(m << 16), 448.0f);
-        y = __frcp_rn(s);
-    }
-    s = __shfl_sync(0xffffffffu, s, leader);
-    y = __shfl_sync(0xffffffffu, y, leader);
-    scale_out = s;
-    if (!in_range) return;
+    return m;
+}
+
+// Eight bf16 values divided by the block's scale s (y = RN(1 / s)) and rounded to E4M3.
+__device__ __forceinline__ uint2 quantize_values(const uint4 raw, float s, float y) {
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
     float v[8], qv[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -75,8 +69,10 @@ __device__ __forceinline__ void quantize_lane(const uint4 raw, bool in_range, in
 #pragma unroll
         for (int i = 0; i < 8; ++i) qv[i] = slow_div(v[i], s);      // rare: scale outside the safe exponent range
     }
+    uint2 out;
     out.x = static_cast<uint32_t>(cvt_e4m3x2(qv[1], qv[0])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[3], qv[2])) << 16);
     out.y = static_cast<uint32_t>(cvt_e4m3x2(qv[5], qv[4])) | (static_cast<uint32_t>(cvt_e4m3x2(qv[7], qv[6])) << 16);
+    return out;
 }
 
 template <int BLOCK>
@@ -103,15 +99,32 @@ __global__ void __launch_bounds__(kQThreads) quantize_kernel(const __nv_bfloat16
             const int64_t col = col0 + it * 256 + lane * 8;
             raw[it] = (row < rows && col < cols) ? __ldg(reinterpret_cast<const uint4*>(x + row * ld + col)) : make_uint4(0, 0, 0, 0);
         }
+        // block maxima of the row's four load rounds, then the scales of all the row's blocks at once: lane L derives
+        // scale and reciprocal of block L of the row tile (one divergent region per row instead of one per round)
+        constexpr int kBlkPerIt = 32 / kLanesPerBlock;
+        constexpr int kBlkPerRow = kQIters * kBlkPerIt;
+        static_assert(kBlkPerRow <= 32, "one lane per block of the row tile");
+        uint32_t mine = 0;
+#pragma unroll
+        for (int it = 0; it < kQIters; ++it) {
+            const uint32_t m = block_amax_bits<BLOCK>(raw[it]);
+            const uint32_t got = __shfl_sync(0xffffffffu, m, (lane % kBlkPerIt) * kLanesPerBlock);
+            if (lane / kBlkPerIt == it) mine = got;
+        }
+        float s_mine = 1.0f, y_mine = 1.0f;
+        if (lane < kBlkPerRow && mine != 0u) {
+            s_mine = __fdiv_rn(__uint_as_float(mine << 16), 448.0f);
+            y_mine = __frcp_rn(s_mine);
+        }
 #pragma unroll
         for (int it = 0; it < kQIters; ++it) {
             const int64_t col = col0 + it * 256 + lane * 8;
             const bool in = row < rows && col < cols;
-            float s;
-            uint2 out;
-            quantize_lane<BLOCK>(raw[it], in, lane, s, out);
+            const int blk = it * kBlkPerIt + lane / kLanesPerBlock;
+            const float s = __shfl_sync(0xffffffffu, s_mine, blk);
+            const float y = __shfl_sync(0xffffffffu, y_mine, blk);
             if (in) {
-                *reinterpret_cast<uint2*>(codes + row * ldq + col) = out;
+                *reinterpret_cast<uint2*>(codes + row * ldq + col) = quantize_values(raw[it], s, y);
                 if ((lane % kLanesPerBlock) == 0) sc[(it * 256 + lane * 8) / BLOCK][r_local] = s;
             }
         }
