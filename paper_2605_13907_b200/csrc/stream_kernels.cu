@@ -354,6 +354,23 @@ __device__ double block_sum(double v, double* scratch /*[32]*/) {
     return tot;
 }
 
+// Sum of partials[b * stride + offset] over b < nblocks by one warp, in a fixed order: lane l takes blocks l, l + 32, ...
+// (loaded sixteen at a time so that the loads overlap), then the shuffle tree of warp_sum.
+__device__ __forceinline__ double warp_ordered_sum(const double* __restrict__ partials, int nblocks, int stride, int offset, int lane) {
+    double acc = 0.0;
+    for (int base = lane; base < nblocks; base += 32 * 16) {
+        double v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int b = base + 32 * j;
+            v[j] = b < nblocks ? partials[b * stride + offset] : 0.0;
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc += v[j];
+    }
+    return warp_sum(acc);
+}
+
 // Valid rows of each sequence: one warp per sequence, 4 mask bytes per lane and load where the row range allows it.
 __global__ void __launch_bounds__(256) seq_count_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ seq_offsets,
                                                          int S, int32_t* __restrict__ n_valid_seq) {
@@ -818,15 +835,13 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
 }
 
 __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nblocks, ais_params p, ais_diag* __restrict__ diag) {
-    // one warp per moment sums the partials (lane l takes blocks l, l + 32, ... in order, then a fixed shuffle tree);
+    // one warp per moment sums the partials in a fixed order;
     // thread 0 then derives the diagnostics
     __shared__ double m[kNumMoments];
     if (blockIdx.x != 0) return;
     {
         const int i = threadIdx.x >> 5, lane = threadIdx.x & 31;
-        double acc = 0.0;
-        for (int b = lane; b < nblocks; b += 32) acc += partials[b * kNumMoments + i];
-        acc = warp_sum(acc);
+        const double acc = warp_ordered_sum(partials, nblocks, kNumMoments, i, lane);
         if (lane == 0) m[i] = acc;
     }
     __syncthreads();
@@ -876,13 +891,11 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
 }
 
 // Sums the per-block partial moments in block order into one vector of kNumMoments doubles.
-// One warp per moment: lane l takes blocks l, l + 32, ... in order, then a fixed shuffle tree.
+// One warp per moment, fixed order.
 __global__ void moments_reduce_kernel(const double* __restrict__ partials, int nblocks, double* __restrict__ moments) {
     if (blockIdx.x != 0) return;
     const int i = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    double m = 0.0;
-    for (int b = lane; b < nblocks; b += 32) m += partials[b * kNumMoments + i];
-    m = warp_sum(m);
+    const double m = warp_ordered_sum(partials, nblocks, kNumMoments, i, lane);
     if (lane == 0) moments[i] = m;
 }
 
@@ -1002,15 +1015,10 @@ __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __
 
 __global__ void loss_finalize_kernel(const double* __restrict__ partials, int nblocks, double beta_kl, float* loss,
                                      ais_diag* diag) {
-    // one warp: lane l takes blocks l, l + 32, ... in order, then a fixed shuffle tree
+    // one warp, fixed order
     if (threadIdx.x >= 32 || blockIdx.x != 0) return;
-    double J = 0.0, KL = 0.0;
-    for (int b = threadIdx.x; b < nblocks; b += 32) {
-        J += partials[2 * b];
-        KL += partials[2 * b + 1];
-    }
-    J = warp_sum(J);
-    KL = warp_sum(KL);
+    const double J = warp_ordered_sum(partials, nblocks, 2, 0, threadIdx.x);
+    const double KL = warp_ordered_sum(partials, nblocks, 2, 1, threadIdx.x);
     if (threadIdx.x != 0) return;
     const double total = -J + beta_kl * KL;
     if (loss) *loss = static_cast<float>(total);
