@@ -43,7 +43,8 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     constexpr int PER = 4 / SG;                     // MMAs (32 K-bytes each) per scale block
     constexpr int MODE = kFwdFp8;
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    // 1024-byte aligned start, as an offset from the array so that the compiler still knows the address space
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t* stage_base = smem;
     uint8_t* scale_base = smem + kStages * kStageBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(scale_base + C::kSlots * C::kSlotBytes);
