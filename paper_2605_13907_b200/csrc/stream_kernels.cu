@@ -1039,7 +1039,7 @@ void launch_moments_kernel(const float* lp_train, const float* lp_roll, const ui
                            const float* adv, int64_t T, int S, float C, double* partials, int32_t* n_valid_seq,
                            float* seq_logw, cudaStream_t stream) {
     if (seq_logw && S > 0) seq_logw_kernel<<<(S + 7) / 8, 256, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, S, seq_logw);
-    if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask) && reinterpret_cast<uintptr_t>(mask) % 16 == 0 && T < (int64_t(1) << 31)) {
+    if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask) && reinterpret_cast<uintptr_t>(mask) % 16 == 0 && T < (int64_t(1) << 31) - 2 * kMomRows) {      // 32-bit row indices inside
         if (seq_logw)
             moments_staged_kernel<true><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
                                                                                   static_cast<int>(T), S, C, partials, n_valid_seq, seq_logw);
