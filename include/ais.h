@@ -100,7 +100,11 @@ typedef struct ais_params {
                              Eq. ais-components instead; d_bar and rho stay per token.                  */
 } ais_params;
 
-/* Everything the reductions produce; lives in DEVICE memory, the caller copies it back. */
+/* Everything the reductions produce; lives in DEVICE memory, the caller copies it back.
+ * The three variances (cv2, std_A, std_Aw) are E[x^2] - E[x]^2 over fp64 sums of terms rounded to fp32; a value
+ * below that rounding noise (2^-20 of the mean square) is reported as exactly 0, so that a batch whose valid rows all
+ * share one advantage and one weight (one valid row, say) gives delta_sigma = 0 and not noise / eps.
+ * status_flags carries AIS_FLAG_EMPTY for N = 0 and AIS_FLAG_TIMEOUT if a bounded wait of the moments kernel ran out. */
 typedef struct ais_diag {
     double n_valid;       /* N = number of rows with mask 1                                  */
     double mean_w;        /* mean of w_bar = min(rho, C)                                     */
