@@ -162,3 +162,50 @@ def test_sequence_level_weights_on_gpu():
     for k in ("alpha", "cv2", "d_bar", "delta_sigma", "n_valid"):
         assert d2[k] == fused[0][k], k
     assert torch.equal(step.w_tilde, fused[1])
+
+
+def test_sequence_level_reductions_over_several_tiles():
+    """The sequence-level variant of the batch reductions on a batch long enough for the kernel that stages 2048-row
+    tiles in shared memory (the end-to-end test of the variant above is smaller than one tile): split pair
+    ais_diag_moments / ais_diag_finalize against the oracle's sequence-level weights."""
+    import paper_2605_13907_b200 as ais
+    rng = np.random.default_rng(4242)
+    T, S, G = 4 * 2048 + 321, 60, 4
+    P = S // G
+    cuts = np.sort(rng.integers(0, T + 1, S - 1))
+    cuts[7] = cuts[6]                                         # an empty sequence
+    offs = np.concatenate([[0], cuts, [T]]).astype(np.int32)
+    lp_t = -rng.uniform(0.1, 6.0, T).astype(np.float32)
+    lp_r = (lp_t + rng.normal(0, 0.02, T)).astype(np.float32)  # small per-token gaps: the sequence products stay moderate
+    mask = (rng.random(T) < 0.8).astype(np.uint8)
+    rew = (rng.random(S) < 0.5).astype(np.float32)
+    op = oais.Params(seq_level=True)
+    ref_adv = oais.advantages(rew.astype(np.float64), G)
+    ref_logw, ref_wbar = oais.ratios_sequence(lp_t, lp_r, mask, offs, op.C)
+    ref = oais.diagnostics(lp_t, lp_r, mask, ref_adv[oais.seq_ids(offs, T)], op, wbar_rows=ref_wbar)
+    ref_wt = oais.rectify(ref_wbar, ref["alpha"], mask)
+
+    params = ais.default_params(seq_level_weights=1)
+    shape = ais.make_shape(T, 128, 1024, P, G, 128)
+    ws = torch.empty(ais.workspace_min_bytes(shape, params), dtype=torch.uint8, device="cuda")
+    c = lambda x: torch.from_numpy(x).cuda()
+    d_lp_t, d_lp_r, d_mask, d_offs = c(lp_t), c(lp_r), c(mask), c(offs)
+    adv = torch.empty(S, device="cuda")
+    nseq = torch.full((S,), -1, dtype=torch.int32, device="cuda")
+    logw = torch.zeros(S, device="cuda")
+    moments = torch.zeros(16, dtype=torch.float64, device="cuda")
+    rho, wt = torch.zeros(T, device="cuda"), torch.zeros(T, device="cuda")
+    diag = torch.zeros(32, dtype=torch.float64, device="cuda")
+    ais.diag_moments(shape, params, d_lp_t, d_lp_r, d_mask, d_offs, c(rew), adv, nseq, moments, ws, seq_logw=logw)
+    ais.diag_finalize(shape, params, moments, d_lp_t, d_lp_r, d_mask, rho, wt, diag, seq_offsets=d_offs, seq_logw=logw)
+    torch.cuda.synchronize()
+    d = ais.Diag.from_buffer_copy(diag.cpu().numpy().tobytes()[:ctypes.sizeof(ais.Diag)]).as_dict()
+    valid = mask.astype(bool)
+    counts = np.array([(mask[offs[s]:offs[s + 1]] != 0).sum() for s in range(S)], np.int32)
+    assert np.array_equal(nseq.cpu().numpy(), counts)
+    assert np.allclose(logw.cpu().numpy(), ref_logw, rtol=1e-5, atol=1e-5)
+    assert d["n_valid"] == float(valid.sum())
+    for k in ("alpha", "alpha_ess", "alpha_mis", "alpha_var", "d_bar", "cv2", "delta_sigma", "mean_abs_dp", "kl_k1"):
+        assert abs(d[k] - ref[k]) <= 1e-4 * max(1.0, abs(ref[k])), (k, d[k], ref[k])
+    got_wt = wt.cpu().numpy()
+    assert np.allclose(got_wt[valid], ref_wt[valid], rtol=1e-4, atol=1e-5) and np.all(got_wt[~valid] == 1)
