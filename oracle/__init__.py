@@ -15,8 +15,10 @@ ais       log-probabilities, importance ratios, GRPO advantages, the three
           AIS-GRPO objective)
 
 Parity status: every function in both modules is pinned by the CPU tests
-(closed forms, brute force, finite differences, an independent float8 library
-used as a black box).  Nothing is "parity unpinned".
+(closed forms and hand numbers, brute force, finite differences, an independent
+float8 library used as a black box), the monitor outputs kl_k1 / mean_abs_dp of
+ais.diagnostics included.  Nothing is "parity unpinned".  The oracle returns
+plain arrays only; byte layouts of the C ABI are not its business.
 """
 
 from . import e4m3, ais  # noqa: F401

@@ -192,24 +192,6 @@ def dequantize_mx(codes, scale_codes) -> np.ndarray:
     return out.reshape(R, K)
 
 
-def pack_mx_scales(scale_codes, row_pad: int = 256) -> np.ndarray:
-    """Layout of the scale codes that the GPU kernels exchange: chunks of 128 rows x 4 blocks (512 bytes) with byte
-    (r % 32) * 16 + ((r % 128) // 32) * 4 + (kb % 4) holding the code of row r, block kb; the two chunks of a
-    256-row group sit side by side: chunk (r // 128, kb // 4) starts at
-    ((r // 256) * (K // 128) + kb // 4) * 1024 + ((r % 256) // 128) * 512.  Rows are padded to a multiple of 256
-    with code 127.  This is the order in which the block-scaled tensor-core instruction wants one stage's scales
-    in tensor memory; it only permutes bytes.  Returns uint8 [rows_padded // 256, K // 128, 2, 512]."""
-    sc = np.asarray(scale_codes, dtype=np.uint8)
-    R, NB = sc.shape
-    if NB % 4 or row_pad % 256:
-        raise ValueError("blocks per row must be a multiple of 4 and the row padding a multiple of 256")
-    Rp = (R + row_pad - 1) // row_pad * row_pad
-    full = np.full((Rp, NB), 127, np.uint8)
-    full[:R] = sc
-    v = full.reshape(Rp // 256, 2, 4, 32, NB // 4, 4)       # [group, half, r1, r0, chunk col, kb]
-    return np.ascontiguousarray(v.transpose(0, 4, 1, 3, 2, 5)).reshape(Rp // 256, NB // 4, 2, 512)
-
-
 # --------------------------------------------------------------------------- microscaling FP4 (E2M1 elements)
 _E2M1_VALUES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
 _FP4_EMAX = 2             # 6 = 1.5 * 2^2
@@ -262,9 +244,3 @@ def dequantize_mxfp4(codes, scale_codes) -> np.ndarray:
     R, K = codes.shape
     vals = decode_e2m1(codes).reshape(R, K // MX_BLOCK, MX_BLOCK)
     return np.ldexp(vals, np.asarray(scale_codes, dtype=np.int64)[:, :, None] - 127).reshape(R, K)
-
-
-def pack_fp4_pairs(codes) -> np.ndarray:
-    """Two 4-bit codes per byte, the element with the lower index in the low nibble."""
-    c = np.asarray(codes, dtype=np.uint8)
-    return (c[..., 0::2] | (c[..., 1::2] << 4)).astype(np.uint8)

@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+import abi_layout
 import workloads
 from oracle import ais as oais
 from oracle import e4m3
@@ -36,9 +37,10 @@ def test_mx_quantiser_bit_exact():
     torch.cuda.synchronize()
     ref_c, ref_s = e4m3.quantize_mx(xb.float().numpy())
     assert np.array_equal(codes.cpu().numpy(), ref_c)
-    ref_p = e4m3.pack_mx_scales(ref_s)
-    assert packed.numel() == ref_p.size == ais.mx_scale_bytes(rows, cols)
-    assert np.array_equal(packed.cpu().numpy().reshape(ref_p.shape), ref_p)
+    assert packed.numel() == abi_layout.mx_scale_bytes(rows, cols) == ais.mx_scale_bytes(rows, cols)
+    got = packed.cpu().numpy()
+    assert np.array_equal(abi_layout.unpack_mx_scales(got, rows, cols), ref_s)
+    assert np.all(abi_layout.mx_scale_padding(got, rows, cols) == 127)
 
 
 @pytest.mark.parametrize("case", ["tiny", "ragged"])
@@ -56,8 +58,8 @@ def test_mx_rollout_path(case):
     T = b.T
     assert int(step.status.item()) == 0
     assert np.array_equal(step.qH.cpu().numpy()[:T], ref["qH"]) and np.array_equal(step.qW.cpu().numpy(), ref["qW"])
-    assert np.array_equal(step.sW.cpu().numpy(), e4m3.pack_mx_scales(ref["sW"]).reshape(-1))
-    assert np.array_equal(step.sH.cpu().numpy(), e4m3.pack_mx_scales(ref["sH"]).reshape(-1))
+    assert np.array_equal(abi_layout.unpack_mx_scales(step.sW.cpu().numpy(), w.V, w.d), ref["sW"])
+    assert np.array_equal(abi_layout.unpack_mx_scales(step.sH.cpu().numpy(), T, w.d), ref["sH"])
     err = np.abs(step.lp_roll.cpu().numpy()[:T] - ref["lp_roll"])
     assert err.max() <= LP_ATOL, err.max()
     assert err.max() <= 1e-4                                 # power-of-two scales are exact: only fp32 accumulation differs
@@ -78,7 +80,7 @@ def test_mx_fullsize_sampled_rows(fmt):
     fp4 = fmt == "fp4"
     quant = e4m3.quantize_mxfp4 if fp4 else e4m3.quantize_mx
     dequant = e4m3.dequantize_mxfp4 if fp4 else e4m3.dequantize_mx
-    stored = e4m3.pack_fp4_pairs if fp4 else (lambda c: c)
+    plain = abi_layout.unpack_fp4_pairs if fp4 else (lambda c: c)
     w = workloads.scaled(workloads.WORKLOADS["qwen3_8b"], block=ais.FP4_MX32 if fp4 else ais.FP8_MX32)
     batch = workloads.make_batch(w, device="cuda")
     T = batch.T
@@ -90,23 +92,20 @@ def test_mx_fullsize_sampled_rows(fmt):
     rows = np.unique(np.concatenate([[0, 127, 128, T - 1, (T // 128) * 128 - 1, (T // 128) * 128], rng.integers(0, T, 42)]))
     Hs = batch.H[torch.as_tensor(rows, device="cuda")].float().cpu().numpy().astype(np.float64)
     qHs, sHs = quant(Hs)
-    assert np.array_equal(step.qH.cpu().numpy()[rows], stored(qHs))
+    assert np.array_equal(plain(step.qH.cpu().numpy()[rows]), qHs)
     Hq = dequant(qHs, sHs)
-    sH_gpu = step.sH.cpu().numpy().reshape(-1, w.d // 128, 2, 512)
-    for i, r in enumerate(rows):
-        for kb in (0, 1, 63, 127):
-            assert sH_gpu[r // 256, kb // 4, (r % 256) // 128, (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4] == sHs[i, kb]
+    sH_gpu = abi_layout.unpack_mx_scales(step.sH.cpu().numpy(), T, w.d)
+    assert np.array_equal(sH_gpu[rows], sHs)
     qW_gpu = step.qW.cpu().numpy()
-    sW_gpu = step.sW.cpu().numpy().reshape(-1, w.d // 128, 2, 512)
+    sW_gpu = abi_layout.unpack_mx_scales(step.sW.cpu().numpy(), w.V, w.d)
     z = np.empty((len(rows), w.V))
     CH = 4096                                               # a multiple of 256: whole scale groups per piece
     for v0 in range(0, w.V, CH):
         Wc = batch.W[v0:v0 + CH].float().cpu().numpy().astype(np.float64)
         qc, sc = quant(Wc)
-        assert np.array_equal(qW_gpu[v0:v0 + CH], stored(qc)), v0
+        assert np.array_equal(plain(qW_gpu[v0:v0 + CH]), qc), v0
         n = Wc.shape[0]
-        packed = e4m3.pack_mx_scales(sc)
-        assert np.array_equal(sW_gpu[v0 // 256:v0 // 256 + packed.shape[0]], packed), v0
+        assert np.array_equal(sW_gpu[v0:v0 + n], sc), v0
         z[:, v0:v0 + n] = Hq @ dequant(qc, sc).T
     tok = batch.tokens.cpu().numpy()[rows]
     msk = batch.mask.cpu().numpy()[rows]
@@ -131,8 +130,10 @@ def test_mxfp4_quantiser_bit_exact():
     torch.cuda.synchronize()
     ref_c, ref_s = e4m3.quantize_mxfp4(xb.float().numpy())
     assert codes.shape == (rows, cols // 2)
-    assert np.array_equal(codes.cpu().numpy(), e4m3.pack_fp4_pairs(ref_c))
-    assert np.array_equal(packed.cpu().numpy(), e4m3.pack_mx_scales(ref_s).reshape(-1))
+    assert np.array_equal(abi_layout.unpack_fp4_pairs(codes.cpu().numpy()), ref_c)
+    got = packed.cpu().numpy()
+    assert np.array_equal(abi_layout.unpack_mx_scales(got, rows, cols), ref_s)
+    assert np.all(abi_layout.mx_scale_padding(got, rows, cols) == 127)
 
 
 @pytest.mark.parametrize("case", ["tiny", "ragged"])
@@ -151,9 +152,9 @@ def test_mxfp4_rollout_path(case):
     ref = oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, oais.MXFP4)
     T = b.T
     assert int(step.status.item()) == 0
-    assert np.array_equal(step.qH.cpu().numpy()[:T], e4m3.pack_fp4_pairs(ref["qH"]))
-    assert np.array_equal(step.qW.cpu().numpy(), e4m3.pack_fp4_pairs(ref["qW"]))
-    assert np.array_equal(step.sW.cpu().numpy(), e4m3.pack_mx_scales(ref["sW"]).reshape(-1))
+    assert np.array_equal(abi_layout.unpack_fp4_pairs(step.qH.cpu().numpy()[:T]), ref["qH"])
+    assert np.array_equal(abi_layout.unpack_fp4_pairs(step.qW.cpu().numpy()), ref["qW"])
+    assert np.array_equal(abi_layout.unpack_mx_scales(step.sW.cpu().numpy(), w.V, w.d), ref["sW"])
     err = np.abs(step.lp_roll.cpu().numpy()[:T] - ref["lp_roll"])
     assert err.max() <= 1e-3, err.max()
     d = step.read_diag()

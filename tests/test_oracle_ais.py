@@ -184,6 +184,39 @@ def test_masked_tokens_are_ignored():
     assert empty["alpha"] == 0.0 and empty["n_valid"] == 0
 
 
+def test_monitor_outputs_hand_numbers_and_direction():
+    """kl_k1 = mean(log pi_roll - log pi_train) over the valid rows, the sample estimate of KL(pi_roll || pi_train)
+    on tokens drawn from the rollout policy, and mean_abs_dp = mean |pi_train - pi_roll| of the sampled tokens
+    (caption of the training-behaviour figure).  Hand numbers from tests/golden/diag_closed_forms.txt; a swap of
+    the two arguments or a flipped sign changes the asymmetric case; masked rows hold garbage."""
+    g = _golden()
+    one = np.ones(2, np.uint8)
+    d = ais.diagnostics(np.log([0.5, 0.25]), np.log([0.25, 0.5]), one, np.ones(2), P0)
+    assert d["mean_abs_dp"] == pytest.approx(g[("monitor_swap", "mean_abs_dp")], abs=1e-15)
+    assert d["kl_k1"] == pytest.approx(g[("monitor_swap", "kl_k1")], abs=1e-15)
+    lt = np.array([math.log(0.5), 7.0, math.log(0.5), -50.0])
+    lr = np.array([math.log(0.25), -3.0, math.log(0.125), 2.0])
+    d = ais.diagnostics(lt, lr, np.array([1, 0, 1, 0], np.uint8), np.ones(4), P0)
+    assert d["mean_abs_dp"] == pytest.approx(g[("monitor_down", "mean_abs_dp")], abs=1e-15)
+    assert d["kl_k1"] == pytest.approx(g[("monitor_down", "kl_k1")], abs=1e-15)
+    assert d["kl_k1"] < 0
+
+
+def test_kl_monitor_equals_the_textbook_divergence_on_an_exact_sample():
+    """Tokens that occur exactly in proportion to pi_roll make the sample mean the expectation: kl_k1 then equals
+    sum_v pi_roll(v) log(pi_roll(v) / pi_train(v)) -- the divergence from the rollout to the trainer, not the other
+    direction -- and mean_abs_dp equals sum_v pi_roll(v) |pi_train(v) - pi_roll(v)|."""
+    p_roll = np.array([0.5, 0.25, 0.125, 0.125])
+    p_train = np.array([0.1, 0.2, 0.3, 0.4])
+    tok = np.array([0, 0, 0, 0, 1, 1, 2, 3])                 # counts 4 : 2 : 1 : 1 = pi_roll
+    d = ais.diagnostics(np.log(p_train[tok]), np.log(p_roll[tok]), np.ones(8, np.uint8), np.ones(8), P0)
+    kl_roll_train = math.fsum(q * math.log(q / p) for q, p in zip(p_roll, p_train))
+    kl_train_roll = math.fsum(p * math.log(p / q) for q, p in zip(p_roll, p_train))
+    assert d["kl_k1"] == pytest.approx(kl_roll_train, rel=1e-13)
+    assert abs(d["kl_k1"] - kl_train_roll) > 0.05 and kl_roll_train > 0
+    assert d["mean_abs_dp"] == pytest.approx(math.fsum(q * abs(p - q) for q, p in zip(p_roll, p_train)), rel=1e-13)
+
+
 # ------------------------------------------------------------------ advantages
 def test_advantages():
     r = np.array([1, 0, 0, 1, 1, 1, 1, 1, 0, 0, 0, 0], dtype=np.float64)

@@ -271,16 +271,30 @@ def test_mx_error_bound():
     assert np.all(q < 512)                                   # the shared exponent never lets an element reach 512
 
 
-def test_mx_scale_packing_positions():
-    """Chunk (r // 128, kb // 4) at [r // 256, kb // 4, (r % 256) // 128], byte (r % 32) * 16 + ((r % 128) // 32) * 4
-    + kb % 4 inside it; padding rows hold 127."""
-    R, NB = 300, 8
-    sc = (np.arange(R)[:, None] * 7 + np.arange(NB)[None, :] * 3) % 250
-    p = e4m3.pack_mx_scales(sc.astype(np.uint8))
-    assert p.shape == (2, 2, 2, 512)
-    for r, kb in [(0, 0), (31, 3), (32, 0), (127, 7), (128, 4), (199, 5), (256, 1), (299, 6)]:
-        assert p[r // 256, kb // 4, (r % 256) // 128, (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4] == sc[r, kb]
-    assert p[1, 0, 0, (310 % 32) * 16 + ((310 % 128) // 32) * 4] == 127
+def test_abi_layout_reader_against_a_scalar_walk():
+    """The test-side reader of the packed scale bytes (tests/abi_layout.py) against a byte-by-byte walk of the order
+    the C header describes: 512-byte chunks of 128 rows x 4 blocks, inside a chunk 32 row slots of 16 bytes, each
+    slot holding the four 32-row quarters of the chunk with their four block bytes; the two chunks of a 256-row
+    group adjacent; chunk columns of a group one after the other; groups one after the other."""
+    import abi_layout
+    R, K = 300, 256                                          # two row groups (the second ragged), two chunk columns
+    NB = K // 32
+    sc = ((np.arange(R)[:, None] * 7 + np.arange(NB)[None, :] * 3) % 250).astype(np.uint8)
+    buf = []
+    for group in range((R + 255) // 256):
+        for chunk_col in range(NB // 4):
+            for half in range(2):
+                for slot in range(32):
+                    for quarter in range(4):
+                        for j in range(4):
+                            r = group * 256 + half * 128 + quarter * 32 + slot
+                            buf.append(int(sc[r, chunk_col * 4 + j]) if r < R else 127)
+    buf = np.array(buf, np.uint8)
+    assert buf.size == abi_layout.mx_scale_bytes(R, K)
+    assert np.array_equal(abi_layout.unpack_mx_scales(buf, R, K), sc)
+    pad = abi_layout.mx_scale_padding(buf, R, K)
+    assert pad.size == (512 - R) * NB and np.all(pad == 127)
+    assert np.array_equal(abi_layout.unpack_fp4_pairs(np.array([[0x21, 0x0F]], np.uint8)), [[1, 2, 15, 0]])
 
 
 # --------------------------------------------------------------------------- microscaling FP4 (E2M1)
@@ -327,4 +341,3 @@ def test_mxfp4_shared_exponent_and_round_trip():
     x = np.ldexp(e4m3.decode_e2m1(codes).reshape(6, 3, 32), k[:, :, None]).reshape(6, 96)
     c, s = e4m3.quantize_mxfp4(x)
     assert np.array_equal(s.astype(np.int64), k + 127) and np.array_equal(e4m3.dequantize_mxfp4(c, s), x)
-    assert np.array_equal(e4m3.pack_fp4_pairs(np.array([[1, 2, 15, 0]], np.uint8)), [[0x21, 0x0F]])
