@@ -13,7 +13,10 @@
  * -----------
  *  - Every data pointer is a DEVICE pointer owned by the caller unless it says "host".  The library
  *    never allocates or frees device memory; scratch comes from the caller's `workspace`
- *    (256-byte aligned, at least ais_workspace_bytes() bytes).
+ *    (256-byte aligned, at least ais_workspace_bytes() bytes).  The one exception is
+ *    ais_logprob_train_static at the end of this header: it takes no workspace, keeps its scratch in an
+ *    array inside the library image, has its own (looser) size and alignment rules, a row limit, and
+ *    calls to it must not overlap on the GPU.
  *  - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it; they never
  *    synchronise the device.  Calls on one stream are ordered; calls that share a workspace must not
  *    overlap on the GPU.
@@ -55,7 +58,11 @@ extern "C" {
 /* bits of a device status word / ais_diag.status_flags */
 #define AIS_FLAG_EMPTY        1u   /* no valid token in the batch: alpha = 0, loss = 0      */
 #define AIS_FLAG_TOKEN_RANGE  2u   /* a valid row has a token id outside [0, V): lp = 0     */
-#define AIS_FLAG_NONFINITE    4u   /* a log-prob of a valid row is not finite               */
+#define AIS_FLAG_NONFINITE    4u   /* a log-prob of a valid row is not finite (a NaN or an infinity
+                                      in its hidden state or in W): that row gets lp = 0 and
+                                      lse = NaN, which makes ais_loss_bwd leave it out of the loss
+                                      and give it a zero row of dH; the batch statistics count it
+                                      as a row with lp_train = lp_roll                        */
 #define AIS_FLAG_TIMEOUT      8u   /* a bounded device-side wait ran out; outputs undefined */
 
 #define AIS_FP8_MX32 (-32)        /* ais_shape.fp8_block: microscaling FP8, E8M0 scale per 32 elements */
@@ -101,9 +108,10 @@ typedef struct ais_params {
 } ais_params;
 
 /* Everything the reductions produce; lives in DEVICE memory, the caller copies it back.
- * The three variances (cv2, std_A, std_Aw) are E[x^2] - E[x]^2 over fp64 sums of terms rounded to fp32; a value
- * below that rounding noise (2^-20 of the mean square) is reported as exactly 0, so that a batch whose valid rows all
- * share one advantage and one weight (one valid row, say) gives delta_sigma = 0 and not noise / eps.
+ * The three variances (cv2, std_A, std_Aw) are E[x^2] - E[x]^2 in fp64 over sums that are accurate relative to the
+ * spread of the data (short runs are summed about one of their own values), so weights that differ by 1e-4 of their
+ * size still give the right variance; what is left is the rounding of the fp64 additions, and a variance below
+ * 2^-44 of the mean square is reported as exactly 0.
  * status_flags carries AIS_FLAG_EMPTY for N = 0 and AIS_FLAG_TIMEOUT if a bounded wait of the moments kernel ran out. */
 typedef struct ais_diag {
     double n_valid;       /* N = number of rows with mask 1                                  */
@@ -130,6 +138,14 @@ typedef struct ais_diag {
 
 int ais_version(void);
 const char* ais_strerror(int status);
+
+/* Bound of every device-side wait of the tensor-core passes, in SM clock ticks (a producer waiting for a free stage,
+ * the MMA issuer for operands, an epilogue warp for an accumulator).  0 restores the default of 4e9 ticks, about two
+ * seconds; a wait that runs out ends its kernel in an orderly way (copies in flight are awaited, tensor memory is
+ * freed) with AIS_FLAG_TIMEOUT in the call's dev_status and undefined outputs, and the next call works normally.
+ * Process-wide, read by every later call; meant for watchdog tuning and for testing the time-out path (a bound of a
+ * few ticks makes the first wait of a pass run out).  Returns AIS_ERR_PARAM for a negative value. */
+int ais_set_wait_cycles(int64_t cycles);
 
 /* Fills *p with the defaults listed above (alpha_override = NaN). `p` is a host pointer. */
 void ais_default_params(ais_params* p);
@@ -323,8 +339,12 @@ int ais_scatter_words(const void* src, const int32_t* row_index, int64_t n, void
  *   - T must not exceed AIS_STATIC_MAX_ROWS; a larger T returns AIS_ERR_LIMIT and enqueues nothing.
  *   - shape->d must be a multiple of 64 and V of 8; P, G and fp8_block are not read.  The vocabulary
  *     is always streamed in 4 ranges.
- *   - The first call on each device resolves the array's device address and prepares the kernels; make
- *     that first call with the device current and before any stream capture begins.
+ *   - The first call on each device resolves the array's device address and prepares the kernels; that is
+ *     also the moment at which the CUDA runtime may load this part of the library onto the device, and the
+ *     1.5 MiB array comes with it.  So the device does take that memory once, at the first call, not at a
+ *     later one: make the first call at start-up, with the device current and before any stream capture
+ *     begins.  If that first call fails for lack of resources it can simply be repeated; only a device of
+ *     the wrong architecture is remembered as unusable.
  *   - All calls on a device share the one array, which keeps what the last call left in it.  Each call
  *     overwrites every slot it later reads, so nothing has to be cleared; but two calls that overlap on
  *     the GPU (different streams, no ordering between them) race on it and give undefined results.

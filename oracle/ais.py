@@ -276,28 +276,27 @@ def kl_term(lp_theta, lp_ref, mask, seq_offsets, P: int, G: int) -> float:
     return float(np.sum(np.where(valid, kl / (P * G * n_tok), 0.0)))
 
 
-def grad_hidden(H, W, tokens, c) -> np.ndarray:
-    """dH[t, :] = c_t (softmax(z_t) - onehot(y_t)) W   in float64."""
-    z = logits(H, W)
+def logit_gradient(z, tokens, c) -> np.ndarray:
+    """d loss / d z[t, :] = c_t (softmax(z_t) - onehot(y_t)): the gradient of -c_t log softmax(z_t)[y_t], the form every
+    term of the objective takes once w_tilde, A and lp_old are held constant."""
+    z = np.asarray(z, dtype=np.float64)
     z = z - z.max(axis=1, keepdims=True)
     p = np.exp(z)
     p /= p.sum(axis=1, keepdims=True)
     T = z.shape[0]
     p[np.arange(T), np.asarray(tokens, np.int64)] -= 1.0
     p *= np.asarray(c, np.float64)[:, None]
-    return p @ np.asarray(W, np.float64)
+    return p
+
+
+def grad_hidden(H, W, tokens, c) -> np.ndarray:
+    """dH[t, :] = c_t (softmax(z_t) - onehot(y_t)) W   in float64."""
+    return logit_gradient(logits(H, W), tokens, c) @ np.asarray(W, np.float64)
 
 
 def grad_weight(H, W, tokens, c) -> np.ndarray:
     """dW[v, :] = sum_t c_t (softmax(z_t)[v] - [v = y_t]) H[t, :]   in float64 (same layout as W: [V, d])."""
-    z = logits(H, W)
-    z = z - z.max(axis=1, keepdims=True)
-    p = np.exp(z)
-    p /= p.sum(axis=1, keepdims=True)
-    T = z.shape[0]
-    p[np.arange(T), np.asarray(tokens, np.int64)] -= 1.0
-    p *= np.asarray(c, np.float64)[:, None]
-    return p.T @ np.asarray(H, np.float64)
+    return logit_gradient(logits(H, W), tokens, c).T @ np.asarray(H, np.float64)
 
 
 # --------------------------------------------------------------------------- whole path

@@ -94,10 +94,17 @@ def lib() -> C.CDLL:
         L.ais_gather_words.argtypes = [vp, vp, i64, vp, vp]
         L.ais_scatter_words.restype = C.c_int
         L.ais_scatter_words.argtypes = [vp, vp, i64, vp, i64, C.c_uint32, vp]
+        L.ais_set_wait_cycles.restype = C.c_int
+        L.ais_set_wait_cycles.argtypes = [i64]
         L.ais_logprob_train_static.restype = C.c_int
         L.ais_logprob_train_static.argtypes = [C.POINTER(Shape)] + [vp] * 8
         _lib = L
     return _lib
+
+
+def set_wait_cycles(cycles: int) -> None:
+    """Bound of the kernels' device-side waits in SM clock ticks; 0 restores the default (about two seconds)."""
+    _check(lib().ais_set_wait_cycles(int(cycles)), "ais_set_wait_cycles")
 
 
 def _check(status: int, what: str) -> None:

@@ -11,7 +11,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libais_b200.so")
 SOURCES = ["api.cu", "lmhead.cu", "lmhead_fp8.cu", "stream_kernels.cu", "noalloc.cu", "compact.cu"]
-HEADERS = ["lmhead.cuh", "lmhead_common.cuh", "ptx.cuh", "stream_kernels.cuh", os.path.join("..", "..", "include", "ais.h")]
+HEADERS = ["host_setup.cuh", "lmhead.cuh", "lmhead_common.cuh", "ptx.cuh", "stream_kernels.cuh", os.path.join("..", "..", "include", "ais.h")]
 
 
 def _nvcc() -> str:

@@ -7,70 +7,85 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "../../include/ais.h"
+#include "host_setup.cuh"
 #include "lmhead.cuh"
 #include "stream_kernels.cuh"
 
+namespace ais {
+
 namespace {
-
-using namespace ais;
-
 constexpr int kMaxDevices = 64;
 struct DeviceInfo {
-    bool ready = false;
-    int status = AIS_OK;
+    bool ready = false;      // set-up succeeded on this device
+    bool wrong_arch = false; // not an sm_100 device: remembered, every later call fails at once
     int num_sms = 0;
 };
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_mutex;
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+std::atomic<long long> g_wait_cycles{0};
+}  // namespace
 
-// Per-device set-up, done once: checks the architecture, raises the kernels' dynamic shared-memory limit
-// and resolves the driver's tensor-map encoder.
+int64_t wait_cycles() { return g_wait_cycles.load(); }
+
+// Per-device set-up, done once per device with that device current: checks the architecture, raises the kernels'
+// dynamic shared-memory limit and resolves the driver's tensor-map encoder.  Only the architecture check is
+// remembered as a failure; any other failed step (a CUDA call that could not get resources, say) is tried again
+// by the next call.
 int device_setup(int* num_sms) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AIS_ERR_DEVICE;
     std::lock_guard<std::mutex> lock(g_mutex);
     DeviceInfo& info = g_dev[dev];
+    if (info.wrong_arch) return AIS_ERR_DEVICE;
     if (!info.ready) {
-        info.ready = true;
-        info.status = AIS_ERR_DEVICE;
         cudaDeviceProp prop;
-        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return info.status;
-        if (prop.major != 10) return info.status;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return AIS_ERR_DEVICE;
+        if (prop.major != 10) {
+            info.wrong_arch = true;
+            return AIS_ERR_DEVICE;
+        }
         if (!g_encode) {
             void* fn = nullptr;
             cudaDriverEntryPointQueryResult qres;
             if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
                 qres != cudaDriverEntryPointSuccess || !fn)
-                return info.status;
+                return AIS_ERR_DEVICE;
             g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
         }
-        if (lmhead_prepare() != cudaSuccess || stream_prepare() != cudaSuccess) return info.status;
+        if (lmhead_prepare() != cudaSuccess || stream_prepare() != cudaSuccess) return AIS_ERR_DEVICE;
         info.num_sms = prop.multiProcessorCount;
-        info.status = AIS_OK;
+        info.ready = true;
     }
     if (num_sms) *num_sms = info.num_sms;
-    return info.status;
+    return AIS_OK;
 }
 
-inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
-
 // 2-D row-major tensor map: dim0 is the contiguous axis.
-bool make_tmap(CUtensorMap* map, CUtensorMapDataType dtype, int elem_bytes, const void* base, uint64_t dim0, uint64_t dim1,
+bool make_tmap(CUtensorMap* map, CUtensorMapDataType dtype, const void* base, uint64_t dim0, uint64_t dim1,
                uint64_t stride1_bytes, uint32_t box0, uint32_t box1, CUtensorMapSwizzle swz) {
+    if (!g_encode) return false;
     cuuint64_t dims[2] = {dim0, dim1};
     cuuint64_t strides[1] = {stride1_bytes};
     cuuint32_t box[2] = {box0, box1};
     cuuint32_t estr[2] = {1, 1};
-    (void)elem_bytes;
     CUresult r = g_encode(map, dtype, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
+
+}  // namespace ais
+
+namespace {
+
+using namespace ais;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 int check_shape(const ais_shape* s) {
     if (!s) return AIS_ERR_NULL;
@@ -152,6 +167,12 @@ constexpr int64_t kBwdRowsRecommended = 2 * 148 * kBM;
 extern "C" {
 
 int ais_version(void) { return AIS_VERSION; }
+
+int ais_set_wait_cycles(int64_t cycles) {
+    if (cycles < 0) return AIS_ERR_PARAM;
+    g_wait_cycles.store(cycles);
+    return AIS_OK;
+}
 
 const char* ais_strerror(int status) {
     switch (status) {
@@ -295,6 +316,7 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     LmheadArgs a;
     memset(&a, 0, sizeof(a));
+    a.wait_cycles = wait_cycles();
     a.rows = shape->T;
     a.row0 = 0;
     a.n_row_tiles = static_cast<int32_t>((shape->T + kBM - 1) / kBM);
@@ -318,8 +340,8 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
 
     CUtensorMap tmA, tmB, tmSA, tmSB;
     if (do_train) {
-        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, H, d, T, shape->ldh * 2, 64, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, H, d, T, shape->ldh * 2, 64, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
             return AIS_ERR_DEVICE;
         a.ksteps = shape->d / 64;
         if (launch_lmhead(kFwdBf16, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
@@ -331,9 +353,9 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
         // power-of-two scales per 32 elements: the block-scaled MMA applies them, the contraction stays in tensor memory
         // FP4 codes are two per byte: the maps see d / 2 bytes per row with half the row stride
         const uint64_t kb = fp4 ? d / 2 : d;
-        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, kb, T, fp4 ? shape->ldh / 2 : shape->ldh, 128, kBM,
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, qH, kb, T, fp4 ? shape->ldh / 2 : shape->ldh, 128, kBM,
                        CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, kb, V, fp4 ? shape->ldw / 2 : shape->ldw, 128, kBN,
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, qW, kb, V, fp4 ? shape->ldw / 2 : shape->ldw, 128, kBN,
                        CU_TENSOR_MAP_SWIZZLE_128B))
             return AIS_ERR_DEVICE;
         a.ksteps = static_cast<int32_t>(kb / 128);
@@ -346,8 +368,8 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
             return AIS_ERR_DEVICE;
     } else if (do_roll && per_tensor) {
         // one scale per tensor: the whole contraction accumulates in tensor memory, the scales meet in the epilogue
-        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
             return AIS_ERR_DEVICE;
         a.ksteps = shape->d / 128;
         a.scale_a = sH;
@@ -358,10 +380,10 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
             return AIS_ERR_DEVICE;
     } else if (do_roll) {
         const uint64_t nkb = d / shape->fp8_block;
-        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap(&tmSA, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, sH, T, nkb, ldsH * 4, kBM, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-            !make_tmap(&tmSB, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, sW, V, nkb, ldsW * 4, kBN, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE))
+        if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmSA, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sH, T, nkb, ldsH * 4, kBM, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+            !make_tmap(&tmSB, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sW, V, nkb, ldsW * 4, kBN, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE))
             return AIS_ERR_DEVICE;
         a.ksteps = shape->d / 128;
         if (launch_lmhead(kFwdFp8, tmA, tmB, tmSA, tmSB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
@@ -470,7 +492,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
     if (launch_seq_counts(mask, seq_offsets, S, nseq, s) != cudaSuccess) return AIS_ERR_DEVICE;
     const int P_norm = shape->P_total > 0 ? shape->P_total : shape->P;
     if (launch_loss_coef(lp_train, lp_old, lp_ref, params->beta_kl, mask, seq_offsets, adv, w_tilde, nseq, shape->T, S, P_norm * shape->G, params->clip_eps,
-                         reinterpret_cast<double*>(ws + L.off_diag), coef, loss, diag, s) != cudaSuccess)
+                         reinterpret_cast<double*>(ws + L.off_diag), coef, loss, diag, lse_train, s) != cudaSuccess)
         return AIS_ERR_DEVICE;
     if (shape->T == 0) return AIS_OK;
     // row tiles whose gradient factors are all zero (masked rows, zero advantage) are skipped by the recompute and dH passes
@@ -484,9 +506,9 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
     const uint64_t V = static_cast<uint64_t>(shape->V), d = static_cast<uint64_t>(shape->d);
 
     CUtensorMap tmW_k, tmW_n, tmU;
-    if (!make_tmap(&tmW_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap(&tmW_n, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, d, V, shape->ldw * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap(&tmU, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, U, V, static_cast<uint64_t>(blk_rows), L.ldU * 2, 64, kBM,
+    if (!make_tmap(&tmW_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap(&tmW_n, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap(&tmU, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, U, V, static_cast<uint64_t>(blk_rows), L.ldU * 2, 64, kBM,
                    CU_TENSOR_MAP_SWIZZLE_128B))
         return AIS_ERR_DEVICE;
 
@@ -494,11 +516,12 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
         const int64_t rows = (shape->T - r0) < blk_rows ? (shape->T - r0) : blk_rows;
         CUtensorMap tmH;
         const __nv_bfloat16* Hc = static_cast<const __nv_bfloat16*>(H) + r0 * shape->ldh;
-        if (!make_tmap(&tmH, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Hc, d, static_cast<uint64_t>(rows), shape->ldh * 2, 64, kBM,
+        if (!make_tmap(&tmH, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Hc, d, static_cast<uint64_t>(rows), shape->ldh * 2, 64, kBM,
                        CU_TENSOR_MAP_SWIZZLE_128B))
             return AIS_ERR_DEVICE;
         LmheadArgs a;
         memset(&a, 0, sizeof(a));
+        a.wait_cycles = wait_cycles();
         a.rows = rows;
         a.row0 = r0;
         a.n_row_tiles = static_cast<int32_t>((rows + kBM - 1) / kBM);
@@ -534,9 +557,9 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
             // dW (+)= U^T H over the rows of this pass: both operands are read with the rows as contraction axis;
             // the maps end at `rows`, so rows the scratch still holds from an earlier pass read as zeros
             CUtensorMap tmU_t, tmH_t;
-            if (!make_tmap(&tmU_t, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, U, V, static_cast<uint64_t>(rows), L.ldU * 2, 64, 64,
+            if (!make_tmap(&tmU_t, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, U, V, static_cast<uint64_t>(rows), L.ldU * 2, 64, 64,
                            CU_TENSOR_MAP_SWIZZLE_128B) ||
-                !make_tmap(&tmH_t, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Hc, d, static_cast<uint64_t>(rows), shape->ldh * 2, 64, 64,
+                !make_tmap(&tmH_t, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Hc, d, static_cast<uint64_t>(rows), shape->ldh * 2, 64, 64,
                            CU_TENSOR_MAP_SWIZZLE_128B))
                 return AIS_ERR_DEVICE;
             LmheadArgs w = a;

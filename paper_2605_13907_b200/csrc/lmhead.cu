@@ -38,6 +38,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     uint64_t* sfull = done + 1;                  // [kStages]   scale warps -> MMA (microscaling passes)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBarriers);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile uint32_t* issued_slot = tmem_slot + 2;     // stage fills the producer has requested (written when it leaves its loop)
 
     constexpr bool TWO_ACC = (MODE == kBwdDh || MODE == kBwdDw);                // two 128-row tiles per CTA, one B slice
     constexpr int STG = TWO_ACC ? kDhStages : kStages;                          // depth of the stage ring
@@ -59,6 +60,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
         mbar_init(done, 1);
         *abort_flag = 0;
+        *issued_slot = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
@@ -86,7 +88,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (!unit_active<MODE>(a, w)) continue;
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
                     for (int ks = 0; ks < a.ksteps; ++ks) {
-                        if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                         uint8_t* sA = stage_base + st.idx * STG_BYTES;
                         uint8_t* sB = sA + A_BYTES;
                         mbar_expect_tx(&full[st.idx], MX ? STG_BYTES + MX_SCALE_BYTES : STG_BYTES);
@@ -131,14 +133,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     }
                 }
             }
-            if (!ok) {
-                // another role gave up: let the copies already in flight land before the CTA exits
-                const uint32_t pending = issued < static_cast<uint32_t>(STG) ? issued : STG;
-                for (uint32_t i = 0; i < pending; ++i) {
-                    const uint32_t n = issued - 1 - i;                 // n-th load overall
-                    mbar_wait_drain(&full[n % STG], (n / STG) & 1u);
-                }
-            }
+            *issued_slot = issued;
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
@@ -153,10 +148,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const Unit w = decode_unit<MODE>(a, u);
                 if (!unit_active<MODE>(a, w)) continue;
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
-                    if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                     tc_fence_after();
                     for (int ks = 0; ks < a.ksteps; ++ks) {
-                        if (!mbar_wait(&full[st.idx], st.phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(&full[st.idx], st.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t sA = smem_u32(stage_base + st.idx * STG_BYTES);
                         const uint32_t sB = sA + A_BYTES;
@@ -185,7 +180,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             // each), then B's (4 columns per 128 rows and chunk).  One block-scaled instruction per 32 bytes
                             // of K, each with its scale id.
                             constexpr int KC = FP4 ? 2 : 1;
-                            if (!mbar_wait(&sfull[st.idx], st.phase, abort_flag)) { ok = false; break; }
+                            if (!mbar_wait(&sfull[st.idx], st.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                             tc_fence_after();
                             const uint32_t tsf = tmem_base + kMxScaleCol + st.idx * kMxSetCols;
 #pragma unroll
@@ -245,7 +240,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             if (!unit_active<MODE>(a, w)) continue;
             for (int t = w.t0; t < w.t1 && ok; ++t) {
                 for (int ks = 0; ks < a.ksteps; ++ks) {
-                    if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                     const uint4* src = reinterpret_cast<const uint4*>(mx_scale_base + st.idx * kMxStageScaleBytes) + lane;
                     const uint32_t tsf = tmem_base + lane_addr + kMxScaleCol + st.idx * kMxSetCols;
 #pragma unroll
@@ -298,7 +293,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             }
             if (MODE == kBwdDh) {
                 // one unit = 256 rows x 256 columns of dH, finished after the whole contraction over the vocabulary
-                if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int sub = 0; sub < 2; ++sub) {
@@ -333,7 +328,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             }
             if (MODE == kBwdDw) {
                 // one unit = 256 vocabulary rows x 256 columns of dW after the contraction over this launch's rows
-                if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int sub = 0; sub < 2; ++sub) {
@@ -392,7 +387,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             for (int t = w.t0; t < w.t1 && ok; ++t) {
                 const int col_base = t * kBN + half * 128;    // first output column of this thread's half
                 {
-                    if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                     tc_fence_after();
                 }
 
@@ -490,7 +485,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
-    if (threadIdx.x == 0 && *abort_flag && a.status) atomicOr(a.status, AIS_FLAG_TIMEOUT);
+    if (threadIdx.x == 0 && *abort_flag) {
+        // some role gave up on a wait: let the producer's copies still in flight land before the CTA exits
+        drain_stage_copies(full, *issued_slot, STG);
+        if (a.status) atomicOr(a.status, AIS_FLAG_TIMEOUT);
+    }
 }
 
 }  // namespace

@@ -71,6 +71,7 @@ struct LmheadArgs {
     __nv_bfloat16* dH;
     int64_t lddh;
     uint32_t* status;
+    int64_t wait_cycles;   // bound of every device-side wait in clock ticks; 0 = the default (about two seconds)
 };
 
 // Launches one pass.  tmSA / tmSB are only read in kFwdFp8 mode.

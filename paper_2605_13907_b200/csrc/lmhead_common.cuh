@@ -24,8 +24,9 @@ struct Pipe {
 
 // Warp-wide wait: every lane polls (so every lane observes the completed phase itself) and the outcome is
 // made uniform, because the tcgen05.ld / __syncwarp that follow need the whole warp.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    const bool r = mbar_wait(bar, parity, abort_flag);
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               long long limit = 0) {
+    const bool r = mbar_wait(bar, parity, abort_flag, limit);
     return __all_sync(0xffffffffu, r);
 }
 
@@ -84,6 +85,17 @@ __device__ __forceinline__ bool unit_active(const LmheadArgs& a, const Unit& w) 
         return a.tile_active[t0] != 0 || (second && a.tile_active[t0 + 1] != 0);
     }
     return a.tile_active[g + w.rt] != 0;
+}
+
+// After every role has left its loops: if the CTA gave up on a wait, the tile copies that the producer issued last
+// (one per stage of the ring at most) may still be in flight.  Wait for them, so that no copy writes into shared
+// memory that the CTA has already given back; `issued` counts the producer's stage fills.
+__device__ __forceinline__ void drain_stage_copies(uint64_t* full, uint32_t issued, uint32_t stages) {
+    const uint32_t pending = issued < stages ? issued : stages;
+    for (uint32_t i = 0; i < pending; ++i) {
+        const uint32_t n = issued - 1 - i;                 // n-th fill overall: stage n % stages, phase n / stages
+        mbar_wait_drain(&full[n % stages], (n / stages) & 1u);
+    }
 }
 
 }  // namespace

@@ -56,6 +56,7 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     uint64_t* done = sempty + C::kSlots;         // [1]        all MMAs of this CTA have completed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kBarriers);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile uint32_t* issued_slot = tmem_slot + 2;     // stage fills the producer has requested (written when it leaves its loop)
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -67,6 +68,7 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         for (int i = 0; i < C::kSlots; ++i) mbar_init(&sempty[i], kEpiWarps);
         mbar_init(done, 1);
         *abort_flag = 0;
+        *issued_slot = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
@@ -95,8 +97,8 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     if (!unit_active<MODE>(a, w)) continue;
                     for (int t = w.t0; t < w.t1 && ok; ++t) {
                         for (int ks = 0; ks < a.ksteps; ++ks) {
-                            if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag)) { ok = false; break; }
-                            if (!mbar_wait(&sempty[sc.idx], sc.phase ^ 1u, abort_flag)) { ok = false; break; }
+                            if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
+                            if (!mbar_wait(&sempty[sc.idx], sc.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                             uint8_t* sA = stage_base + st.idx * kStageBytes;
                             uint8_t* sS = scale_base + sc.idx * C::kSlotBytes;
                             mbar_expect_tx(&full[st.idx], kStageBytes + C::kSlotBytes);
@@ -110,14 +112,7 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         }
                     }
                 }
-                if (!ok) {
-                    // another role gave up: let the copies already in flight land before the CTA exits
-                    const uint32_t pending = issued < static_cast<uint32_t>(kStages) ? issued : kStages;
-                    for (uint32_t i = 0; i < pending; ++i) {
-                        const uint32_t n = issued - 1 - i;
-                        mbar_wait_drain(&full[n % kStages], (n / kStages) & 1u);
-                    }
-                }
+                *issued_slot = issued;
             }
         } else if (warp == 1) {
             // ------------------------------------------------------------------ MMA issuer
@@ -130,12 +125,12 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     if (!unit_active<MODE>(a, w)) continue;
                     const int nst = (w.t1 - w.t0) * a.ksteps;
                     for (int i = 0; i < nst && ok; ++i) {
-                        if (!mbar_wait(&full[st.idx], st.phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(&full[st.idx], st.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                         const uint32_t sA = smem_u32(stage_base + st.idx * kStageBytes);
                         const uint32_t sB = sA + kAStageBytes;
 #pragma unroll
                         for (int g = 0; g < SG; ++g) {
-                            if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag)) { ok = false; break; }
+                            if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                             tc_fence_after();
                             const uint32_t dcol = tmem_base + tb.idx * kBN;
 #pragma unroll
@@ -199,7 +194,7 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     const float* sS = reinterpret_cast<const float*>(scale_base + sc.idx * C::kSlotBytes);
 #pragma unroll 1
                     for (int g = 0; g < SG; ++g) {
-                        if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t buf = tb.idx;
                         ld_piece(buf, 0, 0, va);
@@ -311,7 +306,11 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
-    if (threadIdx.x == 0 && *abort_flag && a.status) atomicOr(a.status, AIS_FLAG_TIMEOUT);
+    if (threadIdx.x == 0 && *abort_flag) {
+        // some role gave up on a wait: let the producer's copies still in flight land before the CTA exits
+        drain_stage_copies(full, *issued_slot, kStages);
+        if (a.status) atomicOr(a.status, AIS_FLAG_TIMEOUT);
+    }
 }
 
 }  // namespace

@@ -40,12 +40,41 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// Every wait in these kernels is bounded.  A wait gives up after kWaitCycles clock ticks (or as soon as
-// another role of the CTA has given up), raises the CTA's abort flag and returns false; the caller then
-// leaves its loops and the kernel ends normally with AIS_FLAG_TIMEOUT set.
+// Every wait in these kernels is bounded.  A wait gives up after `limit` clock ticks (kWaitCycles, about two
+// seconds, unless the caller of the library lowered it) or as soon as another role of the CTA has given up, raises
+// the CTA's abort flag and returns false; the caller then leaves its loops and the kernel ends normally with
+// AIS_FLAG_TIMEOUT set.
 constexpr long long kWaitCycles = 4000000000LL;
+constexpr long long kShortWait = 1000000LL;      // below this limit a wait polls without blocking and reads the clock every time
 
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// A wait with a short limit (a test of the time-out path): non-blocking polls, so that the limit is what ends it.
+__device__ __forceinline__ bool mbar_wait_short(uint64_t* bar, uint32_t parity, volatile int* abort_flag, long long limit) {
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+// `limit` = 0 selects the default bound.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, long long limit = 0) {
+    if (limit != 0 && limit < kShortWait) return mbar_wait_short(bar, parity, abort_flag, limit);
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t it = 0;
@@ -53,14 +82,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return true;
         if ((++it & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > (limit != 0 ? limit : kWaitCycles)) {
                 *abort_flag = 1;
                 return false;
             }
         }
     }
 }
-// Same, but ignores the abort flag (used to drain copies still in flight before leaving).
+// Same, but ignores the abort flag and always takes the long limit (used to drain copies still in flight before
+// leaving: shared memory must not be given up while a copy may still write to it).
 __device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity) {
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {

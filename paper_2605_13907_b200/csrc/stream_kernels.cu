@@ -322,7 +322,13 @@ __global__ void combine_kernel(const float* __restrict__ part_m, const float* __
             } else {
                 out_lp = zy - out_lse;
             }
-            if (!isfinite(out_lse) || !isfinite(out_lp)) flags |= AIS_FLAG_NONFINITE;
+            if (!isfinite(out_lse) || !isfinite(out_lp)) {
+                // a non-finite hidden state or weight reached this row: flag it, give it the neutral log-prob, and mark
+                // its log-sum-exp so that the backward pass leaves the row out (gradient factor 0)
+                flags |= AIS_FLAG_NONFINITE;
+                out_lp = 0.f;
+                out_lse = __int_as_float(0x7fc00000);
+            }
         }
         lp[t] = out_lp;
         if (lse) lse[t] = out_lse;
@@ -459,6 +465,49 @@ __device__ __forceinline__ int seq_of_row(const int32_t* __restrict__ seq_offset
 // sequence of a group's first row comes from a binary search and the following rows only step forward.  The
 // exponentials are evaluated in fp32 (the inputs are fp32 and the sums need seven digits at most), the sums
 // themselves in fp64.  Two groups are in flight per thread so that the fixed grid keeps HBM busy on long batches.
+// rho - 1 = e^x - 1 for a run of n rows.  When every |x| of the run is at most 2^-6 a short series gives it to fp32
+// accuracy RELATIVE TO ITSELF (e^x - 1 from a rounded e^x would be good to 1e-7 absolute only, i.e. to a thousandth of a
+// weight that differs from 1 by 1e-4); otherwise the fast exponential is used, as everywhere else in these kernels.
+template <int N>
+__device__ __forceinline__ void rho_minus_one(const float (&x)[N], float (&u)[N]) {
+    float amax = 0.f;
+#pragma unroll
+    for (int j = 0; j < N; ++j) amax = fmaxf(amax, fabsf(x[j]));
+    if (amax <= 0x1p-6f) {
+#pragma unroll
+        for (int j = 0; j < N; ++j)
+            u[j] = x[j] * fmaf(x[j], fmaf(x[j], fmaf(x[j], 1.0f / 24.0f, 1.0f / 6.0f), 0.5f), 1.0f);
+    } else {
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            float e;
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x[j] * 1.4426950408889634f));
+            u[j] = e - 1.0f;
+        }
+    }
+}
+
+// Sums of w and w^2 over a short run of rows, in double precision, from fp32 sums of shifted values.  The weights
+// enter as u = w - 1 (rho_minus_one above, truncated at C - 1); the run is summed as v = u - p and v^2 about the pivot
+// p = u of its first valid row:  with P = 1 + p,  sum w = n P + sum v  and  sum w^2 = n P^2 + 2 P sum v + sum v^2.
+// The fp32 roundings then scale with the spread of the run and with |w - 1|, not with the size of w, so that the
+// variance formed later as E[w^2] - E[w]^2 in fp64 keeps its digits when the weights differ by 1e-4 of their size,
+// and is exactly zero when they are all equal.  All rows of the run share the advantage A.
+//   acc: 0 N   1 sum w   2 sum w^2   4 sum A   5 sum A^2   6 sum A w   7 sum (A w)^2
+__device__ __forceinline__ void add_run(double* acc, int n, float p, float sv, float sv2, float A) {
+    const double nd = static_cast<double>(n), P = 1.0 + static_cast<double>(p), svd = static_cast<double>(sv);
+    const double Ad = static_cast<double>(A);
+    const double sw = fma(nd, P, svd);
+    const double sw2 = static_cast<double>(sv2) + P * fma(nd, P, 2.0 * svd);
+    acc[0] += nd;
+    acc[1] += sw;
+    acc[2] += sw2;
+    acc[4] = fma(Ad, nd, acc[4]);
+    acc[5] = fma(Ad * Ad, nd, acc[5]);
+    acc[6] = fma(Ad, sw, acc[6]);
+    acc[7] = fma(Ad * Ad, sw2, acc[7]);
+}
+
 template <int VEC>
 struct RowGroup {
     float lt[VEC], lr[VEC];
@@ -499,8 +548,8 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
     // Every warp owns a contiguous range of row groups and its lanes interleave inside it, so a lane's rows only
     // move forward: one binary search for its first group, then the sequence index steps (the next boundary is kept
     // in a register).  Valid rows are counted per sequence on the way (integer atomics: the result does not depend
-    // on their order).  Runs of at most 64 rows are summed in fp32 and those short sums go into the fp64
-    // accumulators, which keeps the fp64 pipe out of the per-row work.
+    // on their order).  The first-order sums (|D|, D, |dp|) take runs of at most 64 rows in fp32 and those short sums go
+    // into the fp64 accumulators; the sums behind the three variances are formed per group of rows by add_run.
     int sq = -1, cur = -1, cnt = 0;
     int64_t next_b = 0;                                   // first row of sequence sq + 1 (or "never" for the last one)
     float f[kNumMoments];
@@ -508,13 +557,12 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
         if (n_valid_seq && cur >= 0 && cnt > 0) atomicAdd(&n_valid_seq[cur], cnt);
         cnt = 0;
     };
-    auto clear = [&]() {
-#pragma unroll
-        for (int i = 0; i < 10; ++i) f[i] = 0.f;
-    };
+    // fp32 runs are kept only for the three first-order sums (3, 8, 9); the sums behind the variances go through add_run
+    auto clear = [&]() { f[3] = 0.f; f[8] = 0.f; f[9] = 0.f; };
     auto commit = [&]() {
-#pragma unroll
-        for (int i = 0; i < 10; ++i) acc[i] += static_cast<double>(f[i]);
+        acc[3] += static_cast<double>(f[3]);
+        acc[8] += static_cast<double>(f[8]);
+        acc[9] += static_cast<double>(f[9]);
     };
     auto seek = [&](int64_t t) {
         if (sq < 0) {
@@ -527,23 +575,15 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
         }
     };
     auto add_row = [&](float lt, float lr, float A) {
-        // two fast exponentials per row (relative error about 1e-6, far inside what the sums need):
-        // rho = e^dl, truncated weight min(rho, C), and |e^lt - e^lr| = e^lr |rho - 1|
-        const float dl = lt - lr;
-        const float rho = __expf(dl);
+        const float dl[1] = {lt - lr};
+        float u[1];
+        rho_minus_one(dl, u);                              // rho - 1; |e^lt - e^lr| = e^lr |rho - 1|
         // sequence-level variant: every row carries its sequence's truncated weight instead of its own
-        const float w = fminf(seq_logw ? __expf(seq_logw[sq]) : rho, C);
-        const float Aw = A * w;
-        f[0] += 1.0f;
-        f[1] += w;
-        f[2] = fmaf(w, w, f[2]);
-        f[3] += fabsf(dl);
-        f[4] += A;
-        f[5] = fmaf(A, A, f[5]);
-        f[6] += Aw;
-        f[7] = fmaf(Aw, Aw, f[7]);
-        f[8] -= dl;
-        f[9] = fmaf(__expf(lr), fabsf(rho - 1.0f), f[9]);
+        const float uw = seq_logw ? fminf(__expf(seq_logw[sq]), C) - 1.0f : fminf(u[0], C - 1.0f);
+        add_run(acc, 1, uw, 0.f, 0.f, A);
+        f[3] += fabsf(dl[0]);
+        f[8] -= dl[0];
+        f[9] = fmaf(__expf(lr), fabsf(u[0]), f[9]);
         if (sq != cur) { flush(); cur = sq; }
         ++cnt;
     };
@@ -555,30 +595,33 @@ __global__ void __launch_bounds__(kDiagThreads) moments_kernel(const float* __re
             // the usual case, all rows of the group in one sequence: one advantage and one weight source for the
             // group, masked rows drop out by selection, and the sums that involve A follow from sum w and sum w^2
             const float A = adv[sq];
-            const float wseq = seq_logw ? __expf(seq_logw[sq]) : 0.f;
-            float n = 0.f, sw = 0.f, sw2 = 0.f;
+            const float useq = seq_logw ? fminf(__expf(seq_logw[sq]), C) - 1.0f : 0.f;
+            float dl[VEC], u[VEC];
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) dl[j] = r.mk[j] != 0 ? r.lt[j] - r.lr[j] : 0.f;
+            rho_minus_one(dl, u);
+            float p = 0.f;
+            int n = 0;
 #pragma unroll
             for (int j = 0; j < VEC; ++j) {
                 const bool on = r.mk[j] != 0;
-                const float dl = r.lt[j] - r.lr[j];
-                const float rho = __expf(dl);
-                const float w = fminf(seq_logw ? wseq : rho, C);
-                n += on ? 1.0f : 0.f;
-                sw += on ? w : 0.f;
-                sw2 += on ? w * w : 0.f;
-                f[3] += on ? fabsf(dl) : 0.f;
-                f[8] -= on ? dl : 0.f;
-                f[9] += on ? __expf(r.lr[j]) * fabsf(rho - 1.0f) : 0.f;
+                f[3] += fabsf(dl[j]);
+                f[8] -= dl[j];
+                f[9] += on ? __expf(r.lr[j]) * fabsf(u[j]) : 0.f;
+                u[j] = seq_logw ? useq : fminf(u[j], C - 1.0f);
+                if (on && n == 0) p = u[j];                        // pivot: the first valid row
+                n += on ? 1 : 0;
             }
-            f[0] += n;
-            f[1] += sw;
-            f[2] += sw2;
-            f[4] = fmaf(A, n, f[4]);
-            f[5] = fmaf(A * A, n, f[5]);
-            f[6] = fmaf(A, sw, f[6]);
-            f[7] = fmaf(A * A, sw2, f[7]);
+            float sv = 0.f, sv2 = 0.f;
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) {
+                const float v = r.mk[j] != 0 ? u[j] - p : 0.f;
+                sv += v;
+                sv2 = fmaf(v, v, sv2);
+            }
+            add_run(acc, n, p, sv, sv2, A);
             if (sq != cur) { flush(); cur = sq; }
-            cnt += static_cast<int>(n);
+            cnt += n;
             return;
         }
 #pragma unroll
@@ -718,29 +761,33 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
     // sums over the rows of a group whose mask byte (rows 0..3 in `m0`, 4..7 in `m1`) is set, all of them in sequence
     // `cur`; returns how many they are
     auto add_rows = [&](const float (&lt)[8], const float (&lr)[8], uint32_t m0, uint32_t m1) -> int {
-        int n = 0;
-        float sw = 0.f, sw2 = 0.f;
+        float dl[8], u[8];
+        bool on[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const bool on = ((j < 4 ? m0 : m1) & (0xFFu << (8 * (j & 3)))) != 0u;
-            const float dl = on ? lt[j] - lr[j] : 0.f;             // a masked row enters with dl = 0 and weight 0
-            const float rho = exp_ftz(dl);
-            const float w = on ? (SEQ ? wseq : fminf(rho, C)) : 0.f;
-            n += on ? 1 : 0;
-            sw += w;
-            sw2 = fmaf(w, w, sw2);
-            f[3] += fabsf(dl);
-            f[8] -= dl;
-            f[9] = fmaf(exp_ftz(on ? lr[j] : 0.f), fabsf(rho - 1.0f), f[9]);     // |e^lt - e^lr| = e^lr |rho - 1|
+            on[j] = ((j < 4 ? m0 : m1) & (0xFFu << (8 * (j & 3)))) != 0u;
+            dl[j] = on[j] ? lt[j] - lr[j] : 0.f;                   // a masked row enters with dl = 0
         }
-        const float nf = static_cast<float>(n);
-        f[0] += nf;
-        f[1] += sw;
-        f[2] += sw2;
-        f[4] = fmaf(A, nf, f[4]);
-        f[5] = fmaf(A * A, nf, f[5]);
-        f[6] = fmaf(A, sw, f[6]);
-        f[7] = fmaf(A * A, sw2, f[7]);
+        rho_minus_one(dl, u);                                      // rho - 1
+        int n = 0;
+        float p = 0.f;                                             // pivot: w - 1 of the first valid row
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            f[3] += fabsf(dl[j]);
+            f[8] -= dl[j];
+            f[9] = fmaf(exp_ftz(on[j] ? lr[j] : 0.f), fabsf(u[j]), f[9]);       // |e^lt - e^lr| = e^lr |rho - 1|
+            u[j] = SEQ ? wseq - 1.0f : fminf(u[j], C - 1.0f);
+            p = (on[j] && n == 0) ? u[j] : p;
+            n += on[j] ? 1 : 0;
+        }
+        float sv = 0.f, sv2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float v = on[j] ? u[j] - p : 0.f;
+            sv += v;
+            sv2 = fmaf(v, v, sv2);
+        }
+        add_run(acc, n, p, sv, sv2, A);
         return n;
     };
 
@@ -781,9 +828,10 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
                     j = j1;
                 }
             }
-            if ((k & 7u) == 7u) {                       // at most 64 rows per fp32 run
-#pragma unroll
-                for (int i = 0; i < 10; ++i) { acc[i] += static_cast<double>(f[i]); f[i] = 0.f; }
+            if ((k & 7u) == 7u) {                       // at most 64 rows per fp32 run of the first-order sums
+                acc[3] += static_cast<double>(f[3]); f[3] = 0.f;
+                acc[8] += static_cast<double>(f[8]); f[8] = 0.f;
+                acc[9] += static_cast<double>(f[9]); f[9] = 0.f;
             }
         }
         if (n_valid_seq) {
@@ -824,8 +872,9 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
         add_rows(lt, lr, 1u, 0u);
         if (n_valid_seq) atomicAdd(&n_valid_seq[sq], 1);
     }
-#pragma unroll
-    for (int i = 0; i < 10; ++i) acc[i] += static_cast<double>(f[i]);
+    acc[3] += static_cast<double>(f[3]);
+    acc[8] += static_cast<double>(f[8]);
+    acc[9] += static_cast<double>(f[9]);
     if (failed) acc[0] = __longlong_as_double(0x7ff8000000000000LL);     // a NaN count marks the batch as not reduced
 #pragma unroll
     for (int i = 0; i < kNumMoments; ++i) {
@@ -859,14 +908,14 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
         d.alpha_adaptive = 0.0; d.kl_k1 = 0.0; d.mean_abs_dp = 0.0;
         d.status_flags |= AIS_FLAG_EMPTY;
     } else {
-        // Population variance from a sum and a sum of squares whose terms were rounded to fp32: a result below the
-        // rounding noise of those terms and of their fp32 partial sums (2^-20 of the mean square) is zero.  Without this a batch whose valid
-        // rows all share one advantage (one row, one sequence) gets std(A w) = 1e-4 |A w| instead of 0, which the
-        // eps of Delta-sigma turns into a huge variance ratio.
+        // Population variance E[x^2] - E[x]^2 in fp64.  The sums reach this point with fp64 accuracy relative to the
+        // spread of the data (add_run), so what is left is the rounding of the fp64 additions themselves: a result
+        // below 2^-44 of the mean square (a few hundred ulps of it; a standard deviation below 2.4e-7 of the rms
+        // value) is that rounding and is reported as exactly zero.
         auto variance = [&](double sum, double sumsq) {
             const double mean = sum / N, ms = sumsq / N;
             const double v = ms - mean * mean;
-            return v > ms * 0x1p-20 ? v : 0.0;
+            return v > ms * 0x1p-44 ? v : 0.0;
         };
         const double mu = m[1] / N;
         const double var = variance(m[1], m[2]);
@@ -950,11 +999,12 @@ __global__ void __launch_bounds__(kDiagThreads) loss_coef_kernel(const float* __
                                                                   const float* __restrict__ adv, const float* __restrict__ w_tilde,
                                                                   const int32_t* __restrict__ n_valid_seq, int64_t T, int S,
                                                                   int S_norm, double clip_eps, double* __restrict__ partials,
-                                                                  float* __restrict__ coef) {
+                                                                  float* __restrict__ coef, const float* __restrict__ lse) {
     __shared__ double scratch[32];
     double J = 0.0, KL = 0.0;
     // one valid row of sequence sq: its share of the objective, of the KL estimate, and its gradient factor
     auto one = [&](int64_t t, int sq, float wtf) -> float {
+        if (!isfinite(lse[t])) return 0.f;       // the forward pass marked this row (non-finite logits): it takes no part
         const double A = adv[sq];
         const int n = n_valid_seq[sq] > 0 ? n_valid_seq[sq] : 1;
         const double norm = 1.0 / (static_cast<double>(S_norm) * static_cast<double>(n));
@@ -1177,16 +1227,17 @@ cudaError_t launch_finalize(const double* moments, const float* lp_train, const 
 cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const float* lp_ref, float beta_kl, const uint8_t* mask,
                              const int32_t* seq_offsets,
                              const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S, int S_norm,
-                             float clip_eps, double* partials, float* coef, float* loss, ais_diag* diag, cudaStream_t stream) {
+                             float clip_eps, double* partials, float* coef, float* loss, ais_diag* diag, const float* lse,
+                             cudaStream_t stream) {
     const float* ref = (beta_kl != 0.f) ? lp_ref : nullptr;
     if (vec4_ok(w_tilde, coef, nullptr, nullptr, mask))
         loss_coef_kernel<4><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, ref, static_cast<double>(beta_kl), mask,
                                                                         seq_offsets, adv, w_tilde, n_valid_seq, T, S, S_norm,
-                                                                        static_cast<double>(clip_eps), partials, coef);
+                                                                        static_cast<double>(clip_eps), partials, coef, lse);
     else
         loss_coef_kernel<1><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_old, ref, static_cast<double>(beta_kl), mask,
                                                                         seq_offsets, adv, w_tilde, n_valid_seq, T, S, S_norm,
-                                                                        static_cast<double>(clip_eps), partials, coef);
+                                                                        static_cast<double>(clip_eps), partials, coef, lse);
     loss_finalize_kernel<<<1, 32, 0, stream>>>(partials, kDiagBlocks, ref ? static_cast<double>(beta_kl) : 0.0, loss, diag);
     return cudaGetLastError();
 }

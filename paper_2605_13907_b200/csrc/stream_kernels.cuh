@@ -59,11 +59,12 @@ cudaError_t launch_finalize(const double* moments, const float* lp_train, const 
                             const float* seq_logw, cudaStream_t stream);
 
 // coef[t] and the loss; n_valid_seq must already hold the valid counts.  S_norm is the number of sequences the
-// objective averages over (all data-parallel ranks together).
+// objective averages over (all data-parallel ranks together).  Rows whose lse is not finite (marked by the forward
+// pass) contribute nothing.
 cudaError_t launch_loss_coef(const float* lp_train, const float* lp_old, const float* lp_ref, float beta_kl, const uint8_t* mask,
                              const int32_t* seq_offsets,
                              const float* adv, const float* w_tilde, const int32_t* n_valid_seq, int64_t T, int S, int S_norm,
                              float clip_eps, double* partials /*[kDiagBlocks][2]*/, float* coef, float* loss, ais_diag* diag,
-                             cudaStream_t stream);
+                             const float* lse, cudaStream_t stream);
 
 }  // namespace ais

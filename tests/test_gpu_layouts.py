@@ -124,6 +124,55 @@ def test_batch_reductions_on_unaligned_and_ragged_vectors(T, shift, S):
     assert np.allclose(got_wt[valid], ref_wt[valid], rtol=1e-4, atol=1e-5) and np.all(got_wt[~valid] == 1)
 
 
+@pytest.mark.parametrize("T,shift", [(3 * 2048 + 77, 0), (1027, 1), (1, 0)])
+def test_small_but_non_zero_variance_is_kept(T, shift):
+    """Every valid row carries the same advantage (the other response of each prompt has no valid row) and a weight of
+    1 +- 1e-4: std(A) is exactly 0 and std(A w) is 0.5e-4, which the eps of the variance-amplification ratio turns into
+    Delta-sigma = 50, so alpha is 0 (Eq. alpha-var).  Sums of squares rounded to fp32 lose this variance (1e-8 of the
+    mean square); the kernels' shifted sums must not.  T = 1 is the case of one valid row, where every variance is 0."""
+    import paper_2605_13907_b200 as ais
+    rng = np.random.default_rng(7 + T)
+    S, G = 4, 2
+    cuts = np.sort(rng.integers(0, T + 1, S - 1))
+    offs = np.concatenate([[0], cuts, [T]]).astype(np.int32)
+    lp_t = -rng.uniform(0.5, 4.0, T).astype(np.float32)
+    lp_r = (lp_t.astype(np.float64) - 1e-4 * rng.choice([-1.0, 1.0], T)).astype(np.float32)
+    mask = np.zeros(T, np.uint8)
+    for s in (0, 2):
+        mask[offs[s]:offs[s + 1]] = (rng.random(offs[s + 1] - offs[s]) < 0.8)
+    if T == 1:
+        offs = np.array([0, 1, 1, 1, 1], np.int32)
+        mask[:] = 1
+    rew = np.array([1, 0, 1, 0], np.float32)
+    op = oais.Params()
+    ref_adv = oais.advantages(rew.astype(np.float64), G)
+    ref = oais.diagnostics(lp_t, lp_r, mask, ref_adv[oais.seq_ids(offs, T)], op)
+    if T > 1:
+        assert ref["std_A"] == 0.0 and 20 < ref["delta_sigma"] < 80 and ref["alpha"] == 0.0 and ref["alpha_ess"] > 0.99
+
+    def shifted(x):
+        buf = torch.empty(x.size + 8, dtype=torch.from_numpy(x).dtype, device="cuda")
+        v = buf[shift:shift + x.size]
+        v.copy_(torch.from_numpy(x))
+        return v
+
+    params = ais.default_params()
+    shape = ais.make_shape(T, 128, 1024, S // G, G, 128)
+    ws = torch.empty(ais.workspace_min_bytes(shape, params), dtype=torch.uint8, device="cuda")
+    adv = torch.empty(S, device="cuda")
+    nseq = torch.zeros(S, dtype=torch.int32, device="cuda")
+    rho, wt = torch.zeros(T, device="cuda"), torch.zeros(T, device="cuda")
+    diag = torch.zeros(32, dtype=torch.float64, device="cuda")
+    ais.diagnostics(shape, params, shifted(lp_t), shifted(lp_r), shifted(mask), torch.from_numpy(offs).cuda(),
+                    torch.from_numpy(rew).cuda(), adv, nseq, rho, wt, diag, ws)
+    torch.cuda.synchronize()
+    d = ais.Diag.from_buffer_copy(diag.cpu().numpy().tobytes()[:ctypes.sizeof(ais.Diag)]).as_dict()
+    assert d["n_valid"] == ref["n_valid"] and d["std_A"] == 0.0
+    assert abs(d["alpha"] - ref["alpha"]) <= 1e-3
+    for k in ("cv2", "std_Aw", "delta_sigma", "alpha_var", "alpha_ess"):
+        assert d[k] == pytest.approx(ref[k], rel=1e-5, abs=1e-15), (k, d[k], ref[k])
+
+
 def test_sequence_level_weights_on_gpu():
     """params.seq_level_weights: every valid row carries min(prod_t rho_t, C) of its sequence (Eq. is-weight).  The
     fused call and the split pair agree with the oracle's sequence-level variant; d_bar and rho stay per token."""

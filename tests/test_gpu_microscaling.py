@@ -7,6 +7,7 @@ import pytest
 import torch
 
 import abi_layout
+import row_sampling
 import workloads
 from oracle import ais as oais
 from oracle import e4m3
@@ -88,8 +89,8 @@ def test_mx_fullsize_sampled_rows(fmt):
     step.forward(batch.H, batch.W, batch.tokens, batch.mask)
     torch.cuda.synchronize()
     assert int(step.status.item()) == 0
-    rng = np.random.default_rng(5)
-    rows = np.unique(np.concatenate([[0, 127, 128, T - 1, (T // 128) * 128 - 1, (T // 128) * 128], rng.integers(0, T, 42)]))
+    rows = row_sampling.sample_rows(batch.seq_offsets.numpy(), T, 1024, np.random.default_rng(5))     # >= 8 of each sequence
+    assert row_sampling.rows_per_sequence(rows, batch.seq_offsets.numpy()).min() >= 8
     Hs = batch.H[torch.as_tensor(rows, device="cuda")].float().cpu().numpy().astype(np.float64)
     qHs, sHs = quant(Hs)
     assert np.array_equal(plain(step.qH.cpu().numpy()[rows]), qHs)

@@ -67,6 +67,9 @@ def _compare_all(batch, step, ref, a, check_grad=True):
     rho = step.rho.cpu().numpy()[:T].astype(np.float64)
     assert np.max(np.abs(rho - ref["rho"]) / ref["rho"]) <= RHO_RTOL
     assert np.all(rho[~valid] == 1)
+    w_tilde = step.w_tilde.cpu().numpy()[:T].astype(np.float64)
+    assert np.max(np.abs(w_tilde - ref["w_tilde"]) / ref["w_tilde"]) <= RHO_RTOL      # 1 + alpha (min(rho, C) - 1)
+    assert np.all(w_tilde[~valid] == 1)
     d = step.read_diag()
     assert abs(d["alpha"] - ref["diag"]["alpha"]) <= ALPHA_ATOL
     assert d["n_valid"] == ref["diag"]["n_valid"]
@@ -201,6 +204,49 @@ def test_alpha_endpoints_and_clip_on_gpu():
     _, ref = _oracle(batch, lp_old=lp_old_gpu.cpu().numpy().astype(np.float64))
     assert np.any((ref["c"] == 0) & (a["mask"] == 1))
     _compare_all(batch, step, ref, a)
+
+
+@pytest.mark.parametrize("C", [2.0, 10.0])
+def test_truncation_threshold_sweep_on_gpu(C):
+    """C = 2 and C = 10 (the thresholds of the paper's variation analysis besides the default 5) through
+    ais_diagnostics and ais_loss_bwd on a batch whose ratios exceed both: the rollout log-probs of some rows are pushed
+    down by 1 .. 3.5 nats, so rho reaches 2.7 .. 33 there.  Prop. 'bounded second moment': 0 <= w_tilde <= 1 + alpha (C - 1)."""
+    ais = _lib()
+    w = workloads.scaled(workloads.WORKLOADS["tiny"], V=768, P=3, G=4, lengths="uniform:30:70", seed=35)
+    batch = _to_cuda(workloads.make_batch(w, device="cpu"))
+    a = workloads.to_numpy(batch)
+    T = batch.T
+    step = ais.AisStep(T, w.d, w.V, w.P, w.G, w.block, params=ais.default_params(C=C))
+    step.forward(batch.H, batch.W, batch.tokens, batch.mask)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(36)
+    shift = np.where(rng.random(T) < 0.15, rng.uniform(1.0, 3.5, T), 0.0)
+    step.lp_roll[:T] -= torch.tensor(shift, dtype=torch.float32, device="cuda")
+    offs, rew = batch.seq_offsets.cuda(), batch.rewards.cuda()
+    step.diagnose(batch.mask, offs, rew)
+    step.backward(batch.H, batch.W, batch.tokens, batch.mask, offs)
+    torch.cuda.synchronize()
+    assert int(step.status.item()) == 0
+    lt = step.lp_train[:T].cpu().numpy().astype(np.float64)
+    lr = step.lp_roll[:T].cpu().numpy().astype(np.float64)
+    p = oais.Params(C=C)
+    adv = oais.advantages(a["rewards"], w.G)
+    _, rho, wbar = oais.ratios(lt, lr, a["mask"], C)
+    assert np.sum(rho > C) >= 5 and np.sum(rho > 10.0) >= 1
+    diag = oais.diagnostics(lt, lr, a["mask"], adv[oais.seq_ids(a["seq_offsets"], T)], p)
+    w_tilde = oais.rectify(wbar, diag["alpha"], a["mask"])
+    d = step.read_diag()
+    assert abs(d["alpha"] - diag["alpha"]) <= ALPHA_ATOL
+    for k in ("mean_w", "cv2", "ess_ratio", "alpha_ess", "d_bar", "delta_sigma", "alpha_var"):
+        assert d[k] == pytest.approx(diag[k], rel=1e-4, abs=1e-7), k
+    g_wt = step.w_tilde[:T].cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(g_wt - w_tilde) / w_tilde) <= RHO_RTOL
+    assert g_wt.min() >= 0.0 and g_wt.max() <= 1.0 + diag["alpha"] * (C - 1.0) + 1e-5
+    assert np.max(np.abs(step.rho[:T].cpu().numpy() - rho) / rho) <= RHO_RTOL
+    loss, c = oais.loss_and_coeff(lt, lt, a["mask"], a["seq_offsets"], adv, w_tilde, w.P, w.G, p.clip_eps)
+    assert abs(float(step.loss.item()) - loss) <= 1e-3 * max(1.0, abs(loss))
+    dH_ref = oais.grad_hidden(a["H"], a["W"], a["tokens"], c)
+    assert _rel_fro(step.dH.float().cpu().numpy()[:T].astype(np.float64), dH_ref) <= DH_REL
 
 
 def test_kl_term_on_gpu():

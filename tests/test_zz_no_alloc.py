@@ -3,9 +3,10 @@
 ais_logprob_train_static serves callers that own nothing but their inputs and outputs - a callback inside
 another framework, or a process whose device memory has all been given to some other pool - and so cannot
 supply the workspace that ais_logprob_fwd needs.  It keeps its scratch in a fixed array inside the library.
-The array is shared by all calls and keeps old contents, so the check is made on two calls in a row with
-different shapes: the second must not be disturbed by what the first left behind.  This file is named to be
-collected last.
+The array is shared by all calls and keeps old contents, so the check is made on calls in a row with different
+shapes: a later one must not be disturbed by what an earlier one left behind, in particular when it streams the
+vocabulary in fewer ranges and so leaves planes of the array untouched.  Every call is compared with the regular
+entry point and with the float64 oracle.  This file is named to be collected last.
 """
 
 import numpy as np
@@ -13,13 +14,14 @@ import pytest
 import torch
 
 import workloads
+from oracle import ais as oais
 
 pytestmark = pytest.mark.gpu
 
 LP_ATOL = 1e-2          # the log-prob tolerance of the other GPU tests
 
 
-def _case(ais, w):
+def _case(ais, w, check_free_memory=False):
     b = workloads.make_batch(w, device="cpu")
     H, W, tok, msk = b.H.cuda(), b.W.cuda(), b.tokens.cuda(), b.mask.cuda()
     T = b.T
@@ -29,14 +31,22 @@ def _case(ais, w):
     lp = torch.full((T,), 7.0, dtype=torch.float32, device="cuda")
     lse = torch.full((T,), 7.0, dtype=torch.float32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
+    free_before = torch.cuda.mem_get_info()[0]
     ais.logprob_train_static(step.shape, H, W, tok, msk, lp, lse, status)
     torch.cuda.synchronize()
-    assert torch.cuda.memory_allocated() == before            # nothing was taken from torch's allocator either
+    assert torch.cuda.memory_allocated() == before            # nothing was taken from torch's allocator
+    if check_free_memory:                                     # nor from the device (not on a device's first call, which
+        assert torch.cuda.mem_get_info()[0] == free_before    # may still load the library image with the array in it)
     assert int(status.item()) == 0 and int(step.status.item()) == 0
     assert float((lp - step.lp_train[:T]).abs().max()) <= LP_ATOL
     assert float((lse - step.lse_train[:T]).abs().max()) <= LP_ATOL
     assert torch.all(lp[msk == 0] == 0)
+    a = workloads.to_numpy(b)
+    ref_lp, ref_lse = oais.logprob_train(a["H"], a["W"], a["tokens"], a["mask"])
+    assert np.max(np.abs(lp.cpu().numpy() - ref_lp)) <= LP_ATOL
+    assert np.max(np.abs(lse.cpu().numpy() - ref_lse)) <= LP_ATOL
     return lp
 
 
@@ -48,9 +58,16 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
     lp1 = _case(ais, w1)
     # second call right after it: fewer rows and another vocabulary size, so stale partials lie beyond and beside its own
     w2 = workloads.scaled(base, d=256, V=1024, P=2, G=2, lengths="uniform:10:60", seed=72)
-    lp2 = _case(ais, w2)
+    lp2 = _case(ais, w2, check_free_memory=True)
+    # third call: two 256-column tiles only, so the vocabulary goes in 2 ranges and 4 of the 8 planes keep what the
+    # calls before wrote there; then a one-range call
+    w3 = workloads.scaled(base, d=256, V=512, P=2, G=2, lengths="uniform:20:90", seed=73)
+    lp3 = _case(ais, w3, check_free_memory=True)
+    w4 = workloads.scaled(base, d=128, V=256, P=1, G=2, lengths="uniform:100:140", seed=74)
+    lp4 = _case(ais, w4, check_free_memory=True)
     assert lp1.shape != lp2.shape
-    assert torch.isfinite(lp1).all() and torch.isfinite(lp2).all()
+    for lp in (lp1, lp2, lp3, lp4):
+        assert torch.isfinite(lp).all()
 
 
 def test_static_scratch_rejects_too_many_rows():
