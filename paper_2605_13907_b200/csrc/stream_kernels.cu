@@ -1,4 +1,6 @@
 // Streaming kernels of the AIS path (everything that is not a dense contraction).
+#include <type_traits>
+
 #include "stream_kernels.cuh"
 #include "ptx.cuh"
 
@@ -689,12 +691,48 @@ __device__ __forceinline__ float exp_ftz(float x) {
     return y;
 }
 
+// Two fp32 operations per instruction (the packed forms of sm_100): the staged kernel is bound by instruction issue
+// right after HBM, and half of its per-row work is additions, multiplications and multiply-adds.
+struct F2 { float x, y; };
+__device__ __forceinline__ F2 add2(F2 a, F2 b) {
+    F2 r;
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tadd.rn.f32x2 rc, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rc;\n\t}" : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return r;
+}
+__device__ __forceinline__ F2 sub2(F2 a, F2 b) {
+    F2 r;
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tsub.rn.f32x2 rc, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rc;\n\t}" : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return r;
+}
+__device__ __forceinline__ F2 mul2(F2 a, F2 b) {
+    F2 r;
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmul.rn.f32x2 rc, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rc;\n\t}" : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return r;
+}
+__device__ __forceinline__ F2 fma2(F2 a, F2 b, F2 c) {
+    F2 r;
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return r;
+}
+__device__ __forceinline__ float ex2_ftz(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 // The waiting part of a bounded mbarrier wait, kept out of line so that the loop around it stays small.
 __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, int* abort_flag) {
     return mbar_wait(bar, parity, abort_flag);
 }
 
-template <bool SEQ>   // SEQ: every row carries its sequence's truncated weight instead of its own
+// SEQ: every row carries its sequence's truncated weight instead of its own.  EXACT: the second of two launches (see
+// add_rows below): a block returns at once unless the first launch found all of its log-probability gaps tiny.
+template <bool SEQ, bool EXACT>
 __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const float* __restrict__ lp_train,
                                                                          const float* __restrict__ lp_roll,
                                                                          const uint8_t* __restrict__ mask,
@@ -714,6 +752,13 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
     const int per = (ntiles + gridDim.x - 1) / gridDim.x;
     const int tile0 = blockIdx.x * per < ntiles ? blockIdx.x * per : ntiles;
     const int tile1 = tile0 + per < ntiles ? tile0 + per : ntiles;
+    if (EXACT) {
+        // slots 10 and 11 of the block's partial sums: its groups with a gap above 2^-6 and its groups of valid rows without,
+        // as counted by the first launch; slot 0 is NaN when that launch gave up on a wait
+        const double big = partials[blockIdx.x * kNumMoments + 10], small = partials[blockIdx.x * kNumMoments + 11];
+        const double n0 = partials[blockIdx.x * kNumMoments];
+        if (big != 0.0 || small == 0.0 || n0 != n0) return;
+    }
     if (tid == 0) {
         for (int i = 0; i < kMomStages; ++i) mbar_init(&full[i], 1);
         abort_flag = 0;
@@ -728,19 +773,36 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
         bulk_load(dst + kMomRows * 4, lp_roll + r0, kMomRows * 4, &full[st]);
         bulk_load(dst + kMomRows * 8, mask + r0, kMomRows, &full[st]);
     };
-    int issued = tile0;                                 // first tile not yet requested (thread 0)
-    if (tid == 0)
-        for (; issued < tile1 && issued < tile0 + kMomStages; ++issued) issue(issued, issued - tile0);
 
-    double acc[10];
-    float f[10];
-#pragma unroll
-    for (int i = 0; i < 10; ++i) { acc[i] = 0.0; f[i] = 0.f; }
+    // Everything a thread sums stays in fp32 while it walks its tiles and turns into fp64 once, at the end: the first-order
+    // sums (|D|, D, |dp|) as they are, the sums behind the three variances as SHIFTED sums about pivots taken from the
+    // thread's own data -- v = (w - 1) - pivot for the weights, dA = A - A_pivot for the advantages, and
+    // x = A w - A_pivot (1 + pivot) = A v + dA (1 + pivot) for their product -- so that the fp32 roundings scale with the
+    // spread of the data and not with its size, and are exactly zero when all rows are equal.  A thread sees at most
+    // T / 151,552 rows.
+    float f3, f9, g_v, g_v2, g_dA, g_dA2, g_x, g_x2;
+    F2 f8p;                                             // sum of D, two rows at a time
+    int nrows;                                          // valid rows of the thread
+    int nbig, nsmall;                                   // groups with a gap above 2^-6 / with all gaps below (see add_rows)
+    float pivot, A_pivot, dA;
+    bool have_pivot;                                    // both pivots come from the thread's first group with a valid row
     constexpr int kNever = 0x7fffffff;
-    int sq = -1, cur = -1;
-    int next_b = 0;                                     // first row of sequence sq + 1 (or "never" for the last one)
+    int sq, cur;
+    int next_b;                                         // first row of sequence sq + 1 (or "never" for the last one)
     float A = 0.f, wseq = 0.f;                          // advantage and sequence-level weight of sequence `cur`
     int wsq = -1, wcnt = 0;                             // lane 0: valid rows of the warp's strips counted for sequence wsq
+    auto reset = [&]() {
+        f3 = f9 = g_v = g_v2 = g_dA = g_dA2 = g_x = g_x2 = 0.f;
+        f8p = F2{0.f, 0.f};
+        nrows = 0;
+        nbig = 0;
+        nsmall = 0;
+        pivot = A_pivot = dA = 0.f;
+        have_pivot = false;
+        sq = cur = -1;
+        next_b = 0;
+    };
+    reset();
     auto seek = [&](int t) {
         if (sq < 0) {
             sq = seq_of_row(seq_offsets, S, t);
@@ -755,113 +817,176 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
         if (sq != cur) {
             cur = sq;
             A = adv[sq];
+            dA = have_pivot ? A - A_pivot : 0.f;
             if (SEQ) wseq = fminf(__expf(seq_logw[sq]), C);
         }
     };
-    // sums over the rows of a group whose mask byte (rows 0..3 in `m0`, 4..7 in `m1`) is set, all of them in sequence
-    // `cur`; returns how many they are
+    // Sums over the rows of a group whose mask byte (rows 0..3 in `m0`, 4..7 in `m1`) is set, all of them in sequence
+    // `cur`; returns how many they are.  Rows go two at a time through the packed fp32 instructions.  The weight pivot
+    // is w - 1 of the first valid row this thread meets and stays: any value of the data serves.
+    // rho - 1 comes from the fast exponential, which is good to 1e-7 ABSOLUTE: enough unless the gaps D themselves are
+    // tiny, when it is only a thousandth of a weight that differs from 1 by 1e-4.  The EXACT form of this kernel uses a
+    // short series for groups whose |D| are all at most 2^-6 (their sum is), which gives e^D - 1 to fp32 accuracy
+    // relative to itself.  It is slower (the second path costs registers and scheduling freedom: a fifth of the
+    // bandwidth), so the fast form runs first and counts each block's groups above 2^-6, and the exact form is launched
+    // after it: there only the blocks that met no such group walk their tiles again and replace their partial sums.
     auto add_rows = [&](const float (&lt)[8], const float (&lr)[8], uint32_t m0, uint32_t m1) -> int {
-        float dl[8], u[8];
+        const uint32_t v0 = __vcmpne4(m0, 0u), v1 = __vcmpne4(m1, 0u);     // 0xFF in the byte of every valid row
+        const int n = (__popc(v0) + __popc(v1)) >> 3;
         bool on[8];
+        float dl[8], u[8], e[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) on[j] = ((j < 4 ? v0 : v1) & (0x80u << (8 * (j & 3)))) != 0u;
+        float s3 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+            const F2 d = sub2(F2{lt[j], lt[j + 1]}, F2{lr[j], lr[j + 1]});
+            dl[j] = on[j] ? d.x : 0.f;                             // a masked row enters with D = 0
+            dl[j + 1] = on[j + 1] ? d.y : 0.f;
+            f8p = add2(f8p, F2{dl[j], dl[j + 1]});
+            s3 += fabsf(dl[j]);
+            s3 += fabsf(dl[j + 1]);
+        }
+        f3 += s3;
+        if (EXACT && s3 <= 0x1p-6f) {
+#pragma unroll
+            for (int j = 0; j < 8; j += 2) {
+                const F2 x = {dl[j], dl[j + 1]};
+                F2 q = fma2(x, F2{1.0f / 24.0f, 1.0f / 24.0f}, F2{1.0f / 6.0f, 1.0f / 6.0f});
+                q = fma2(x, q, F2{0.5f, 0.5f});
+                q = fma2(x, q, F2{1.0f, 1.0f});
+                q = mul2(x, q);
+                u[j] = q.x;
+                u[j + 1] = q.y;
+            }
+        } else {
+            if (!EXACT) {
+                nbig += s3 > 0x1p-6f ? 1 : 0;
+                nsmall += (s3 <= 0x1p-6f && n > 0) ? 1 : 0;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; j += 2) {
+                const F2 x = mul2(F2{dl[j], dl[j + 1]}, F2{1.4426950408889634f, 1.4426950408889634f});
+                const F2 r = add2(F2{ex2_ftz(x.x), ex2_ftz(x.y)}, F2{-1.0f, -1.0f});
+                u[j] = r.x;
+                u[j + 1] = r.y;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {                           // |e^lt - e^lr| = e^lr |rho - 1|
+            const F2 y = mul2(F2{on[j] ? lr[j] : 0.f, on[j + 1] ? lr[j + 1] : 0.f}, F2{1.4426950408889634f, 1.4426950408889634f});
+            e[j] = ex2_ftz(y.x);
+            e[j + 1] = ex2_ftz(y.y);
+        }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            on[j] = ((j < 4 ? m0 : m1) & (0xFFu << (8 * (j & 3)))) != 0u;
-            dl[j] = on[j] ? lt[j] - lr[j] : 0.f;                   // a masked row enters with dl = 0
+            f9 = fmaf(e[j], fabsf(u[j]), f9);
+            u[j] = SEQ ? wseq - 1.0f : fminf(u[j], C - 1.0f);      // truncated weight minus one
         }
-        rho_minus_one(dl, u);                                      // rho - 1
-        int n = 0;
-        float p = 0.f;                                             // pivot: w - 1 of the first valid row
+        if (!have_pivot) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            f[3] += fabsf(dl[j]);
-            f[8] -= dl[j];
-            f[9] = fmaf(exp_ftz(on[j] ? lr[j] : 0.f), fabsf(u[j]), f[9]);       // |e^lt - e^lr| = e^lr |rho - 1|
-            u[j] = SEQ ? wseq - 1.0f : fminf(u[j], C - 1.0f);
-            p = (on[j] && n == 0) ? u[j] : p;
-            n += on[j] ? 1 : 0;
+            for (int j = 7; j >= 0; --j) pivot = on[j] ? u[j] : pivot;
+            A_pivot = A;
+            dA = 0.f;
+            have_pivot = n > 0;
         }
-        float sv = 0.f, sv2 = 0.f;
+        F2 sv = {0.f, 0.f}, sv2 = {0.f, 0.f};
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float v = on[j] ? u[j] - p : 0.f;
-            sv += v;
-            sv2 = fmaf(v, v, sv2);
+        for (int j = 0; j < 8; j += 2) {
+            const F2 d = sub2(F2{u[j], u[j + 1]}, F2{pivot, pivot});
+            const F2 v = {on[j] ? d.x : 0.f, on[j + 1] ? d.y : 0.f};
+            sv = add2(sv, v);
+            sv2 = fma2(v, v, sv2);
         }
-        add_run(acc, n, p, sv, sv2, A);
+        const float svs = sv.x + sv.y, sv2s = sv2.x + sv2.y, nf = static_cast<float>(n);
+        const float c1 = dA * (1.0f + pivot);                      // x = A v + c1 on every valid row of the group
+        g_v += svs;
+        g_v2 += sv2s;
+        g_dA = fmaf(dA, nf, g_dA);
+        g_dA2 = fmaf(dA * dA, nf, g_dA2);
+        g_x += fmaf(A, svs, c1 * nf);
+        g_x2 += fmaf(A * A, sv2s, fmaf(2.0f * A * c1, svs, c1 * c1 * nf));
+        nrows += n;
         return n;
     };
 
+    // The walk over the block's tiles; the first launch also adds up the valid rows per sequence on the way.
+    constexpr bool count = !EXACT;
     bool failed = false;
-    for (int tile = tile0; tile < tile1; ++tile) {
-        const unsigned k = static_cast<unsigned>(tile - tile0);
-        const unsigned st = k % kMomStages;
-        // the group's sequence, advantage and weight source do not depend on the tile's data: fetched before the wait
-        const int t0 = tile * kMomRows + 8 * tid;
-        seek(t0);
-        const bool single = t0 + 8 <= next_b;          // the usual case: the eight rows belong to one sequence
-        if (single) enter();
-        const uint32_t parity = (k / kMomStages) & 1u;
-        bool ok = mbar_try_wait(&full[st], parity);
-        if (!ok) ok = mbar_wait_slow(&full[st], parity, &abort_flag);
-        int n = 0;
-        if (ok) {
-            const uint8_t* src = stages + st * kMomStageBytes;
-            const float4* pa = reinterpret_cast<const float4*>(src) + 2 * tid;
-            const float4* pb = reinterpret_cast<const float4*>(src + kMomRows * 4) + 2 * tid;
-            const float4 a0 = pa[0], a1 = pa[1], b0 = pb[0], b1 = pb[1];
-            const uint2 mk = reinterpret_cast<const uint2*>(src + kMomRows * 8)[tid];
-            const float lt[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-            const float lr[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-            if (single) {
-                if ((mk.x | mk.y) != 0u) n = add_rows(lt, lr, mk.x, mk.y);
-            } else if ((mk.x | mk.y) != 0u) {
-                const uint64_t m64 = (static_cast<uint64_t>(mk.y) << 32) | mk.x;
-                int j = 0;
-                while (j < 8) {                         // a boundary inside the group: one run of rows per sequence
-                    seek(t0 + j);
-                    const int left = next_b - (t0 + j);
-                    const int j1 = left < 8 - j ? j + left : 8;
-                    enter();
-                    const uint64_t run = (j1 == 8 ? ~uint64_t(0) : (uint64_t(1) << (8 * j1)) - 1u) & ~((uint64_t(1) << (8 * j)) - 1u);
-                    const int nr = add_rows(lt, lr, static_cast<uint32_t>(m64 & run), static_cast<uint32_t>((m64 & run) >> 32));
-                    if (n_valid_seq && nr > 0) atomicAdd(&n_valid_seq[sq], nr);
-                    j = j1;
-                }
-            }
-            if ((k & 7u) == 7u) {                       // at most 64 rows per fp32 run of the first-order sums
-                acc[3] += static_cast<double>(f[3]); f[3] = 0.f;
-                acc[8] += static_cast<double>(f[8]); f[8] = 0.f;
-                acc[9] += static_cast<double>(f[9]); f[9] = 0.f;
-            }
-        }
-        if (n_valid_seq) {
-            // valid rows per sequence: a warp's 256-row strip usually lies in one sequence, whose count lane 0 keeps in
-            // a register until the strip moves on (integer atomics: the result does not depend on their order)
-            const int sq0 = __shfl_sync(0xffffffffu, sq, 0);
-            if (__all_sync(0xffffffffu, single && sq == sq0)) {
-                const int tot = __reduce_add_sync(0xffffffffu, n);
-                if (lane == 0) {
-                    if (sq0 != wsq) {
-                        if (wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
-                        wsq = sq0;
-                        wcnt = 0;
+    {
+        constexpr int base = 0;
+        int issued = tile0;                             // first tile not yet requested (thread 0)
+        if (tid == 0)
+            for (; issued < tile1 && issued < tile0 + kMomStages; ++issued) issue(issued, (base + issued - tile0) % kMomStages);
+        for (int tile = tile0; tile < tile1; ++tile) {
+            const unsigned k = static_cast<unsigned>(base + tile - tile0);
+            const unsigned st = k % kMomStages;
+            // the group's sequence, advantage and weight source do not depend on the tile's data: fetched before the wait
+            const int t0 = tile * kMomRows + 8 * tid;
+            seek(t0);
+            const bool single = t0 + 8 <= next_b;          // the usual case: the eight rows belong to one sequence
+            if (single) enter();
+            const uint32_t parity = (k / kMomStages) & 1u;
+            bool ok = mbar_try_wait(&full[st], parity);
+            if (!ok) ok = mbar_wait_slow(&full[st], parity, &abort_flag);
+            int n = 0;
+            if (ok) {
+                const uint8_t* src = stages + st * kMomStageBytes;
+                const float4* pa = reinterpret_cast<const float4*>(src) + 2 * tid;
+                const float4* pb = reinterpret_cast<const float4*>(src + kMomRows * 4) + 2 * tid;
+                const float4 a0 = pa[0], a1 = pa[1], b0 = pb[0], b1 = pb[1];
+                const uint2 mk = reinterpret_cast<const uint2*>(src + kMomRows * 8)[tid];
+                const float lt[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                const float lr[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                if (single) {
+                    if ((mk.x | mk.y) != 0u) n = add_rows(lt, lr, mk.x, mk.y);
+                } else if ((mk.x | mk.y) != 0u) {
+                    const uint64_t m64 = (static_cast<uint64_t>(mk.y) << 32) | mk.x;
+                    int j = 0;
+                    while (j < 8) {                         // a boundary inside the group: one run of rows per sequence
+                        seek(t0 + j);
+                        const int left = next_b - (t0 + j);
+                        const int j1 = left < 8 - j ? j + left : 8;
+                        enter();
+                        const uint64_t run = (j1 == 8 ? ~uint64_t(0) : (uint64_t(1) << (8 * j1)) - 1u) & ~((uint64_t(1) << (8 * j)) - 1u);
+                        const int nr = add_rows(lt, lr, static_cast<uint32_t>(m64 & run), static_cast<uint32_t>((m64 & run) >> 32));
+                        if (count && n_valid_seq && nr > 0) atomicAdd(&n_valid_seq[sq], nr);
+                        j = j1;
                     }
-                    wcnt += tot;
                 }
-            } else if (single && n > 0) {
-                atomicAdd(&n_valid_seq[sq], n);
             }
+            if (count && n_valid_seq) {
+                // valid rows per sequence: a warp's 256-row strip usually lies in one sequence, whose count lane 0 keeps in
+                // a register until the strip moves on (integer atomics: the result does not depend on their order)
+                const int sq0 = __shfl_sync(0xffffffffu, sq, 0);
+                if (__all_sync(0xffffffffu, single && sq == sq0)) {
+                    const int tot = __reduce_add_sync(0xffffffffu, n);
+                    if (lane == 0) {
+                        if (sq0 != wsq) {
+                            if (wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
+                            wsq = sq0;
+                            wcnt = 0;
+                        }
+                        wcnt += tot;
+                    }
+                } else if (single && n > 0) {
+                    atomicAdd(&n_valid_seq[sq], n);
+                }
+            }
+            // everyone is done with the stage (or someone gave up): the stage can take the tile three ahead
+            if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
+            if (tid == 0 && issued < tile1) { issue(issued, st); ++issued; }
         }
-        // everyone is done with the stage (or someone gave up): the stage can take the tile three ahead
-        if (__syncthreads_or(ok ? 0 : 1)) { failed = true; break; }
-        if (tid == 0 && issued < tile1) { issue(issued, st); ++issued; }
+        if (failed && tid == 0) {
+            // let the copies still in flight land before the block's shared memory is given up
+            for (int i = 0; i < issued - tile0; ++i)
+                if (issued - tile0 - i <= kMomStages) {
+                    const unsigned q = static_cast<unsigned>(base + i);
+                    mbar_wait_drain(&full[q % kMomStages], (q / kMomStages) & 1u);
+                }
+        }
     }
-    if (failed && tid == 0) {
-        // let the copies still in flight land before the block's shared memory is given up
-        for (int k = 0; k < issued - tile0; ++k)
-            if (issued - tile0 - k <= kMomStages) mbar_wait_drain(&full[k % kMomStages], static_cast<uint32_t>((k / kMomStages) & 1));
-    }
-    if (n_valid_seq && lane == 0 && wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
+    if (count && n_valid_seq && lane == 0 && wsq >= 0 && wcnt > 0) atomicAdd(&n_valid_seq[wsq], wcnt);
     // rows after the last whole tile: the first threads of the grid, one row each
     for (int t = ntiles * kMomRows + static_cast<int>(blockIdx.x * blockDim.x) + tid; t < T; t += gridDim.x * blockDim.x) {
         if (!mask[t]) continue;
@@ -870,16 +995,34 @@ __global__ void __launch_bounds__(kDiagThreads, 4) moments_staged_kernel(const f
         enter();
         const float lt[8] = {lp_train[t], 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, lr[8] = {lp_roll[t], 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         add_rows(lt, lr, 1u, 0u);
-        if (n_valid_seq) atomicAdd(&n_valid_seq[sq], 1);
+        if (count && n_valid_seq) atomicAdd(&n_valid_seq[sq], 1);
     }
-    acc[3] += static_cast<double>(f[3]);
-    acc[8] += static_cast<double>(f[8]);
-    acc[9] += static_cast<double>(f[9]);
+    double acc[10];
+    {
+        // from the shifted sums to the sums of w, w^2, A, A^2, A w, (A w)^2 in fp64, once per thread:
+        // w = P + v with P = 1 + pivot;  A = Ap + dA;  A w = K + x with K = Ap P
+        const double P = 1.0 + static_cast<double>(pivot), Ap = static_cast<double>(A_pivot), K = Ap * P;
+        const double N = static_cast<double>(nrows);
+        const double SV = static_cast<double>(g_v), SDA = static_cast<double>(g_dA), SX = static_cast<double>(g_x);
+        acc[0] = N;
+        acc[1] = fma(P, N, SV);
+        acc[2] = static_cast<double>(g_v2) + P * fma(P, N, 2.0 * SV);
+        acc[3] = static_cast<double>(f3);
+        acc[4] = fma(Ap, N, SDA);
+        acc[5] = static_cast<double>(g_dA2) + Ap * fma(Ap, N, 2.0 * SDA);
+        acc[6] = fma(K, N, SX);
+        acc[7] = static_cast<double>(g_x2) + K * fma(K, N, 2.0 * SX);
+        acc[8] = -(static_cast<double>(f8p.x) + static_cast<double>(f8p.y));
+        acc[9] = static_cast<double>(f9);
+    }
     if (failed) acc[0] = __longlong_as_double(0x7ff8000000000000LL);     // a NaN count marks the batch as not reduced
+    // slots 10 and 11: what the second launch looks at (no moments; the reductions over the blocks leave them out)
+    const double big = EXACT ? 0.0 : block_sum(static_cast<double>(nbig), scratch);
+    const double small = EXACT ? 0.0 : block_sum(static_cast<double>(nsmall), scratch);
 #pragma unroll
     for (int i = 0; i < kNumMoments; ++i) {
         const double tot = i < 10 ? block_sum(acc[i < 10 ? i : 0], scratch) : 0.0;
-        if (tid == 0) partials[blockIdx.x * kNumMoments + i] = tot;
+        if (tid == 0) partials[blockIdx.x * kNumMoments + i] = i == 10 ? big : i == 11 ? small : tot;
     }
 }
 
@@ -944,7 +1087,7 @@ __global__ void diag_finalize_kernel(const double* __restrict__ partials, int nb
 __global__ void moments_reduce_kernel(const double* __restrict__ partials, int nblocks, double* __restrict__ moments) {
     if (blockIdx.x != 0) return;
     const int i = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const double m = warp_ordered_sum(partials, nblocks, kNumMoments, i, lane);
+    const double m = i < 10 ? warp_ordered_sum(partials, nblocks, kNumMoments, i, lane) : 0.0;   // 10, 11 are no moments
     if (lane == 0) moments[i] = m;
 }
 
@@ -1090,12 +1233,15 @@ void launch_moments_kernel(const float* lp_train, const float* lp_roll, const ui
                            float* seq_logw, cudaStream_t stream) {
     if (seq_logw && S > 0) seq_logw_kernel<<<(S + 7) / 8, 256, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, S, seq_logw);
     if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask) && reinterpret_cast<uintptr_t>(mask) % 16 == 0 && T < (int64_t(1) << 31) - 2 * kMomRows) {      // 32-bit row indices inside
-        if (seq_logw)
-            moments_staged_kernel<true><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
-                                                                                  static_cast<int>(T), S, C, partials, n_valid_seq, seq_logw);
-        else
-            moments_staged_kernel<false><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv,
-                                                                                   static_cast<int>(T), S, C, partials, n_valid_seq, seq_logw);
+        // the fast form, then the exact form for the blocks whose gaps were all tiny (usually none: those blocks return at once)
+        const int Ti = static_cast<int>(T);
+        if (seq_logw) {
+            moments_staged_kernel<true, false><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, Ti, S, C, partials, n_valid_seq, seq_logw);
+            moments_staged_kernel<true, true><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, Ti, S, C, partials, n_valid_seq, seq_logw);
+        } else {
+            moments_staged_kernel<false, false><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, Ti, S, C, partials, n_valid_seq, seq_logw);
+            moments_staged_kernel<false, true><<<kDiagBlocks, kDiagThreads, kMomSmemBytes, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, Ti, S, C, partials, n_valid_seq, seq_logw);
+        }
     } else if (vec4_ok(lp_train, lp_roll, nullptr, nullptr, mask))
         moments_kernel<4><<<kDiagBlocks, kDiagThreads, 0, stream>>>(lp_train, lp_roll, mask, seq_offsets, adv, T, S, C, partials,
                                                                       n_valid_seq, seq_logw);
@@ -1118,9 +1264,13 @@ void launch_rectify_kernel(const float* lp_train, const float* lp_roll, const ui
 }  // namespace
 
 cudaError_t stream_prepare() {
-    cudaError_t e = cudaFuncSetAttribute(moments_staged_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMomSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(moments_staged_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMomSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(moments_staged_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMomSmemBytes);
+    e = cudaFuncSetAttribute(moments_staged_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMomSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(moments_staged_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMomSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(moments_staged_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMomSmemBytes);
 }
 
 // ------------------------------------------------------------------------------------------------ launchers
