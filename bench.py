@@ -260,14 +260,17 @@ def measure_rank(args, rank: int, world: int, local: int) -> dict:
         batch = packed
     T, n_valid = batch.T, batch.n_valid
     params = ais.default_params(vocab_chunk=w.vocab_chunk)
+    if args.w_dv:
+        batch.W = batch.W.t().contiguous()                             # the same head stored [d, V]
     step = ais.AisStep(T, w.d, w.V, w.P, w.G, w.block, device=dev, params=params, workspace_bytes_cap=args.workspace_gb << 30,
-                       group=(dist.group.WORLD if world > 1 else None), P_total=w.P * world)
+                       group=(dist.group.WORLD if world > 1 else None), P_total=w.P * world,
+                       w_layout=ais.W_DV if args.w_dv else ais.W_VD)
     offs = batch.seq_offsets.to(dev)
     rew = batch.rewards.to(dev)
     stream = torch.cuda.current_stream(dev)
 
     # variant (not the headline step): also produce the LM-head weight gradient, one more T x d x V pass
-    dW_buf = torch.empty(w.V, w.d, dtype=torch.float32, device=dev) if args.with_dw else None
+    dW_buf = torch.empty((w.d, w.V) if args.w_dv else (w.V, w.d), dtype=torch.float32, device=dev) if args.with_dw else None
 
     def one_step(ev=None):
         marks = []
@@ -280,7 +283,7 @@ def measure_rank(args, rank: int, world: int, local: int) -> dict:
         mark()
         ais.quantize_fp8(batch.H, w.block, step.qH, step.sH)
         mark()
-        ais.quantize_fp8(batch.W, w.block, step.qW, step.sW)
+        step.quantize_weights(batch.W)
         mark()
         ais.logprob_fwd(step.shape, step.params, batch.H, batch.W, None, None, None, None, batch.tokens, batch.mask,
                         step.lp_train, step.lse_train, None, None, step.status, step.workspace)
@@ -303,7 +306,7 @@ def measure_rank(args, rank: int, world: int, local: int) -> dict:
     # the HBM-bound kernels timed alone, before the long power-capped loop (burst conditions, like the copy that
     # measured the bandwidth they are compared with); inside the step they are bound by launch latency
     streaming = None
-    if rank == 0 and world == 1 and w.block > 0 and not args.prompts and not args.no_streaming:
+    if rank == 0 and world == 1 and w.block > 0 and not args.prompts and not args.no_streaming and not args.w_dv:
         streaming = streaming_scale(dev, batch.W, w.block, args.streaming_rows, H=batch.H)
     for _ in range(args.warmup):
         one_step()
@@ -636,6 +639,8 @@ def build_parser() -> argparse.ArgumentParser:
                     help="variant (not the headline workload): microscaling FP8, power-of-two scale per 32 elements")
     ap.add_argument("--fp8-per-tensor", action="store_true",
                     help="variant (not the headline workload): per-tensor dynamic FP8 scaling instead of per-block scales")
+    ap.add_argument("--w-dv", action="store_true",
+                    help="variant (not the headline layout): the LM head stored [d, V] instead of [V, d]")
     ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
                     help="process-group backend of the ranks; gloo only together with --measure (tests of the rank logic on CPU)")
     ap.add_argument("--measure", default="",

@@ -25,7 +25,8 @@
  *    out, no valid token) are OR-ed into the caller's `dev_status` word / ais_diag.status_flags and the
  *    affected outputs take their documented neutral values; the kernels never trap.
  *  - Layouts: H is row-major [T, ldh] bf16 (ldh >= d).  W is row-major [V, ldw] bf16, one row per
- *    vocabulary entry (the layout of a torch lm_head.weight), so logits are z = H W^T.
+ *    vocabulary entry (the layout of a torch lm_head.weight), so logits are z = H W^T; with
+ *    ais_shape.w_layout = AIS_W_DV it is row-major [d, ldw] instead (z = H W).
  *    FP8 codes keep the layout of their source matrix ([rows, cols] uint8).  Scales are "block-major":
  *    scales[kb * ld_scales + row] is the scale of block kb (elements kb*B .. kb*B+B-1 along d) of `row`.
  *  - Rows with mask[t] == 0 yield lp = 0, lse = 0, rho = 1, w_tilde = 1 and a zero row of dH.
@@ -43,7 +44,7 @@
 extern "C" {
 #endif
 
-#define AIS_VERSION 100
+#define AIS_VERSION 110
 
 /* status codes */
 #define AIS_OK                 0
@@ -65,6 +66,9 @@ extern "C" {
                                       as a row with lp_train = lp_roll                        */
 #define AIS_FLAG_TIMEOUT      8u   /* a bounded device-side wait ran out; outputs undefined */
 
+#define AIS_W_VD 0                /* ais_shape.w_layout: W is row-major [V, ldw], one row per vocabulary entry     */
+#define AIS_W_DV 1                /* ais_shape.w_layout: W is row-major [d, ldw], one row per hidden unit          */
+
 #define AIS_FP8_MX32 (-32)        /* ais_shape.fp8_block: microscaling FP8, E8M0 scale per 32 elements */
 #define AIS_FP4_MX32 (-4)         /* ais_shape.fp8_block: microscaling FP4 (E2M1 elements), E8M0 scale per 32    */
 
@@ -79,8 +83,13 @@ typedef struct ais_shape {
                              AIS_FP8_MX32 = power-of-two scale per 32 (ais_quantize_mxfp8);
                              AIS_FP4_MX32 = the same with 4-bit elements (ais_quantize_mxfp4)*/
     int32_t P_total;      /* prompts over all data-parallel ranks (loss normaliser); 0 = P    */
+    int32_t w_layout;     /* AIS_W_VD (0): W [V, ldw] as a torch lm_head.weight; AIS_W_DV: W [d, ldw], the form in
+                             which the paper writes the head.  Both give the same log-probs bit for bit (the
+                             tensor cores read either storage order; nothing is transposed in memory).  AIS_W_DV:
+                             ldw >= V, a multiple of 8; V a multiple of 8; fp8_block 32, 64 or 128 only; W's codes
+                             are [V, d] with row stride d (ais_quantize_fp8_cols); dW comes out [d, lddw].  */
     int64_t ldh;          /* row stride of H (and of its codes) in elements                  */
-    int64_t ldw;          /* row stride of W (and of its codes) in elements                  */
+    int64_t ldw;          /* row stride of W in elements (AIS_W_VD: also of its codes)       */
 } ais_shape;
 
 /* Hyper-parameters (Algorithm 1 'Require' line; Appendix 'AIS hyperparameters'; PPO clipping of the
@@ -168,6 +177,16 @@ size_t ais_workspace_min_bytes(const ais_shape* shape, const ais_params* params)
  */
 int ais_quantize_fp8(const void* x, int64_t rows, int64_t cols, int64_t ld, int block,
                      uint8_t* codes, int64_t ldq, float* scales, int64_t lds, void* stream);
+
+/*
+ * The same quantisation for a matrix whose blocks run down its columns: an LM head stored [d, V] (AIS_W_DV).
+ * x       [rows, ld] bf16, row-major; rows (= d) a multiple of 128; cols (= V) a multiple of 8
+ * codes   [cols, ldq] uint8: TRANSPOSED, codes[v, k] belongs to x[k, v]; ldq >= rows, a multiple of 16   (written)
+ * scales  [rows/block, lds] float: scales[kb, v] is the scale of x[kb*block .. kb*block+block-1, v]       (written)
+ * The result is element for element what ais_quantize_fp8 gives for the transposed matrix.
+ */
+int ais_quantize_fp8_cols(const void* x, int64_t rows, int64_t cols, int64_t ld, int block,
+                          uint8_t* codes, int64_t ldq, float* scales, int64_t lds, void* stream);
 
 /*
  * Per-tensor dynamic scaling, the setting of the paper's own rollouts (Appendix "FP8 rollout"): one scale
@@ -284,7 +303,7 @@ int ais_diag_finalize(const ais_shape* shape, const ais_params* params, const do
  * The softmax is recomputed from H, W and lse_train; w_tilde, A, lp_old and lp_ref are constants.
  * dH [T, ldh] bf16 (written, zero rows where mask = 0), loss: one float on the device (may be NULL),
  * diag: if not NULL its `loss` and `kl_ref` fields are written too.
- * dW (may be NULL): gradient with respect to the LM head in W's layout, [V, lddw] fp32,
+ * dW (may be NULL): gradient with respect to the LM head in W's layout, [V, lddw] fp32 ([d, lddw] with AIS_W_DV),
  *     dW[v,:] = sum_t c_t (softmax(z[t,:])[v] - [v == tokens[t]]) H[t,:]
  * overwritten when dw_accumulate == 0, added to otherwise (micro-batch accumulation); costs one more
  * T x d x V tensor-core pass over the scratch that dH uses.

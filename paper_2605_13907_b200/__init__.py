@@ -8,6 +8,6 @@ calls raise.
 
 from .binding import (  # noqa: F401
     AisError, Params, Diag, Shape, lib, lib_path, default_params, make_shape, workspace_bytes, workspace_min_bytes,
-    quantize_fp8, FP8_MX32, FP4_MX32, mx_scale_bytes, logprob_fwd, diagnostics, loss_bwd, AisStep, logprob_train_static, STATIC_MAX_ROWS, diag_moments, diag_finalize, NUM_MOMENTS, RowCompaction,
+    quantize_fp8, quantize_fp8_cols, W_VD, W_DV, FP8_MX32, FP4_MX32, mx_scale_bytes, logprob_fwd, diagnostics, loss_bwd, AisStep, logprob_train_static, STATIC_MAX_ROWS, diag_moments, diag_finalize, NUM_MOMENTS, RowCompaction,
     FLAG_EMPTY, FLAG_TOKEN_RANGE, FLAG_NONFINITE, FLAG_TIMEOUT, set_wait_cycles,
 )

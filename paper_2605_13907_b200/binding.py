@@ -22,7 +22,7 @@ class AisError(RuntimeError):
 
 class Shape(C.Structure):
     _fields_ = [("T", C.c_int64), ("d", C.c_int32), ("V", C.c_int32), ("P", C.c_int32), ("G", C.c_int32),
-                ("fp8_block", C.c_int32), ("P_total", C.c_int32), ("ldh", C.c_int64), ("ldw", C.c_int64)]
+                ("fp8_block", C.c_int32), ("P_total", C.c_int32), ("w_layout", C.c_int32), ("ldh", C.c_int64), ("ldw", C.c_int64)]
 
 
 class Params(C.Structure):
@@ -65,6 +65,8 @@ def lib() -> C.CDLL:
             f.argtypes = [C.POINTER(Shape), C.POINTER(Params)]
         L.ais_quantize_fp8.restype = C.c_int
         L.ais_quantize_fp8.argtypes = [vp, i64, i64, i64, C.c_int, vp, i64, vp, i64, vp]
+        L.ais_quantize_fp8_cols.restype = C.c_int
+        L.ais_quantize_fp8_cols.argtypes = [vp, i64, i64, i64, C.c_int, vp, i64, vp, i64, vp]
         L.ais_quantize_fp8_tensor.restype = C.c_int
         L.ais_quantize_fp8_tensor.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp]
         L.ais_mx_scale_bytes.restype = sz
@@ -130,9 +132,13 @@ def default_params(**overrides) -> Params:
     return p
 
 
+W_VD, W_DV = 0, 1       # ais_shape.w_layout: W stored [V, d] (a torch lm_head.weight) or [d, V]
+
+
 def make_shape(T: int, d: int, V: int, P: int, G: int, fp8_block: int, ldh: int | None = None, ldw: int | None = None,
-               P_total: int = 0) -> Shape:
-    return Shape(T=T, d=d, V=V, P=P, G=G, fp8_block=fp8_block, P_total=P_total, ldh=ldh or d, ldw=ldw or d)
+               P_total: int = 0, w_layout: int = W_VD) -> Shape:
+    return Shape(T=T, d=d, V=V, P=P, G=G, fp8_block=fp8_block, P_total=P_total, w_layout=w_layout, ldh=ldh or d,
+                 ldw=ldw or (V if w_layout == W_DV else d))
 
 
 def workspace_bytes(shape: Shape, params: Params) -> int:
@@ -189,6 +195,20 @@ def quantize_fp8(x: torch.Tensor, block: int, codes: torch.Tensor | None = None,
         scales = torch.empty(cols // block, max(lds, 4), dtype=torch.float32, device=x.device)
     _check(lib().ais_quantize_fp8(_ptr(x), rows, cols, x.stride(0), block, _ptr(codes), codes.stride(0), _ptr(scales),
                                   scales.stride(0), _stream(x)), "ais_quantize_fp8")
+    return codes, scales
+
+
+def quantize_fp8_cols(x: torch.Tensor, block: int, codes: torch.Tensor | None = None, scales: torch.Tensor | None = None):
+    """x [K, N] bf16 with the blocks running down the columns (an LM head stored [d, V]) ->
+    (codes [N, K] uint8, transposed; scales [K/block, lds] float32, block-major)."""
+    _require_cuda(x, codes, scales)
+    K, N = x.shape
+    if codes is None:
+        codes = torch.empty(N, K, dtype=torch.uint8, device=x.device)
+    if scales is None:
+        scales = torch.empty(K // block, max((N + 3) // 4 * 4, 4), dtype=torch.float32, device=x.device)
+    _check(lib().ais_quantize_fp8_cols(_ptr(x), K, N, x.stride(0), block, _ptr(codes), codes.stride(0), _ptr(scales),
+                                       scales.stride(0), _stream(x)), "ais_quantize_fp8_cols")
     return codes, scales
 
 
@@ -312,11 +332,13 @@ class AisStep:
 
     def __init__(self, T: int, d: int, V: int, P: int, G: int, fp8_block: int, device="cuda", params: Params | None = None,
                  workspace_bytes_cap: int | None = None, want_grad: bool = True, group=None, P_total: int = 0,
-                 ldh: int | None = None, ldw: int | None = None):
+                 ldh: int | None = None, ldw: int | None = None, w_layout: int = W_VD):
         self.device = torch.device(device)
         self.group = group                       # torch.distributed process group: alpha over all its ranks
-        ldh, ldw = ldh or d, ldw or d            # row strides of H / W; their codes and dH use the same strides
-        self.shape = make_shape(T, d, V, P, G, fp8_block, ldh=ldh, ldw=ldw, P_total=P_total)
+        ldh = ldh or d                           # row strides of H / W; H's codes and dH use H's stride
+        ldw = ldw or (V if w_layout == W_DV else d)
+        self.shape = make_shape(T, d, V, P, G, fp8_block, ldh=ldh, ldw=ldw, P_total=P_total, w_layout=w_layout)
+        self.w_layout = w_layout
         self.params = params or default_params()
         S = P * G
         dev = self.device
@@ -336,7 +358,8 @@ class AisStep:
             self.qW = torch.empty(V, ldw // 2, dtype=torch.uint8, device=dev)[:, :d // 2]
         else:
             self.qH = torch.empty(max(T, 1), ldh, dtype=torch.uint8, device=dev)[:, :d]
-            self.qW = torch.empty(V, ldw, dtype=torch.uint8, device=dev)[:, :d]
+            # a [d, V] head is quantised into codes [V, d] of row stride d; a [V, d] head's codes share its stride
+            self.qW = torch.empty(V, d if w_layout == W_DV else ldw, dtype=torch.uint8, device=dev)[:, :d]
         if fp8_block in (FP8_MX32, FP4_MX32):
             self.sH = torch.empty(mx_scale_bytes(T, d), dtype=torch.uint8, device=dev)
             self.sW = torch.empty(mx_scale_bytes(V, d), dtype=torch.uint8, device=dev)
@@ -361,7 +384,10 @@ class AisStep:
         self.w_quantized = False
 
     def quantize_weights(self, W: torch.Tensor) -> None:
-        quantize_fp8(W, self.shape.fp8_block, self.qW, self.sW)
+        if self.w_layout == W_DV:
+            quantize_fp8_cols(W, self.shape.fp8_block, self.qW, self.sW)
+        else:
+            quantize_fp8(W, self.shape.fp8_block, self.qW, self.sW)
         self.w_quantized = True
 
     def forward(self, H, W, tokens, mask, requantize_w: bool = True) -> None:

@@ -97,8 +97,16 @@ int check_shape(const ais_shape* s) {
         return AIS_ERR_SHAPE;
     if (s->fp8_block == AIS_FP4_MX32 && (s->d % 256 != 0 || s->ldh % 32 != 0 || s->ldw % 32 != 0)) return AIS_ERR_SHAPE;
     if (s->fp8_block > 0 && s->d % s->fp8_block != 0) return AIS_ERR_SHAPE;
-    if (s->ldh < s->d || s->ldw < s->d) return AIS_ERR_SHAPE;
-    if (s->ldh % 16 != 0 || s->ldw % 16 != 0) return AIS_ERR_ALIGN;
+    if (s->w_layout != AIS_W_VD && s->w_layout != AIS_W_DV) return AIS_ERR_SHAPE;
+    if (s->w_layout == AIS_W_DV) {
+        // [d, V] head: the block-scaled variants and the per-tensor variant take the [V, d] layout only
+        if (s->fp8_block != 32 && s->fp8_block != 64 && s->fp8_block != 128) return AIS_ERR_SHAPE;
+        if (s->ldh < s->d || s->ldw < s->V) return AIS_ERR_SHAPE;
+        if (s->ldh % 16 != 0 || s->ldw % 8 != 0) return AIS_ERR_ALIGN;
+    } else {
+        if (s->ldh < s->d || s->ldw < s->d) return AIS_ERR_SHAPE;
+        if (s->ldh % 16 != 0 || s->ldw % 16 != 0) return AIS_ERR_ALIGN;
+    }
     if (static_cast<int64_t>(s->P) * s->G > (1 << 24)) return AIS_ERR_SHAPE;
     if (s->P_total != 0 && (s->P_total < s->P || static_cast<int64_t>(s->P_total) * s->G > (int64_t(1) << 30))) return AIS_ERR_SHAPE;
     return AIS_OK;
@@ -231,6 +239,20 @@ int ais_quantize_fp8(const void* x, int64_t rows, int64_t cols, int64_t ld, int 
                : AIS_ERR_DEVICE;
 }
 
+int ais_quantize_fp8_cols(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes, int64_t ldq,
+                          float* scales, int64_t lds, void* stream) {
+    if (!x || !codes || !scales) return AIS_ERR_NULL;
+    if (rows < 0 || cols < 0 || (block != 32 && block != 64 && block != 128)) return AIS_ERR_SHAPE;
+    if (rows % 128 != 0 || cols % 8 != 0 || ld < cols || ldq < rows || lds < cols) return AIS_ERR_SHAPE;
+    if (ld % 8 != 0 || ldq % 16 != 0 || !aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 4)) return AIS_ERR_ALIGN;
+    if (cols > (int64_t(1) << 31) - 1024 || rows > (int64_t(1) << 24)) return AIS_ERR_SHAPE;
+    int st = device_setup(nullptr);
+    if (st != AIS_OK) return st;
+    return launch_quantize_cols(x, rows, cols, ld, block, codes, ldq, scales, lds, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? AIS_OK
+               : AIS_ERR_DEVICE;
+}
+
 int ais_quantize_fp8_tensor(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq, float* scale,
                             void* stream) {
     if (!x || !codes || !scale) return AIS_ERR_NULL;
@@ -339,12 +361,16 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     const uint64_t T = static_cast<uint64_t>(shape->T), V = static_cast<uint64_t>(shape->V), d = static_cast<uint64_t>(shape->d);
 
     CUtensorMap tmA, tmB, tmSA, tmSB;
+    const bool dv = shape->w_layout == AIS_W_DV;
     if (do_train) {
+        // W [V, d]: K-major boxes of 64 hidden units x 256 vocabulary rows.  W [d, V]: the vocabulary is the contiguous
+        // axis, boxes of 64 vocabulary columns x 64 hidden units (four of them per stage)
         if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, H, d, T, shape->ldh * 2, 64, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B))
+            !(dv ? make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, V, d, shape->ldw * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)
+                 : make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B)))
             return AIS_ERR_DEVICE;
         a.ksteps = shape->d / 64;
-        if (launch_lmhead(kFwdBf16, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
+        if (launch_lmhead(dv ? kFwdBf16Dv : kFwdBf16, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_train, lse_train, dev_status, s) !=
             cudaSuccess)
             return AIS_ERR_DEVICE;
@@ -381,7 +407,7 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
     } else if (do_roll) {
         const uint64_t nkb = d / shape->fp8_block;
         if (!make_tmap(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, qH, d, T, shape->ldh, 128, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, qW, d, V, shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, qW, d, V, dv ? d : shape->ldw, 128, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
             !make_tmap(&tmSA, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sH, T, nkb, ldsH * 4, kBM, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE) ||
             !make_tmap(&tmSB, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sW, V, nkb, ldsW * 4, kBN, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE))
             return AIS_ERR_DEVICE;
@@ -476,7 +502,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
     if (!H || !W || !tokens || !mask || !seq_offsets || !lse_train || !lp_train || !adv || !w_tilde || !dH) return AIS_ERR_NULL;
     if (!aligned(H, 16) || !aligned(W, 16) || !aligned(dH, 16)) return AIS_ERR_ALIGN;
     if (dW && (!aligned(dW, 16) || lddw % 4 != 0)) return AIS_ERR_ALIGN;
-    if (dW && lddw < shape->d) return AIS_ERR_SHAPE;
+    if (dW && lddw < (shape->w_layout == AIS_W_DV ? shape->V : shape->d)) return AIS_ERR_SHAPE;
     const Layout L = make_layout(shape, params);
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.fixed_bytes + static_cast<size_t>(kBM) * L.u_row_bytes)
         return AIS_ERR_WORKSPACE;
@@ -505,9 +531,16 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
     __nv_bfloat16* U = reinterpret_cast<__nv_bfloat16*>(ws + L.off_u);
     const uint64_t V = static_cast<uint64_t>(shape->V), d = static_cast<uint64_t>(shape->d);
 
+    // tmW_k: W for the recompute pass (contraction over d), tmW_n: W for the dH pass (contraction over V).  With W [V, d]
+    // the first is K-major (boxes of 64 hidden units x 256 vocabulary rows) and the second MN-major (64 x 64 boxes);
+    // with W [d, V] it is the other way round (64 x 64 boxes of vocabulary columns x hidden units; boxes of 64 vocabulary
+    // columns x 256 hidden units).
+    const bool dv = shape->w_layout == AIS_W_DV;
     CUtensorMap tmW_k, tmW_n, tmU;
-    if (!make_tmap(&tmW_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap(&tmW_n, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+    if (!(dv ? make_tmap(&tmW_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, V, d, shape->ldw * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)
+             : make_tmap(&tmW_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B)) ||
+        !(dv ? make_tmap(&tmW_n, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, V, d, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B)
+             : make_tmap(&tmW_n, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) ||
         !make_tmap(&tmU, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, U, V, static_cast<uint64_t>(blk_rows), L.ldU * 2, 64, kBM,
                    CU_TENSOR_MAP_SWIZZLE_128B))
         return AIS_ERR_DEVICE;
@@ -542,7 +575,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
         a.nsplit = L.nsplit;
         a.ksteps = shape->d / 64;
         int units = a.n_row_tiles * a.nsplit;
-        if (launch_lmhead(kBwdP, tmH, tmW_k, tmH, tmW_k, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
+        if (launch_lmhead(dv ? kBwdPDv : kBwdP, tmH, tmW_k, tmH, tmW_k, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
             return AIS_ERR_DEVICE;
         // dH = c (.) (U W)
         a.ncols = shape->d;
@@ -551,7 +584,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
         a.nsplit = 1;
         a.ksteps = (shape->V + 63) / 64;
         units = a.n_row_tiles * a.n_col_tiles;
-        if (launch_lmhead(kBwdDh, tmU, tmW_n, tmU, tmW_n, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
+        if (launch_lmhead(dv ? kBwdDhDv : kBwdDh, tmU, tmW_n, tmU, tmW_n, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
             return AIS_ERR_DEVICE;
         if (dW) {
             // dW (+)= U^T H over the rows of this pass: both operands are read with the rows as contraction axis;
@@ -562,18 +595,22 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
                 !make_tmap(&tmH_t, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Hc, d, static_cast<uint64_t>(rows), shape->ldh * 2, 64, 64,
                            CU_TENSOR_MAP_SWIZZLE_128B))
                 return AIS_ERR_DEVICE;
+            // output in W's layout: [V, d] = U^T H, or [d, V] = H^T U with the two operands changing places
+            const int out_rows = dv ? shape->d : shape->V, out_cols = dv ? shape->V : shape->d;
             LmheadArgs w = a;
-            w.rows = shape->V;
+            w.rows = out_rows;
             w.row0 = 0;
-            w.n_row_tiles = static_cast<int32_t>((shape->V + kDhRows - 1) / kDhRows);
-            w.ncols = shape->d;
-            w.n_col_tiles = (shape->d + kBN - 1) / kBN;
+            w.n_row_tiles = static_cast<int32_t>((out_rows + kDhRows - 1) / kDhRows);
+            w.ncols = out_cols;
+            w.n_col_tiles = (out_cols + kBN - 1) / kBN;
             w.ksteps = static_cast<int32_t>((rows + 63) / 64);
             w.dW = dW;
             w.lddw = lddw;
             w.dw_accumulate = (dw_accumulate || r0 > 0) ? 1 : 0;
             units = w.n_row_tiles * w.n_col_tiles;
-            if (launch_lmhead(kBwdDw, tmU_t, tmH_t, tmU_t, tmH_t, w, units < num_sms ? units : num_sms, s) != cudaSuccess)
+            const CUtensorMap& tmRow = dv ? tmH_t : tmU_t;
+            const CUtensorMap& tmCol = dv ? tmU_t : tmH_t;
+            if (launch_lmhead(kBwdDw, tmRow, tmCol, tmRow, tmCol, w, units < num_sms ? units : num_sms, s) != cudaSuccess)
                 return AIS_ERR_DEVICE;
         }
     }

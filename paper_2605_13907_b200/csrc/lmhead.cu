@@ -40,7 +40,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile uint32_t* issued_slot = tmem_slot + 2;     // stage fills the producer has requested (written when it leaves its loop)
 
-    constexpr bool TWO_ACC = (MODE == kBwdDh || MODE == kBwdDw);                // two 128-row tiles per CTA, one B slice
+    constexpr int BASE = base_mode(MODE);                                       // what is computed, whatever W's layout
+    constexpr bool B_MN = b_mn_major(MODE);                                     // B tile arrives as four 64-column boxes
+    constexpr bool TWO_ACC = (BASE == kBwdDh || BASE == kBwdDw);                // two 128-row tiles per CTA, one B slice
     constexpr int STG = TWO_ACC ? kDhStages : kStages;                          // depth of the stage ring
     constexpr int STG_BYTES = TWO_ACC ? kDhStageBytes : kStageBytes;
     constexpr int A_BYTES = TWO_ACC ? 2 * kAStageBytes : kAStageBytes;
@@ -84,8 +86,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             uint32_t issued = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
-                const Unit w = decode_unit<MODE>(a, u);
-                if (!unit_active<MODE>(a, w)) continue;
+                const Unit w = decode_unit<BASE>(a, u);
+                if (!unit_active<BASE>(a, w)) continue;
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
                     for (int ks = 0; ks < a.ksteps; ++ks) {
                         if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
@@ -108,10 +110,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             bulk_load(sS + KC * kMxChunkBytes, a.sf_b + (static_cast<int64_t>(t) * a.nk4 + k4) * (2 * kMxChunkBytes),
                                       KC * 2 * kMxChunkBytes, &full[st.idx]);
                         }
-                        if (MODE == kBwdDh) {
+                        if (BASE == kBwdDh) {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kDhRows);
                             tma_load_2d(sA + kAStageBytes, &tmA, &full[st.idx], kelem, w.rt * kDhRows + kBM);
-                        } else if (MODE == kBwdDw) {
+                        } else if (BASE == kBwdDw) {
                             // A is U[t, v]: the output row v is the contiguous axis -> four 64-wide boxes of 64 rows t
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
@@ -119,9 +121,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         } else {
                             tma_load_2d(sA, &tmA, &full[st.idx], kelem, w.rt * kBM);
                         }
-                        if (MODE == kBwdDh || MODE == kBwdDw) {
-                            // B is W[v, n] (dH) or H[t, n] (dW): n (the output column) is the contiguous axis -> four
-                            // 64-column boxes
+                        if (B_MN) {
+                            // B is stored with the output column as the contiguous axis (W[v, n] in the dH pass, H[t, n] in
+                            // the dW pass, W[k, v] in the forward passes over a [d, V] head) -> four 64-column boxes
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
                                 tma_load_2d(sB + j * (kBStageBytes / 4), &tmB, &full[st.idx], t * kBN + j * 64, kelem);
@@ -141,12 +143,12 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         if (lane == 0) {
             constexpr uint32_t idesc =
                 (MODE == kFwdFp8T || MX) ? make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0)
-                                  : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, MODE == kBwdDw ? 1 : 0, TWO_ACC ? 1 : 0);
+                                  : make_idesc(kFmtBF16, kFmtBF16, kBM, kBN, BASE == kBwdDw ? 1 : 0, B_MN ? 1 : 0);
             Pipe st(STG), tb(NBUF);
             bool ok = true;
             for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
-                const Unit w = decode_unit<MODE>(a, u);
-                if (!unit_active<MODE>(a, w)) continue;
+                const Unit w = decode_unit<BASE>(a, u);
+                if (!unit_active<BASE>(a, w)) continue;
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
                     if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                     tc_fence_after();
@@ -155,16 +157,17 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         tc_fence_after();
                         const uint32_t sA = smem_u32(stage_base + st.idx * STG_BYTES);
                         const uint32_t sB = sA + A_BYTES;
-                        if (MODE == kBwdDh) {
+                        if (BASE == kBwdDh) {
                             // two row tiles share every B slice: accumulators at TMEM columns 0 and 256
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
-                                const uint64_t bdesc = smem_desc_sw128(sB + j * 2048, kBStageBytes / 4, 1024);
+                                const uint64_t bdesc = B_MN ? smem_desc_sw128(sB + j * 2048, kBStageBytes / 4, 1024)
+                                                            : smem_desc_sw128(sB + j * 32, 16, 1024);
                                 const uint32_t accum = (ks > 0 || j > 0) ? 1u : 0u;
                                 mma_f16(tmem_base, smem_desc_sw128(sA + j * 32, 16, 1024), bdesc, idesc, accum);
                                 mma_f16(tmem_base + kBN, smem_desc_sw128(sA + kAStageBytes + j * 32, 16, 1024), bdesc, idesc, accum);
                             }
-                        } else if (MODE == kBwdDw) {
+                        } else if (BASE == kBwdDw) {
                             // both operands have the contraction axis t as rows of 128 bytes: 16 rows (2048 bytes) per
                             // MMA; 64-wide chunks of the output axis are 8 KB apart
 #pragma unroll
@@ -203,7 +206,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 const uint64_t adesc = smem_desc_sw128(sA + j * 32, 16, 1024);
-                                const uint64_t bdesc = smem_desc_sw128(sB + j * 32, 16, 1024);
+                                const uint64_t bdesc = B_MN ? smem_desc_sw128(sB + j * 2048, kBStageBytes / 4, 1024)
+                                                            : smem_desc_sw128(sB + j * 32, 16, 1024);
                                 if (MODE == kFwdFp8T) mma_f8(dcol, adesc, bdesc, idesc, (ks > 0 || j > 0) ? 1u : 0u);
                                 else mma_f16(dcol, adesc, bdesc, idesc, (ks > 0 || j > 0) ? 1u : 0u);
                             }
@@ -236,8 +240,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         Pipe st(STG);
         bool ok = true;
         for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
-            const Unit w = decode_unit<MODE>(a, u);
-            if (!unit_active<MODE>(a, w)) continue;
+            const Unit w = decode_unit<BASE>(a, u);
+            if (!unit_active<BASE>(a, w)) continue;
             for (int t = w.t0; t < w.t1 && ok; ++t) {
                 for (int ks = 0; ks < a.ksteps; ++ks) {
                     if (!mbar_wait_warp(&full[st.idx], st.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
@@ -264,10 +268,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         bool ok = true;
         uint32_t flags = 0;
         for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
-            const Unit w = decode_unit<MODE>(a, u);
-            if (!unit_active<MODE>(a, w)) {
+            const Unit w = decode_unit<BASE>(a, u);
+            if (!unit_active<BASE>(a, w)) {
                 // nothing was loaded or multiplied for this unit: write the neutral output where later passes read it
-                if (MODE == kBwdDh) {
+                if (BASE == kBwdDh) {
 #pragma unroll
                     for (int sub = 0; sub < 2; ++sub) {
                         const int64_t lr = static_cast<int64_t>(w.rt) * kDhRows + sub * kBM + r_in_tile;
@@ -278,7 +282,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                 if (w.t0 * kBN + half * 128 + j * 8 < a.ncols) dst[j] = make_uint4(0, 0, 0, 0);
                         }
                     }
-                } else if (MODE == kBwdP) {
+                } else if (BASE == kBwdP) {
                     const int64_t lr = static_cast<int64_t>(w.rt) * kBM + r_in_tile;
                     if (lr < a.rows) {
                         for (int t = w.t0; t < w.t1; ++t) {
@@ -291,7 +295,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 }
                 continue;       // forward passes: the rows are masked, the merge kernel never reads their partials
             }
-            if (MODE == kBwdDh) {
+            if (BASE == kBwdDh) {
                 // one unit = 256 rows x 256 columns of dH, finished after the whole contraction over the vocabulary
                 if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                 tc_fence_after();
@@ -326,7 +330,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 tb.advance();
                 continue;
             }
-            if (MODE == kBwdDw) {
+            if (BASE == kBwdDw) {
                 // one unit = 256 vocabulary rows x 256 columns of dW after the contraction over this launch's rows
                 if (!mbar_wait_warp(&tfull[0], tb.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                 tc_fence_after();
@@ -378,7 +382,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             const float tscale = (MODE == kFwdFp8T) ? (*a.scale_a) * (*a.scale_b) : 1.f;
             float lse2 = 0.f;
             float cf = 0.f;                                    // recompute: c_t, folded into the scratch
-            if (MODE == kBwdP && row_ok) {
+            if (BASE == kBwdP && row_ok) {
                 lse2 = a.lse[grow] * kLog2e;
                 cf = a.coef[grow];
                 if (cf == 0.f) valid = false;                  // rows without gradient are written as exact zeros
@@ -421,7 +425,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             for (int i = 0; i < 32; ++i) x[i] *= tscale;
                         }
                     }
-                    if (MODE == kFwdBf16 || MODE == kFwdFp8T || MX) {
+                    if (BASE == kFwdBf16 || MODE == kFwdFp8T || MX) {
                         if (y >= col0 && y < col0 + 32) {
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
@@ -441,7 +445,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         for (int i = 0; i < 32; ++i) add += ex2(fmaf(x[i], kLog2e, -m_new));
                         s = fmaf(s, ex2(m2 - m_new), add);
                         m2 = m_new;
-                    } else if (MODE == kBwdP) {
+                    } else if (BASE == kBwdP) {
                         if (row_ok && col0 < a.ncols) {
                             uint32_t pk[16];
 #pragma unroll
@@ -466,7 +470,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 }
                 tb.advance();
             }
-            if (ok && row_ok && (MODE == kFwdBf16 || MODE == kFwdFp8T || MX)) {
+            if (ok && row_ok && (BASE == kFwdBf16 || MODE == kFwdFp8T || MX)) {
                 const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow;
                 a.part_m[o] = m2 * kLn2;
                 a.part_s[o] = s;
@@ -512,6 +516,9 @@ cudaError_t launch_lmhead(int mode, const CUtensorMap& tmA, const CUtensorMap& t
         case kBwdDw:   return launch_mode<kBwdDw>(tmA, tmB, args, num_ctas, stream);
         case kFwdMx:   return launch_mode<kFwdMx>(tmA, tmB, args, num_ctas, stream);
         case kFwdMx4:  return launch_mode<kFwdMx4>(tmA, tmB, args, num_ctas, stream);
+        case kFwdBf16Dv: return launch_mode<kFwdBf16Dv>(tmA, tmB, args, num_ctas, stream);
+        case kBwdPDv:    return launch_mode<kBwdPDv>(tmA, tmB, args, num_ctas, stream);
+        case kBwdDhDv:   return launch_mode<kBwdDhDv>(tmA, tmB, args, num_ctas, stream);
     }
     return cudaErrorInvalidValue;
 }
@@ -531,6 +538,12 @@ cudaError_t lmhead_prepare() {
     e = cudaFuncSetAttribute(lmhead_kernel<kBwdDw>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(lmhead_kernel<kFwdMx>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(lmhead_kernel<kFwdBf16Dv>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(lmhead_kernel<kBwdPDv>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(lmhead_kernel<kBwdDhDv>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(lmhead_kernel<kFwdMx4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }

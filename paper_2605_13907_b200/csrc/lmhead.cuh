@@ -15,8 +15,23 @@ enum LmheadMode : int {
     kFwdFp8T = 4,   // E4M3 codes with one scale per tensor: whole contraction in tensor memory, one multiply after
     kBwdDw   = 5,   // dW += U^T H, contraction over the rows (both operands read with the contraction axis as rows)
     kFwdMx   = 6,   // E4M3 codes with one power-of-two (E8M0) scale per 32 elements: hardware block-scaled MMA
-    kFwdMx4  = 7    // packed E2M1 (FP4) codes with one E8M0 scale per 32 elements
+    kFwdMx4  = 7,   // packed E2M1 (FP4) codes with one E8M0 scale per 32 elements
+    // the same three bf16 passes with W stored [d, V] (one row per hidden unit): the forward passes then read W as an
+    // MN-major B operand (four 64-column boxes per stage, like the dH pass of the other layout) and the dH pass reads it
+    // K-major (like the forward passes of the other layout)
+    kFwdBf16Dv = 8,
+    kBwdPDv    = 9,
+    kBwdDhDv   = 10
 };
+
+// What a mode computes (its epilogue and work-unit shape), whatever the layout of W.
+__host__ __device__ constexpr int base_mode(int mode) {
+    return mode == kFwdBf16Dv ? kFwdBf16 : mode == kBwdPDv ? kBwdP : mode == kBwdDhDv ? kBwdDh : mode;
+}
+// B operand stored with the output column as the contiguous axis (MN-major)?
+__host__ __device__ constexpr bool b_mn_major(int mode) {
+    return mode == kBwdDh || mode == kBwdDw || mode == kFwdBf16Dv || mode == kBwdPDv;
+}
 
 constexpr int kBM = 128;                 // rows per tile (TMEM lanes)
 constexpr int kBN = 256;                 // columns per tile (TMEM columns of one accumulator)

@@ -53,7 +53,7 @@ extern "C" int ais_logprob_train_static(const ais_shape* shape, const void* H, c
                                         const uint8_t* mask, float* lp_train, float* lse_train, uint32_t* dev_status,
                                         void* stream) {
     if (!shape || !H || !W || !tokens || !mask || !lp_train) return AIS_ERR_NULL;
-    if (shape->T < 0 || shape->d <= 0 || shape->V <= 0) return AIS_ERR_SHAPE;
+    if (shape->T < 0 || shape->d <= 0 || shape->V <= 0 || shape->w_layout != AIS_W_VD) return AIS_ERR_SHAPE;
     if (shape->d % 64 != 0 || shape->V % 8 != 0 || shape->ldh < shape->d || shape->ldw < shape->d) return AIS_ERR_SHAPE;
     if (shape->ldh % 8 != 0 || shape->ldw % 8 != 0) return AIS_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(H) | reinterpret_cast<uintptr_t>(W)) % 16 != 0) return AIS_ERR_ALIGN;

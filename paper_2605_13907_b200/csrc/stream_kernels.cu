@@ -141,6 +141,78 @@ __global__ void __launch_bounds__(kQThreads) quantize_kernel(const __nv_bfloat16
 }
 
 // ------------------------------------------------------------------------------------------------
+// The same quantisation for a matrix stored with the blocks running DOWN its columns (an LM head kept as [d, V]):
+// block kb of column v is x[kb B .. kb B + B - 1, v].  The codes leave transposed, [V, ldq] with the block elements
+// contiguous, which is the K-major operand the rollout pass wants; the scales leave block-major [d / B, lds] as always.
+// A CTA stages a tile of 128 rows x 128 columns in shared memory (16-byte loads along the rows), then thread
+// (v, h) walks rows 64 h .. 64 h + 63 of column v: maximum, scale, exact division, sixteen codes per 16-byte store.
+// ------------------------------------------------------------------------------------------------
+constexpr int kQcTile = 128;
+constexpr int kQcPitch = kQcTile + 8;          // uint16 elements per shared-memory row: 272 bytes, 16-byte aligned rows
+
+template <int BLOCK>
+__global__ void __launch_bounds__(256) quantize_cols_kernel(const __nv_bfloat16* __restrict__ x, int64_t K, int64_t N, int64_t ld,
+                                                            uint8_t* __restrict__ codes, int64_t ldq,
+                                                            float* __restrict__ scales, int64_t lds) {
+    __shared__ __align__(16) uint16_t tile[kQcTile][kQcPitch];
+    __shared__ uint32_t half_max[2][kQcTile];
+    const int tid = threadIdx.x;
+    const int64_t k0 = static_cast<int64_t>(blockIdx.y) * kQcTile, v0 = static_cast<int64_t>(blockIdx.x) * kQcTile;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int c = tid + 256 * i, r = c >> 4, c8 = (c & 15) * 8;
+        uint4 raw = make_uint4(0, 0, 0, 0);
+        if (k0 + r < K && v0 + c8 < N) raw = __ldg(reinterpret_cast<const uint4*>(x + (k0 + r) * ld + v0 + c8));
+        *reinterpret_cast<uint4*>(&tile[r][c8]) = raw;
+    }
+    __syncthreads();
+    const int v = tid & (kQcTile - 1), h = tid >> 7;
+    constexpr int kRun = BLOCK < 64 ? BLOCK : 64;          // rows of one block inside this thread's 64
+    constexpr int kRuns = 64 / kRun;
+    uint32_t amax[kRuns];
+#pragma unroll
+    for (int b = 0; b < kRuns; ++b) {
+        uint32_t m = 0;
+#pragma unroll 8
+        for (int j = 0; j < kRun; ++j) m = max(m, static_cast<uint32_t>(tile[64 * h + b * kRun + j][v]) & 0x7FFFu);
+        amax[b] = m;
+    }
+    if (BLOCK == 128) {                                      // the block spans both halves of the column
+        half_max[h][v] = amax[0];
+        __syncthreads();
+        amax[0] = max(half_max[0][v], half_max[1][v]);
+    }
+    const bool in = v0 + v < N;
+#pragma unroll
+    for (int b = 0; b < kRuns; ++b) {
+        float s = 1.0f, y = 1.0f;
+        if (amax[b] != 0u) {
+            s = __fdiv_rn(__uint_as_float(amax[b] << 16), 448.0f);
+            y = __frcp_rn(s);
+        }
+        const bool fast = s > 0x1p-100f && s < 0x1p100f;
+#pragma unroll
+        for (int g = 0; g < kRun / 16; ++g) {
+            float q[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float xv = __uint_as_float(static_cast<uint32_t>(tile[64 * h + b * kRun + g * 16 + j][v]) << 16);
+                q[j] = fast ? exact_div(xv, s, y) : slow_div(xv, s);
+            }
+            uint4 out;
+            out.x = static_cast<uint32_t>(cvt_e4m3x2(q[1], q[0])) | (static_cast<uint32_t>(cvt_e4m3x2(q[3], q[2])) << 16);
+            out.y = static_cast<uint32_t>(cvt_e4m3x2(q[5], q[4])) | (static_cast<uint32_t>(cvt_e4m3x2(q[7], q[6])) << 16);
+            out.z = static_cast<uint32_t>(cvt_e4m3x2(q[9], q[8])) | (static_cast<uint32_t>(cvt_e4m3x2(q[11], q[10])) << 16);
+            out.w = static_cast<uint32_t>(cvt_e4m3x2(q[13], q[12])) | (static_cast<uint32_t>(cvt_e4m3x2(q[15], q[14])) << 16);
+            if (in && k0 + 64 * h + b * kRun + g * 16 < K)
+                *reinterpret_cast<uint4*>(codes + (v0 + v) * ldq + k0 + 64 * h + b * kRun + g * 16) = out;
+        }
+        const int64_t kb = (k0 + 64 * h + b * kRun) / BLOCK;
+        if (in && kb * BLOCK < K && (BLOCK < 128 || h == 0)) scales[kb * lds + v0 + v] = s;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Microscaling FP8: 32 consecutive elements share a power-of-two scale 2^X, X = floor(log2 amax) - 8, stored as the
 // biased exponent X + 127 (clamped to 0..254; 127 for an all-zero block); the elements are x / 2^X on the E4M3 grid
 // (round to nearest even, saturating).  With bf16 inputs everything is exact integer work on exponent fields: the
@@ -1257,6 +1329,20 @@ cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t l
         case 32:  quantize_kernel<32><<<grid, kQThreads, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scales, lds); break;
         case 64:  quantize_kernel<64><<<grid, kQThreads, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scales, lds); break;
         case 128: quantize_kernel<128><<<grid, kQThreads, 0, stream>>>(xp, rows, cols, ld, codes, ldq, scales, lds); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_cols(const void* x, int64_t K, int64_t N, int64_t ld, int block, uint8_t* codes, int64_t ldq,
+                                 float* scales, int64_t lds, cudaStream_t stream) {
+    if (K == 0 || N == 0) return cudaSuccess;
+    dim3 grid(static_cast<unsigned>((N + kQcTile - 1) / kQcTile), static_cast<unsigned>((K + kQcTile - 1) / kQcTile));
+    const __nv_bfloat16* xp = static_cast<const __nv_bfloat16*>(x);
+    switch (block) {
+        case 32:  quantize_cols_kernel<32><<<grid, 256, 0, stream>>>(xp, K, N, ld, codes, ldq, scales, lds); break;
+        case 64:  quantize_cols_kernel<64><<<grid, 256, 0, stream>>>(xp, K, N, ld, codes, ldq, scales, lds); break;
+        case 128: quantize_cols_kernel<128><<<grid, 256, 0, stream>>>(xp, K, N, ld, codes, ldq, scales, lds); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();

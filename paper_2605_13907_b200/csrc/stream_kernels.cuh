@@ -19,6 +19,10 @@ cudaError_t stream_prepare();
 cudaError_t launch_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int block, uint8_t* codes,
                             int64_t ldq, float* scales, int64_t lds, cudaStream_t stream);
 
+// Blocks running down the columns of x [K, ld] (K a multiple of 128): codes transposed [N, ldq], scales [K / block, lds].
+cudaError_t launch_quantize_cols(const void* x, int64_t K, int64_t N, int64_t ld, int block, uint8_t* codes, int64_t ldq,
+                                 float* scales, int64_t lds, cudaStream_t stream);
+
 // Microscaling: E8M0 scale per 32 elements, packed in 512-byte chunks of 128 rows x 4 blocks; `scale_bytes` is the
 // size of the whole packed array (rows padded to a multiple of 256), filled with the neutral code first.
 cudaError_t launch_quantize_mx(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, int64_t ldq,

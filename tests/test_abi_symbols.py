@@ -69,3 +69,26 @@ def test_microscaling_entry_points_validate_on_the_host():
         assert fn(null, 4, 128, 128, one, 128, one, null) == -1       # AIS_ERR_NULL
         assert fn(one, 4, 100, 128, one, 128, one, null) == -2        # AIS_ERR_SHAPE: columns not a multiple of 128
         assert fn(one, 4, 256, 128, one, 256, one, null) == -2        # row stride shorter than the row
+
+
+def test_head_layout_rules_are_checked_on_the_host():
+    """ais_shape.w_layout: [d, V] heads need ldw >= V (a multiple of 8), take fp32 block scales only, and the column
+    quantiser refuses shapes it cannot tile; an unknown layout value is an invalid shape."""
+    import paper_2605_13907_b200 as ais
+    p = ais.default_params()
+    ok = ais.make_shape(1000, 4096, 151936, 8, 8, 128, w_layout=ais.W_DV)
+    assert ok.ldw == 151936 and ais.workspace_bytes(ok, p) > 0
+    assert ais.workspace_bytes(ais.make_shape(1000, 4096, 151936, 8, 8, 128, ldw=4096, w_layout=ais.W_DV), p) == 0    # ldw < V
+    assert ais.workspace_bytes(ais.make_shape(1000, 4096, 151936, 8, 8, 128, ldw=151940, w_layout=ais.W_DV), p) == 0  # not a multiple of 8
+    assert ais.workspace_bytes(ais.make_shape(1000, 4096, 151936, 8, 8, 0, w_layout=ais.W_DV), p) == 0                # per-tensor: [V, d] only
+    assert ais.workspace_bytes(ais.make_shape(1000, 4096, 151936, 8, 8, ais.FP8_MX32, w_layout=ais.W_DV), p) == 0
+    assert ais.workspace_bytes(ais.make_shape(1000, 4096, 151936, 8, 8, 128, w_layout=7), p) == 0
+    lib = ais.lib()
+    null = ctypes.c_void_p(None)
+    one = ctypes.c_void_p(256)                                         # never dereferenced: the checks below fail first
+    fn = lib.ais_quantize_fp8_cols
+    assert fn(null, 128, 64, 64, 128, one, 128, one, 64, null) == -1  # AIS_ERR_NULL
+    assert fn(one, 100, 64, 64, 128, one, 128, one, 64, null) == -2   # rows not a multiple of 128
+    assert fn(one, 128, 64, 64, 48, one, 128, one, 64, null) == -2    # block size
+    assert fn(one, 128, 64, 64, 128, one, 64, one, 64, null) == -2    # codes' row stride shorter than a column
+    assert fn(one, 128, 64, 64, 128, one, 136, one, 64, null) == -3   # codes' row stride not a multiple of 16

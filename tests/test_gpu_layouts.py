@@ -258,3 +258,54 @@ def test_sequence_level_reductions_over_several_tiles():
         assert abs(d[k] - ref[k]) <= 1e-4 * max(1.0, abs(ref[k])), (k, d[k], ref[k])
     got_wt = wt.cpu().numpy()
     assert np.allclose(got_wt[valid], ref_wt[valid], rtol=1e-4, atol=1e-5) and np.all(got_wt[~valid] == 1)
+
+
+@pytest.mark.parametrize("case", ["ragged", "block32"])
+def test_head_stored_d_by_v_gives_the_same_results(case):
+    """ais_shape.w_layout = AIS_W_DV: the LM head as [d, V] (the form in which the paper writes it) with a padded row
+    stride.  Codes and scales of the column-block quantiser equal the row quantiser's on the transposed matrix, the
+    log-probs of both passes are the same bits as with the [V, d] head, dH and dW (which comes out [d, V]) agree with
+    the oracle."""
+    import paper_2605_13907_b200 as ais
+    base = workloads.WORKLOADS["tiny"]
+    w = workloads.scaled(base, d=384, V=1336, P=3, G=4, lengths="uniform:5:90", seed=21) if case == "ragged" else \
+        workloads.scaled(base, d=256, V=2048, P=2, G=4, block=32, lengths="uniform:40:120", seed=22)
+    b = workloads.make_batch(w, device="cpu")
+    a = workloads.to_numpy(b)
+    ref = oais.full_path(a["H"], a["W"], a["tokens"], a["mask"], a["seq_offsets"], a["rewards"], w.P, w.G, w.block)
+    H, W, tok, msk = b.H.cuda(), b.W.cuda(), b.tokens.cuda(), b.mask.cuda()
+    offs, rew = b.seq_offsets.cuda(), b.rewards.cuda()
+    T = b.T
+    ldw = w.V + 24                                            # padded row stride of the [d, V] head
+    Wbig = torch.randn(w.d, ldw).to(torch.bfloat16).cuda()
+    Wbig[:, :w.V] = W.t()
+    Wdv = Wbig[:, :w.V]
+
+    vd = ais.AisStep(T, w.d, w.V, w.P, w.G, w.block)
+    dW_vd = torch.zeros(w.V, w.d, dtype=torch.float32, device="cuda")
+    vd.forward(H, W, tok, msk)
+    vd.diagnose(msk, offs, rew)
+    vd.backward(H, W, tok, msk, offs, dW=dW_vd)
+    dv = ais.AisStep(T, w.d, w.V, w.P, w.G, w.block, ldw=ldw, w_layout=ais.W_DV)
+    dW_dv = torch.full((w.d, w.V), 3.0, dtype=torch.float32, device="cuda")
+    dv.forward(H, Wdv, tok, msk)
+    dv.diagnose(msk, offs, rew)
+    dv.backward(H, Wdv, tok, msk, offs, dW=dW_dv)
+    torch.cuda.synchronize()
+    assert int(vd.status.item()) == 0 and int(dv.status.item()) == 0
+    # quantiser: bit-exact against the oracle (and therefore against the row quantiser)
+    assert np.array_equal(dv.qW.cpu().numpy(), ref["qW"])
+    assert np.array_equal(dv.sW.cpu().numpy()[:, :w.V].T.view(np.uint32), ref["sW"].view(np.uint32))
+    assert torch.equal(dv.qW, vd.qW) and torch.equal(dv.sW[:, :w.V], vd.sW[:, :w.V])
+    # log-probs: the same bits whichever way W is stored
+    for name in ("lp_train", "lse_train", "lp_roll"):
+        assert torch.equal(getattr(dv, name)[:T], getattr(vd, name)[:T]), name
+    assert np.max(np.abs(dv.lp_train[:T].cpu().numpy() - ref["lp_train"])) <= 1e-2
+    assert np.max(np.abs(dv.lp_roll[:T].cpu().numpy() - ref["lp_roll"])) <= 1e-2
+    assert dv.read_diag()["alpha"] == vd.read_diag()["alpha"]
+    dH = dv.dH[:T].float().cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(dH - ref["dH"]) <= 1e-2 * np.linalg.norm(ref["dH"])
+    assert float((dv.dH[:T].float() - vd.dH[:T].float()).norm()) <= 2e-3 * float(vd.dH[:T].float().norm())
+    got = dW_dv.cpu().numpy().astype(np.float64)
+    assert np.linalg.norm(got - ref["dW"].T) <= 1e-2 * np.linalg.norm(ref["dW"])
+    assert float((dW_dv - dW_vd.t()).norm()) <= 2e-3 * float(dW_vd.norm())
