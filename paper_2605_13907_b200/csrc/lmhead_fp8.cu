@@ -2,19 +2,23 @@
 //
 // The scales are arbitrary fp32 numbers, so the hardware's block-scaled MMA kinds (power-of-two scales) do not
 // apply: every scale block's partial sum is accumulated alone in tensor memory, read back and promoted on the
-// CUDA cores as acc += (sH[row] sW[col]) * partial.  One persistent CTA per SM:
+// CUDA cores as acc += (partial * sH[row]) * sW[col], two columns per instruction (packed fp32).  One persistent CTA per SM:
 //   warp 0      TMA producer: one stage = 128 K-bytes of A (128 rows) and B (256 rows) plus the stage's scale
 //               vectors, all completing on the stage's barrier
-//   warp 1      MMA issuer: SG blocks per stage, PER = 4 / SG instructions per block, one commit per block;
-//               two 256-column tensor-memory buffers alternate between blocks
+//   warps 1, 2  MMA issuers: SG blocks per stage, PER = 4 / SG instructions per block, one commit per block; two
+//               256-column tensor-memory buffers alternate between blocks, issuer i owning buffer i
 //   warps 4-11  promotion + streaming log-sum-exp: warp w reads lane quarter w % 4, column half (w - 4) / 4 in the
 //               16x256b fragment shape (a thread owns 4 rows x 32 columns, so it needs 4 + 32 scale values per
 //               block).  The four 32-register pieces of a partial tile are software-pipelined: the load of piece
-//               p + 1 is in flight during the arithmetic of piece p, and the buffer goes back to the MMA issuer as
+//               p + 1 is in flight during the arithmetic of piece p, and the buffer goes back to its MMA issuer as
 //               soon as the last piece has landed.
-// The epilogue never waits for the scales separately: the MMA issuer saw the stage barrier complete before it
+// The epilogue never waits for the scales separately: an MMA issuer saw the stage barrier complete before it
 // issued the block whose completion the epilogue waits for.  The first warpgroup hands registers to the other
 // two (384 threads x 168 registers at launch = 128 x 40 + 256 x 232).
+// What sets the pace is the chain of one promotion warp per block -- wait for the block, four tensor-memory loads of
+// about 190 clocks each with the arithmetic of the piece before in their shadow, hand-over -- which is why the
+// arithmetic is packed (it then fits the shadow) and why the MMA side is spread over two threads (one thread, sharing
+// its scheduler with two promotion warps, needed about 1,300 clocks per block for wait, four MMAs and two commits).
 #include <type_traits>
 
 #include "lmhead_common.cuh"
@@ -63,10 +67,10 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const int num_units = a.n_row_tiles * a.nsplit;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], SG > 1 ? 2 : 1); }   // both issuers use a stage when it holds several blocks
         for (int i = 0; i < 2; ++i) { mbar_init(&tfull[i], 1); mbar_init(&tempty[i], kEpiWarps); }
         for (int i = 0; i < C::kSlots; ++i) mbar_init(&sempty[i], kEpiWarps);
-        mbar_init(done, 1);
+        mbar_init(done, 2);
         *abort_flag = 0;
         *issued_slot = 0;
         fence_barrier_init();
@@ -114,36 +118,45 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 }
                 *issued_slot = issued;
             }
-        } else if (warp == 1) {
-            // ------------------------------------------------------------------ MMA issuer
+        } else if (warp == 1 || warp == 2) {
+            // ------------------------------------------------------------------ MMA issuers
+            // Two of them, on two schedulers: issuer `me` owns tensor-memory buffer `me` and takes every other scale
+            // block (block n of the CTA goes to buffer n % 2).  One thread cannot keep up: it shares its scheduler with
+            // two promotion warps, and wait + four MMAs + two commits took it about 1,300 clocks per block against the
+            // 542 the tensor core needs.  The two threads are independent: different buffers, different barriers.
             if (lane == 0) {
+                const uint32_t me = warp - 1;
                 constexpr uint32_t idesc = make_idesc(kFmtE4M3, kFmtE4M3, kBM, kBN, 0, 0);
-                Pipe st(kStages), tb(2);
+                const uint64_t desc0 = smem_desc_sw128(0, 16, 1024);           // descriptor of address 0: add (address >> 4)
+                const uint32_t dcol = tmem_base + me * kBN;
+                Pipe st(kStages);
+                uint32_t tphase = 0;                                            // phase of this issuer's buffer barriers
+                uint32_t nstage = 0;                                            // stages seen so far (SG == 1: parity picks the owner)
                 bool ok = true;
                 for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
                     const Unit w = decode_unit<MODE>(a, u);
                     if (!unit_active<MODE>(a, w)) continue;
                     const int nst = (w.t1 - w.t0) * a.ksteps;
-                    for (int i = 0; i < nst && ok; ++i) {
-                        if (!mbar_wait(&full[st.idx], st.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
-                        const uint32_t sA = smem_u32(stage_base + st.idx * kStageBytes);
-                        const uint32_t sB = sA + kAStageBytes;
+                    for (int i = 0; i < nst && ok; ++i, ++nstage) {
+                        if (SG > 1 || (nstage & 1u) == me) {
+                            if (!mbar_wait(&full[st.idx], st.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
+                            const uint64_t adesc = desc0 + (smem_u32(stage_base + st.idx * kStageBytes) >> 4);
 #pragma unroll
-                        for (int g = 0; g < SG; ++g) {
-                            if (!mbar_wait(&tempty[tb.idx], tb.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
-                            tc_fence_after();
-                            const uint32_t dcol = tmem_base + tb.idx * kBN;
+                            for (int g = 0; g < SG; ++g) {
+                                if (SG > 1 && (g & 1) != static_cast<int>(me)) continue;
+                                if (!mbar_wait(&tempty[me], tphase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
+                                tc_fence_after();
 #pragma unroll
-                            for (int j = 0; j < PER; ++j) {
-                                const uint32_t off = (g * PER + j) * 32;
-                                mma_f8(dcol, smem_desc_sw128(sA + off, 16, 1024), smem_desc_sw128(sB + off, 16, 1024), idesc,
-                                       j > 0 ? 1u : 0u);
+                                for (int j = 0; j < PER; ++j) {
+                                    const uint64_t ad = adesc + 2 * (g * PER + j);       // 32 bytes of K further on
+                                    mma_f8(dcol, ad, ad + (kAStageBytes >> 4), idesc, j > 0 ? 1u : 0u);
+                                }
+                                tc_commit(&tfull[me]);
+                                tphase ^= 1u;
                             }
-                            tc_commit(&tfull[tb.idx]);
-                            tb.advance();
+                            if (!ok) break;
+                            tc_commit(&empty[st.idx]);
                         }
-                        if (!ok) break;
-                        tc_commit(&empty[st.idx]);
                         st.advance();
                     }
                 }
@@ -185,11 +198,11 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 m4[r] = kNegBig; s4[r] = 0.f; zy4[r] = -INFINITY;
             }
             for (int t = w.t0; t < w.t1 && ok; ++t) {
-                float acc[4][16][2];                       // [row][8-column group][column of the pair]
+                F2 acc[4][16];                             // [row][8-column group]: the pair of columns 8 n + 2 cp, + 1
 #pragma unroll
                 for (int r = 0; r < 4; ++r)
 #pragma unroll
-                    for (int n = 0; n < 16; ++n) { acc[r][n][0] = 0.f; acc[r][n][1] = 0.f; }
+                    for (int n = 0; n < 16; ++n) acc[r][n] = F2{0.f, 0.f};
                 for (int ks = 0; ks < a.ksteps && ok; ++ks) {
                     const float* sS = reinterpret_cast<const float*>(scale_base + sc.idx * C::kSlotBytes);
 #pragma unroll 1
@@ -198,9 +211,12 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         tc_fence_after();
                         const uint32_t buf = tb.idx;
                         ld_piece(buf, 0, 0, va);
-                        float sh[4];
+                        F2 sh[4];
 #pragma unroll
-                        for (int r = 0; r < 4; ++r) sh[r] = sS[g * kBM + q * 32 + (r >> 1) * 16 + (r & 1) * 8 + rg];
+                        for (int r = 0; r < 4; ++r) {
+                            const float x = sS[g * kBM + q * 32 + (r >> 1) * 16 + (r & 1) * 8 + rg];
+                            sh[r] = F2{x, x};
+                        }
                         const float2* sw2 = reinterpret_cast<const float2*>(sS + (C::kSlotBOffset / 4) + g * kBN + half * 128) + cp;
                         // (lane half of the quarter) x (column half of the piece); the indices are compile-time constants so
                         // that the accumulators stay in registers
@@ -208,13 +224,12 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                             constexpr int hh = decltype(HH)::value, nb = decltype(NB)::value;
 #pragma unroll
                             for (int mq = 0; mq < 8; ++mq) {
-                                const float2 sw = sw2[(nb * 8 + mq) * 4];          // columns 8n + 2cp, +1 of this thread
+                                const float2 swf = sw2[(nb * 8 + mq) * 4];         // columns 8n + 2cp, +1 of this thread
+                                const F2 sw = {swf.x, swf.y};
 #pragma unroll
                                 for (int e = 0; e < 2; ++e) {
-                                    acc[hh * 2 + e][nb * 8 + mq][0] =
-                                        fmaf(sh[hh * 2 + e] * sw.x, __uint_as_float(v[4 * mq + 2 * e]), acc[hh * 2 + e][nb * 8 + mq][0]);
-                                    acc[hh * 2 + e][nb * 8 + mq][1] =
-                                        fmaf(sh[hh * 2 + e] * sw.y, __uint_as_float(v[4 * mq + 2 * e + 1]), acc[hh * 2 + e][nb * 8 + mq][1]);
+                                    const F2 x = {__uint_as_float(v[4 * mq + 2 * e]), __uint_as_float(v[4 * mq + 2 * e + 1])};
+                                    acc[hh * 2 + e][nb * 8 + mq] = fma2(mul2(x, sh[hh * 2 + e]), sw, acc[hh * 2 + e][nb * 8 + mq]);
                                 }
                             }
                         };
@@ -253,25 +268,25 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         // the compiler into acc[k], and a dynamically indexed array leaves the register file
 #pragma unroll
                         for (int n = 0; n < 16; ++n) {
-                            zy4[r] = fmaxf(zy4[r], (yy == 8 * n) ? acc[r][n][0] : -INFINITY);
-                            zy4[r] = fmaxf(zy4[r], (yy == 8 * n + 1) ? acc[r][n][1] : -INFINITY);
+                            zy4[r] = fmaxf(zy4[r], (yy == 8 * n) ? acc[r][n].x : -INFINITY);
+                            zy4[r] = fmaxf(zy4[r], (yy == 8 * n + 1) ? acc[r][n].y : -INFINITY);
                         }
                     }
                     if (t * kBN + kBN > a.ncols) {
 #pragma unroll
                         for (int n = 0; n < 16; ++n) {
-                            if (cbase + 8 * n >= a.ncols) acc[r][n][0] = -INFINITY;
-                            if (cbase + 8 * n + 1 >= a.ncols) acc[r][n][1] = -INFINITY;
+                            if (cbase + 8 * n >= a.ncols) acc[r][n].x = -INFINITY;
+                            if (cbase + 8 * n + 1 >= a.ncols) acc[r][n].y = -INFINITY;
                         }
                     }
-                    float cm = acc[r][0][0];
+                    float cm = acc[r][0].x;
 #pragma unroll
-                    for (int n = 0; n < 16; ++n) cm = fmaxf(cm, fmaxf(acc[r][n][0], acc[r][n][1]));
+                    for (int n = 0; n < 16; ++n) cm = fmaxf(cm, fmaxf(acc[r][n].x, acc[r][n].y));
                     const float m_new = fmaxf(m4[r], cm * kLog2e);
                     float add = 0.f;
 #pragma unroll
                     for (int n = 0; n < 16; ++n)
-                        add += ex2(fmaf(acc[r][n][0], kLog2e, -m_new)) + ex2(fmaf(acc[r][n][1], kLog2e, -m_new));
+                        add += ex2(fmaf(acc[r][n].x, kLog2e, -m_new)) + ex2(fmaf(acc[r][n].y, kLog2e, -m_new));
                     s4[r] = fmaf(s4[r], ex2(m4[r] - m_new), add);
                     m4[r] = m_new;
                 }
