@@ -76,4 +76,4 @@ def test_backward_fraction_counts_only_rows_in_live_tiles():
     w = local["workload"]
     want = 2.0 * w.d * w.V * (600 + 512) / 0.120 / 1e12
     assert abs(line["roofline"]["passes"]["bwd"]["tflops"] - want) < 1e-9 * want
-    assert line["roofline"]["passes"]["fwd_roll_fp8"]["ceiling"]["frac_of_fp8_tensor_rate"] < 0.7
+    assert 0.5 < line["roofline"]["passes"]["fwd_roll_fp8"]["ceiling"]["frac_of_fp8_tensor_rate"] < 0.7
