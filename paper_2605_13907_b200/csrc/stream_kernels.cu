@@ -65,8 +65,17 @@ __device__ __forceinline__ uint2 quantize_values(const uint4 raw, float s, float
         v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
     }
     if (s > 0x1p-100f && s < 0x1p100f) {
+        // exact_div on two values per instruction (the packed fp32 forms round each half like the scalar ones)
+        const F2 ys = {y, y}, ns = {-s, -s};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) qv[i] = exact_div(v[i], s, y);
+        for (int i = 0; i < 8; i += 2) {
+            const F2 x = {v[i], v[i + 1]};
+            F2 q = mul2(x, ys);
+            q = fma2(fma2(ns, q, x), ys, q);
+            q = fma2(fma2(ns, q, x), ys, q);
+            qv[i] = copysignf(q.x, x.x);
+            qv[i + 1] = copysignf(q.y, x.y);
+        }
     } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i) qv[i] = slow_div(v[i], s);      // rare: scale outside the safe exponent range
@@ -757,11 +766,6 @@ constexpr int kMomStages = 3;
 constexpr int kMomStageBytes = kMomRows * 9;
 constexpr int kMomSmemBytes = kMomStages * kMomStageBytes + 128;
 
-__device__ __forceinline__ float exp_ftz(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x * 1.4426950408889634f));
-    return y;
-}
 
 // (add2 / sub2 / mul2 / fma2: the packed two-element fp32 instructions, ptx.cuh.)  The staged kernel is bound by
 // instruction issue right after HBM, and half of its per-row work is additions, multiplications and multiply-adds.

@@ -206,6 +206,21 @@ def test_fullsize_sampled_parity(name):
             assert bool((pstep.lp_train[:pb.T][pad] == 0).all()) and bool((pstep.rho[:pb.T][pad] == 1).all())
             assert bool((pstep.w_tilde[:pb.T][pad] == 1).all()) and bool((pstep.dH[:pb.T][pad] == 0).all())
             assert abs(float(pstep.loss.item()) - loss) <= 1e-4 * max(1.0, abs(loss))
+            del pstep, pb
+
+        # ---- the same head stored [d, V] (ais_shape.w_layout = AIS_W_DV) at full size: both log-prob vectors must be the
+        # same bits as with the [V, d] head that was checked against the oracle above, codes and scales too
+        if name == "qwen3_8b":
+            Wdv = batch.W.t().contiguous()
+            dstep = ais.AisStep(T, w.d, w.V, w.P, w.G, w.block, params=params, workspace_bytes_cap=48 << 30, w_layout=ais.W_DV)
+            dstep.step(batch.H, Wdv, batch.tokens, batch.mask, offs_d, rew_d)
+            torch.cuda.synchronize()
+            assert int(dstep.status.item()) == 0
+            assert torch.equal(dstep.qW, step.qW) and torch.equal(dstep.sW[:, :w.V], step.sW[:, :w.V])
+            assert torch.equal(dstep.lp_train[:T], step.lp_train[:T]) and torch.equal(dstep.lp_roll[:T], step.lp_roll[:T])
+            assert dstep.read_diag()["alpha"] == d["alpha"]
+            ddH = dstep.dH[idx].float().cpu().numpy().astype(np.float64)
+            assert np.linalg.norm(ddH - dH_all) <= DH_REL * np.linalg.norm(dH_all)
     finally:
         pool.terminate()
         pool.join()
