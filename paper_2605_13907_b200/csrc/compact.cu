@@ -167,7 +167,10 @@ int ais_scatter_rows(const void* src, int64_t src_stride_bytes, const int32_t* r
     if (row_bytes % 16 != 0 || src_stride_bytes % 16 != 0 || dst_stride_bytes % 16 != 0 || !aligned(src, 16) || !aligned(dst, 16))
         return AIS_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (dst_rows > 0 && cudaMemsetAsync(dst, 0, static_cast<size_t>(dst_rows) * dst_stride_bytes, s) != cudaSuccess) return AIS_ERR_DEVICE;
+    // only the row_bytes of every row: the padding between rows (and whatever follows the last row) is the caller's
+    if (dst_rows > 0 && cudaMemset2DAsync(dst, static_cast<size_t>(dst_stride_bytes), 0, static_cast<size_t>(row_bytes),
+                                          static_cast<size_t>(dst_rows), s) != cudaSuccess)
+        return AIS_ERR_DEVICE;
     if (n == 0) return AIS_OK;
     scatter_rows_kernel<<<grid_for(n * (row_bytes / 16)), kThreads, 0, s>>>(static_cast<const uint8_t*>(src), src_stride_bytes, row_index,
                                                                              n, row_bytes / 16, static_cast<uint8_t*>(dst),
