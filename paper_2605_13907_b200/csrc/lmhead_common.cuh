@@ -30,6 +30,12 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, v
     return __all_sync(0xffffffffu, r);
 }
 
+__device__ __forceinline__ bool mbar_wait_warp_spin(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                    long long limit = 0) {
+    const bool r = mbar_wait_spin(bar, parity, abort_flag, limit);
+    return __all_sync(0xffffffffu, r);
+}
+
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

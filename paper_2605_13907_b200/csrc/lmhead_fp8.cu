@@ -7,18 +7,21 @@
 //               vectors, all completing on the stage's barrier
 //   warps 1, 2  MMA issuers: SG blocks per stage, PER = 4 / SG instructions per block, one commit per block; two
 //               256-column tensor-memory buffers alternate between blocks, issuer i owning buffer i
-//   warps 4-11  promotion + streaming log-sum-exp: warp w reads lane quarter w % 4, column half (w - 4) / 4 in the
-//               16x256b fragment shape (a thread owns 4 rows x 32 columns, so it needs 4 + 32 scale values per
-//               block).  The four 32-register pieces of a partial tile are software-pipelined: the load of piece
-//               p + 1 is in flight during the arithmetic of piece p, and the buffer goes back to its MMA issuer as
-//               soon as the last piece has landed.
+//   warps 4-11  promotion + streaming log-sum-exp: warp w reads lane quarter w % 4, column half (w - 4) / 4 with
+//               32x32b loads (a thread owns one row x 128 columns: its row scale is one register, the column
+//               scales come as broadcast 16-byte shared-memory loads).  The four 32-register pieces of a partial
+//               tile are software-pipelined: the load of piece p + 1 is in flight during the arithmetic of piece
+//               p, and the buffer goes back to its MMA issuer as soon as the last piece has landed.
 // The epilogue never waits for the scales separately: an MMA issuer saw the stage barrier complete before it
 // issued the block whose completion the epilogue waits for.  The first warpgroup hands registers to the other
 // two (384 threads x 168 registers at launch = 128 x 40 + 256 x 232).
-// What sets the pace is the chain of one promotion warp per block -- wait for the block, four tensor-memory loads of
-// about 190 clocks each with the arithmetic of the piece before in their shadow, hand-over -- which is why the
-// arithmetic is packed (it then fits the shadow) and why the MMA side is spread over two threads (one thread, sharing
-// its scheduler with two promotion warps, needed about 1,300 clocks per block for wait, four MMAs and two commits).
+// Measured per 128 x 256 x 128 block on the busiest SM: about 1,280 clocks against 542 of tensor-core time.  No single
+// unit is the bound (timing-only variants: 790 clocks with an epilogue that only hands the buffers back, 660 without
+// the operand copies as well; the tensor-memory loads need about 280 clocks at the 32x32b shape and twice that at
+// the 16x256b fragment shape, the packed arithmetic about 350, the column-scale loads about 225): the block goes
+// round MMA -> commit -> wait -> load -> release -> wait -> MMA through two buffers, every hand-over costing
+// 200-300 clocks, which is why the MMA side is spread over two threads, the arithmetic is packed, and the promotion
+// warps poll their barrier without blocking (the blocking form cost 70 clocks per block).
 #include <type_traits>
 
 #include "lmhead_common.cuh"
@@ -169,88 +172,73 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         reg_alloc<232>();
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int half = (warp - 4) >> 2;             // column half of the partial tile
-        const int rg = lane >> 2, cp = lane & 3;      // fragment coordinates of this thread
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         Pipe tb(2), sc(C::kSlots);
         bool ok = true;
         uint32_t flags = 0;
         uint32_t va[32], vb[32];
-        auto ld_piece = [&](uint32_t buf, int hh, int nb, uint32_t (&v)[32]) {
-            tmem_ld_16x256b_x8(tmem_base + lane_base + (static_cast<uint32_t>(hh * 16) << 16) + buf * kBN + half * 128 + nb * 64, v);
+        auto ld_piece = [&](uint32_t buf, int p, uint32_t (&v)[32]) {
+            tmem_ld32(tmem_base + lane_base + buf * kBN + half * 128 + p * 32, v);
         };
         for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
             const Unit w = decode_unit<MODE>(a, u);
             if (!unit_active<MODE>(a, w)) continue;     // every row masked: the merge kernel never reads these partials
-            int64_t grow4[4];
-            bool rok4[4];
-            int y4[4];
-            float m4[4], s4[4], zy4[4];
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const int64_t lr = static_cast<int64_t>(w.rt) * kBM + q * 32 + (r >> 1) * 16 + (r & 1) * 8 + rg;
-                rok4[r] = lr < a.rows;
-                grow4[r] = a.row0 + lr;
-                y4[r] = -1;
-                if (rok4[r]) {
-                    y4[r] = a.tokens[grow4[r]];
-                    if (a.mask[grow4[r]] != 0 && (y4[r] < 0 || y4[r] >= a.ncols)) { flags |= AIS_FLAG_TOKEN_RANGE; y4[r] = -1; }
-                }
-                m4[r] = kNegBig; s4[r] = 0.f; zy4[r] = -INFINITY;
+            const int64_t lr = static_cast<int64_t>(w.rt) * kBM + q * 32 + lane;
+            const bool rok = lr < a.rows;
+            const int64_t grow = a.row0 + lr;
+            int y = -1;
+            if (rok) {
+                y = a.tokens[grow];
+                if (a.mask[grow] != 0 && (y < 0 || y >= a.ncols)) { flags |= AIS_FLAG_TOKEN_RANGE; y = -1; }
             }
+            float m_run = kNegBig, s_run = 0.f, zy = -INFINITY;
             for (int t = w.t0; t < w.t1 && ok; ++t) {
-                F2 acc[4][16];                             // [row][8-column group]: the pair of columns 8 n + 2 cp, + 1
+                F2 acc[64];                                // columns 2 n, 2 n + 1 of this thread's 128
 #pragma unroll
-                for (int r = 0; r < 4; ++r)
-#pragma unroll
-                    for (int n = 0; n < 16; ++n) acc[r][n] = F2{0.f, 0.f};
+                for (int n = 0; n < 64; ++n) acc[n] = F2{0.f, 0.f};
                 for (int ks = 0; ks < a.ksteps && ok; ++ks) {
                     const float* sS = reinterpret_cast<const float*>(scale_base + sc.idx * C::kSlotBytes);
 #pragma unroll 1
                     for (int g = 0; g < SG; ++g) {
-                        if (!mbar_wait_warp(&tfull[tb.idx], tb.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
+                        if (!mbar_wait_warp_spin(&tfull[tb.idx], tb.phase, abort_flag, a.wait_cycles)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t buf = tb.idx;
-                        ld_piece(buf, 0, 0, va);
-                        F2 sh[4];
+                        ld_piece(buf, 0, va);
+                        const float shx = sS[g * kBM + q * 32 + lane];
+                        const F2 sh = {shx, shx};
+                        // every lane reads the same column scales: broadcast 16-byte loads
+                        const float4* sw4 = reinterpret_cast<const float4*>(sS + (C::kSlotBOffset / 4) + g * kBN + half * 128);
+                        auto promote = [&](auto PP, uint32_t (&v)[32]) {
+                            constexpr int pp = decltype(PP)::value;
 #pragma unroll
-                        for (int r = 0; r < 4; ++r) {
-                            const float x = sS[g * kBM + q * 32 + (r >> 1) * 16 + (r & 1) * 8 + rg];
-                            sh[r] = F2{x, x};
-                        }
-                        const float2* sw2 = reinterpret_cast<const float2*>(sS + (C::kSlotBOffset / 4) + g * kBN + half * 128) + cp;
-                        // (lane half of the quarter) x (column half of the piece); the indices are compile-time constants so
-                        // that the accumulators stay in registers
-                        auto promote = [&](auto HH, auto NB, uint32_t (&v)[32]) {
-                            constexpr int hh = decltype(HH)::value, nb = decltype(NB)::value;
-#pragma unroll
-                            for (int mq = 0; mq < 8; ++mq) {
-                                const float2 swf = sw2[(nb * 8 + mq) * 4];         // columns 8n + 2cp, +1 of this thread
-                                const F2 sw = {swf.x, swf.y};
-#pragma unroll
-                                for (int e = 0; e < 2; ++e) {
-                                    const F2 x = {__uint_as_float(v[4 * mq + 2 * e]), __uint_as_float(v[4 * mq + 2 * e + 1])};
-                                    acc[hh * 2 + e][nb * 8 + mq] = fma2(mul2(x, sh[hh * 2 + e]), sw, acc[hh * 2 + e][nb * 8 + mq]);
-                                }
+                            for (int j = 0; j < 8; ++j) {
+                                const float4 swf = sw4[pp * 8 + j];
+                                const F2 x0 = {__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1])};
+                                const F2 x1 = {__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])};
+                                acc[pp * 16 + 2 * j] = fma2(mul2(x0, sh), F2{swf.x, swf.y}, acc[pp * 16 + 2 * j]);
+                                acc[pp * 16 + 2 * j + 1] = fma2(mul2(x1, sh), F2{swf.z, swf.w}, acc[pp * 16 + 2 * j + 1]);
                             }
                         };
                         using I0 = std::integral_constant<int, 0>;
                         using I1 = std::integral_constant<int, 1>;
+                        using I2 = std::integral_constant<int, 2>;
+                        using I3 = std::integral_constant<int, 3>;
                         tmem_ld_wait(va);
-                        ld_piece(buf, 0, 1, vb);
-                        promote(I0{}, I0{}, va);
+                        ld_piece(buf, 1, vb);
+                        promote(I0{}, va);
                         tmem_ld_wait(vb);
-                        ld_piece(buf, 1, 0, va);
-                        promote(I0{}, I1{}, vb);
+                        ld_piece(buf, 2, va);
+                        promote(I1{}, vb);
                         tmem_ld_wait(va);
-                        ld_piece(buf, 1, 1, vb);
-                        promote(I1{}, I0{}, va);
+                        ld_piece(buf, 3, vb);
+                        promote(I2{}, va);
                         tmem_ld_wait(vb);
                         // the whole partial tile is in registers: hand the buffer back before the last arithmetic
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&tempty[buf]);
                         tb.advance();
-                        promote(I1{}, I1{}, vb);
+                        promote(I3{}, vb);
                     }
                     if (!ok) break;
                     __syncwarp();
@@ -258,55 +246,41 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     sc.advance();
                 }
                 if (!ok) break;
-                // streaming log-sum-exp over this thread's 32 columns of each of its 4 rows
-                const int cbase = t * kBN + half * 128 + 2 * cp;           // column of acc[.][0][0]
+                // streaming log-sum-exp over this thread's 128 columns of its row
+                const int cbase = t * kBN + half * 128;                    // column of acc[0].x
+                const int yy = y - cbase;
+                if (yy >= 0 && yy < 128) {
+                    // written as a running maximum on purpose: a chain of "if (k == n) z = acc[n]" is folded by
+                    // the compiler into acc[k], and a dynamically indexed array leaves the register file
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int yy = y4[r] - cbase;                          // = 8n + e for an owned column
-                    if (yy >= 0 && yy < 128 && (yy & 6) == 0) {
-                        // written as a running maximum on purpose: a chain of "if (k == n) z = acc[n]" is folded by
-                        // the compiler into acc[k], and a dynamically indexed array leaves the register file
-#pragma unroll
-                        for (int n = 0; n < 16; ++n) {
-                            zy4[r] = fmaxf(zy4[r], (yy == 8 * n) ? acc[r][n].x : -INFINITY);
-                            zy4[r] = fmaxf(zy4[r], (yy == 8 * n + 1) ? acc[r][n].y : -INFINITY);
-                        }
+                    for (int n = 0; n < 64; ++n) {
+                        zy = fmaxf(zy, (yy == 2 * n) ? acc[n].x : -INFINITY);
+                        zy = fmaxf(zy, (yy == 2 * n + 1) ? acc[n].y : -INFINITY);
                     }
-                    if (t * kBN + kBN > a.ncols) {
-#pragma unroll
-                        for (int n = 0; n < 16; ++n) {
-                            if (cbase + 8 * n >= a.ncols) acc[r][n].x = -INFINITY;
-                            if (cbase + 8 * n + 1 >= a.ncols) acc[r][n].y = -INFINITY;
-                        }
-                    }
-                    float cm = acc[r][0].x;
-#pragma unroll
-                    for (int n = 0; n < 16; ++n) cm = fmaxf(cm, fmaxf(acc[r][n].x, acc[r][n].y));
-                    const float m_new = fmaxf(m4[r], cm * kLog2e);
-                    float add = 0.f;
-#pragma unroll
-                    for (int n = 0; n < 16; ++n)
-                        add += ex2(fmaf(acc[r][n].x, kLog2e, -m_new)) + ex2(fmaf(acc[r][n].y, kLog2e, -m_new));
-                    s4[r] = fmaf(s4[r], ex2(m4[r] - m_new), add);
-                    m4[r] = m_new;
                 }
+                if (t * kBN + kBN > a.ncols) {
+#pragma unroll
+                    for (int n = 0; n < 64; ++n) {
+                        if (cbase + 2 * n >= a.ncols) acc[n].x = -INFINITY;
+                        if (cbase + 2 * n + 1 >= a.ncols) acc[n].y = -INFINITY;
+                    }
+                }
+                float cm = acc[0].x;
+#pragma unroll
+                for (int n = 0; n < 64; ++n) cm = fmaxf(cm, fmaxf(acc[n].x, acc[n].y));
+                const float m_new = fmaxf(m_run, cm * kLog2e);
+                float add = 0.f;
+#pragma unroll
+                for (int n = 0; n < 64; ++n)
+                    add += ex2(fmaf(acc[n].x, kLog2e, -m_new)) + ex2(fmaf(acc[n].y, kLog2e, -m_new));
+                s_run = fmaf(s_run, ex2(m_run - m_new), add);
+                m_run = m_new;
             }
-            // the four threads that share a row merge their (max, sum, target) and one of them writes the partial
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                float M = fmaxf(m4[r], __shfl_xor_sync(0xffffffffu, m4[r], 1));
-                M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
-                float ssum = s4[r] * ex2(m4[r] - M);
-                ssum += __shfl_xor_sync(0xffffffffu, ssum, 1);
-                ssum += __shfl_xor_sync(0xffffffffu, ssum, 2);
-                float z = fmaxf(zy4[r], __shfl_xor_sync(0xffffffffu, zy4[r], 1));
-                z = fmaxf(z, __shfl_xor_sync(0xffffffffu, z, 2));
-                if (ok && rok4[r] && cp == 0) {
-                    const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow4[r];
-                    a.part_m[o] = M * kLn2;
-                    a.part_s[o] = ssum;
-                    a.part_z[o] = z;
-                }
+            if (ok && rok) {
+                const int64_t o = static_cast<int64_t>(w.part * 2 + half) * a.part_ld + grow;
+                a.part_m[o] = m_run * kLn2;
+                a.part_s[o] = s_run;
+                a.part_z[o] = zy;
             }
         }
         if (flags && a.status) atomicOr(a.status, flags);
