@@ -39,12 +39,12 @@ import workloads  # noqa: E402
 # DRAM bytes (read + write) of one launch of each tensor-core kernel on the bench workload, from one profiler capture of
 # the 1-prompt case (10,585 rows, all of them in live tiles) scaled to the full launch: the forward passes re-read W, or
 # its codes and scales, once per group of 37 row tiles (3 sweeps at 1 prompt, 15 at 8 prompts); the two backward kernels
-# (7.08 GB and 18.18 GB at 1 prompt, taken together here because one call enqueues both; an earlier capture of the same dH
-# kernel read 13.99 GB: its operands are shared through L2, and how well depends on how closely the CTAs stay in step) grow
-# with the rows in live tiles.
+# (7.05 GB and 15.06 GB at 1 prompt, taken together here because one call enqueues both; two other captures of the same dH
+# kernel read 13.99 and 18.18 GB: its operands are shared through L2, and how well depends on how closely the CTAs stay in
+# step) grow with the rows in live tiles.
 # None for workloads and kernels that were not captured.
 TRAFFIC = {
-    "qwen3_8b": {"fwd_train_bf16": 3.831e9 * 15 / 3, "fwd_roll_fp8": 1.987e9 * 15 / 3, "bwd": (7.084e9 + 18.18e9) * 63387 / 10585},
+    "qwen3_8b": {"fwd_train_bf16": 3.829e9 * 15 / 3, "fwd_roll_fp8": 1.978e9 * 15 / 3, "bwd": (7.046e9 + 15.06e9) * 63387 / 10585},
 }
 METRIC = "AIS-corrected fwd+bwd tokens/sec"
 UNIT = "tokens/s"
