@@ -325,7 +325,8 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params,
  *                       offsets of the packed batch) and row_index [>= N] (original row of packed row i, increasing
  *                       inside every sequence; N = packed_offsets[S]).
  *   ais_gather_rows   : dst[i,:] = src[row_index[i],:] for rows of row_bytes bytes (multiple of 16; strides in bytes).
- *   ais_scatter_rows  : dst is zero-filled (dst_rows rows), then dst[row_index[i],:] = src[i,:].
+ *   ais_scatter_rows  : the row_bytes of each of dst's dst_rows rows are zero-filled (padding between rows is left
+ *                       alone), then dst[row_index[i],:] = src[i,:].
  *   ais_gather_words / ais_scatter_words : the same for vectors of 32-bit elements (tokens, log-probs, rho, w_tilde);
  *                       the scatter first fills dst[0 .. dst_rows) with fill_bits (0 for log-probs, the bits of 1.0f
  *                       for rho and w_tilde).
