@@ -36,15 +36,11 @@ sys.path.insert(0, ROOT)
 
 import workloads  # noqa: E402
 
-# DRAM bytes (read + write) of one launch of each tensor-core kernel on the bench workload, from one profiler capture of
-# the 1-prompt case (10,585 rows, all of them in live tiles) scaled to the full launch: the forward passes re-read W, or
-# its codes and scales, once per group of 37 row tiles (3 sweeps at 1 prompt, 15 at 8 prompts); the two backward kernels
-# (7.05 GB and 15.06 GB at 1 prompt, taken together here because one call enqueues both; two other captures of the same dH
-# kernel read 13.99 and 18.18 GB: its operands are shared through L2, and how well depends on how closely the CTAs stay in
-# step) grow with the rows in live tiles.
-# None for workloads and kernels that were not captured.
+# DRAM bytes (read + write) of one launch of each tensor-core kernel on a bench workload, from a one-pass profiler capture
+# of the full-size step (the two DRAM byte counters alone need no replay): the two backward kernels are taken together
+# because one call enqueues both.  None for workloads, variants and kernels that were not captured.
 TRAFFIC = {
-    "qwen3_8b": {"fwd_train_bf16": 3.829e9 * 15 / 3, "fwd_roll_fp8": 1.978e9 * 15 / 3, "bwd": (7.046e9 + 15.06e9) * 63387 / 10585},
+    "qwen3_8b": {"fwd_train_bf16": 19.28e9, "fwd_roll_fp8": 9.95e9, "bwd": (31.03e9 + 21.50e9) + (66.69e9 + 0.57e9)},
 }
 METRIC = "AIS-corrected fwd+bwd tokens/sec"
 UNIT = "tokens/s"

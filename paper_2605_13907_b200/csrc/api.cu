@@ -138,6 +138,7 @@ struct Layout {
     size_t off_part_m, off_part_s, off_part_z;   // forward partials
     size_t off_diag;                              // reduction partials (doubles)
     size_t off_flags;                             // one byte per 128-row tile: anything to compute there?
+    size_t off_pace;                              // ring of counters that keeps the CTAs of a tensor-core launch in step
     size_t off_coef, off_nseq;                    // backward: c_t, valid rows per sequence
     size_t off_seqw;                              // sequence-level variant: log weight per sequence
     size_t off_u;                                 // backward scratch
@@ -157,6 +158,7 @@ Layout make_layout(const ais_shape* s, const ais_params* p) {
     L.off_part_s = off; off += part_bytes;
     L.off_part_z = off; off += part_bytes;
     L.off_flags = off;  off += align_up(static_cast<size_t>(L.t_ld / kBM + 2), 256);
+    L.off_pace = off;   off += align_up(static_cast<size_t>(kPaceRing) * sizeof(uint32_t), 256);
     L.off_diag = off;   off += align_up(static_cast<size_t>(kDiagBlocks) * kNumMoments * sizeof(double), 256);
     L.off_coef = off;   off += align_up(static_cast<size_t>(L.t_ld) * sizeof(float), 256);
     L.off_nseq = off;   off += align_up(static_cast<size_t>(s->P) * s->G * sizeof(int32_t), 256);
@@ -169,6 +171,19 @@ Layout make_layout(const ais_shape* s, const ais_params* p) {
 }
 
 constexpr int64_t kBwdRowsRecommended = 2 * 148 * kBM;
+
+// Zeroes the pacing ring and points the launch at it.  tiles_per_unit = the largest number of column tiles a unit of
+// the launch walks; a launch of a single wave has nobody to keep in step with over time and runs without pacing only
+// when it has a single CTA.
+cudaError_t arm_pace(LmheadArgs& a, uint8_t* ws, const Layout& L, int tiles_per_unit, int ctas, cudaStream_t s) {
+    a.pace = nullptr;
+    a.pace_per_unit = 0;
+    if (ctas < 2) return cudaSuccess;
+    const int64_t fills = static_cast<int64_t>(tiles_per_unit) * a.ksteps;
+    a.pace = reinterpret_cast<uint32_t*>(ws + L.off_pace);
+    a.pace_per_unit = static_cast<int32_t>((fills + kPaceFills - 1) / kPaceFills);
+    return cudaMemsetAsync(a.pace, 0, static_cast<size_t>(kPaceRing) * sizeof(uint32_t), s);
+}
 
 }  // namespace
 
@@ -370,6 +385,7 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
                  : make_tmap(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, W, d, V, shape->ldw * 2, 64, kBN, CU_TENSOR_MAP_SWIZZLE_128B)))
             return AIS_ERR_DEVICE;
         a.ksteps = shape->d / 64;
+        if (arm_pace(a, ws, L, (a.n_col_tiles + a.nsplit - 1) / a.nsplit, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_lmhead(dv ? kFwdBf16Dv : kFwdBf16, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_train, lse_train, dev_status, s) !=
             cudaSuccess)
@@ -388,6 +404,7 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
         a.sf_a = static_cast<const uint8_t*>(sH_);
         a.sf_b = static_cast<const uint8_t*>(sW_);
         a.nk4 = shape->d / 128;
+        if (arm_pace(a, ws, L, (a.n_col_tiles + a.nsplit - 1) / a.nsplit, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_lmhead(fp4 ? kFwdMx4 : kFwdMx, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_roll, lse_roll, dev_status, s) !=
             cudaSuccess)
@@ -400,6 +417,7 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
         a.ksteps = shape->d / 128;
         a.scale_a = sH;
         a.scale_b = sW;
+        if (arm_pace(a, ws, L, (a.n_col_tiles + a.nsplit - 1) / a.nsplit, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_lmhead(kFwdFp8T, tmA, tmB, tmA, tmB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_roll, lse_roll, dev_status, s) !=
             cudaSuccess)
@@ -412,6 +430,7 @@ int ais_logprob_fwd(const ais_shape* shape, const ais_params* params, const void
             !make_tmap(&tmSB, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, sW, V, nkb, ldsW * 4, kBN, a.sgroups, CU_TENSOR_MAP_SWIZZLE_NONE))
             return AIS_ERR_DEVICE;
         a.ksteps = shape->d / 128;
+        if (arm_pace(a, ws, L, (a.n_col_tiles + a.nsplit - 1) / a.nsplit, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_lmhead(kFwdFp8, tmA, tmB, tmSA, tmSB, a, ctas, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_combine(a.part_m, a.part_s, a.part_z, L.nparts, L.t_ld, mask, shape->T, lp_roll, lse_roll, dev_status, s) !=
             cudaSuccess)
@@ -575,6 +594,8 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
         a.nsplit = L.nsplit;
         a.ksteps = shape->d / 64;
         int units = a.n_row_tiles * a.nsplit;
+        if (arm_pace(a, ws, L, (a.n_col_tiles + a.nsplit - 1) / a.nsplit, units < num_sms ? units : num_sms, s) != cudaSuccess)
+            return AIS_ERR_DEVICE;
         if (launch_lmhead(dv ? kBwdPDv : kBwdP, tmH, tmW_k, tmH, tmW_k, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
             return AIS_ERR_DEVICE;
         // dH = c (.) (U W)
@@ -584,6 +605,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
         a.nsplit = 1;
         a.ksteps = (shape->V + 63) / 64;
         units = a.n_row_tiles * a.n_col_tiles;
+        if (arm_pace(a, ws, L, 1, units < num_sms ? units : num_sms, s) != cudaSuccess) return AIS_ERR_DEVICE;
         if (launch_lmhead(dv ? kBwdDhDv : kBwdDh, tmU, tmW_n, tmU, tmW_n, a, units < num_sms ? units : num_sms, s) != cudaSuccess)
             return AIS_ERR_DEVICE;
         if (dW) {
@@ -610,6 +632,7 @@ int ais_loss_bwd(const ais_shape* shape, const ais_params* params, const void* H
             units = w.n_row_tiles * w.n_col_tiles;
             const CUtensorMap& tmRow = dv ? tmH_t : tmU_t;
             const CUtensorMap& tmCol = dv ? tmU_t : tmH_t;
+            if (arm_pace(w, ws, L, 1, units < num_sms ? units : num_sms, s) != cudaSuccess) return AIS_ERR_DEVICE;
             if (launch_lmhead(kBwdDw, tmRow, tmCol, tmRow, tmCol, w, units < num_sms ? units : num_sms, s) != cudaSuccess)
                 return AIS_ERR_DEVICE;
         }

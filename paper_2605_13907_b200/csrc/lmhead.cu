@@ -85,11 +85,18 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             Pipe st(STG);
             uint32_t issued = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+            Pacer pacer(a.pace, a.pace_per_unit);
+            int n = 0;                                          // ordinal of this CTA's unit (its wave)
+            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x, ++n) {
                 const Unit w = decode_unit<BASE>(a, u);
-                if (!unit_active<BASE>(a, w)) continue;
+                if (!unit_active<BASE>(a, w)) {
+                    if (pacer.ring) pacer.top_up(n, 0);
+                    continue;
+                }
+                int fills = 0;                                  // stage fills of this unit so far
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
-                    for (int ks = 0; ks < a.ksteps; ++ks) {
+                    for (int ks = 0; ks < a.ksteps; ++ks, ++fills) {
+                        if (pacer.ring && fills % kPaceFills == 0) pacer.announce(n, fills / kPaceFills);
                         if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                         uint8_t* sA = stage_base + st.idx * STG_BYTES;
                         uint8_t* sB = sA + A_BYTES;
@@ -134,7 +141,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         st.advance();
                     }
                 }
+                if (pacer.ring) pacer.top_up(n, (fills + kPaceFills - 1) / kPaceFills);
             }
+            if (pacer.ring)                                     // units of the last wave that this CTA does not have
+                for (const int waves = (num_units + gridDim.x - 1) / gridDim.x; n < waves; ++n) pacer.top_up(n, 0);
             *issued_slot = issued;
         }
     } else if (warp == 1) {

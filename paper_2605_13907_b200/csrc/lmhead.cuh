@@ -55,6 +55,10 @@ constexpr int kEpiWarps = 8;
 constexpr int kMxThreads = 512;          // microscaling passes: warps 12..15 move the block scales into tensor memory
 constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kStages * kMxStageScaleBytes + kNumBarriers * 8 + 64;
 
+// Pacing of the CTAs of a launch (lmhead_common.cuh): stage fills per announcement, counters in the ring.
+constexpr int kPaceFills = 16;
+constexpr int kPaceRing = 4096;
+
 struct LmheadArgs {
     int64_t rows;          // valid rows handled by this launch
     int64_t row0;          // global index of local row 0 (per-row vectors are indexed globally)
@@ -87,6 +91,8 @@ struct LmheadArgs {
     int64_t lddh;
     uint32_t* status;
     int64_t wait_cycles;   // bound of every device-side wait in clock ticks; 0 = the default (about two seconds)
+    uint32_t* pace;        // ring of kPaceRing zeroed counters that keeps the CTAs of the launch in step; NULL = no pacing
+    int32_t pace_per_unit; // announcements per unit = ceil(largest number of stage fills of a unit / fills per announcement)
 };
 
 // Launches one pass.  tmSA / tmSB are only read in kFwdFp8 mode.

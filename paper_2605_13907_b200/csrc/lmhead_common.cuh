@@ -22,6 +22,44 @@ struct Pipe {
     }
 };
 
+// Pacing of the persistent CTAs of one launch.  CTAs that share operand tiles through L2 (the column slices of a row
+// pair, the row tiles of a vocabulary range) only hit there while they stay within a few dozen stage fills of each
+// other, and left alone they drift apart by several per cent of a unit per unit.  Each CTA's producer therefore
+// announces every kPaceFills-th stage fill of its n-th unit on a ring of counters in the workspace and lets the slowest
+// CTA catch up to within kPaceLag announcements before it goes on.  The wait is advisory and bounded: after
+// kPaceWait clock ticks the producer goes on regardless, and after three such give-ups in a row it stops waiting
+// for the rest of the launch (it still announces), so CTAs that are not all resident at once cost time, not progress.
+// Every announcement index receives exactly gridDim.x arrivals: units without work and the missing units of the
+// last wave are announced in one go.
+constexpr int kPaceLag = 2;
+constexpr long long kPaceWait = 200000;  // clock ticks
+
+struct Pacer {
+    uint32_t* ring;      // nullptr: no pacing
+    int per_unit;        // announcements per unit (the same for every unit of the launch)
+    int strikes = 0;
+    __device__ Pacer(uint32_t* r, int c) : ring(r), per_unit(c) {}
+    __device__ __forceinline__ void announce(int n, int c) {
+        const long long k = static_cast<long long>(n) * per_unit + c;
+        atomicAdd(&ring[k % kPaceRing], 1u);
+        const long long kw = k - kPaceLag;
+        if (kw < 0 || strikes >= 3) return;
+        const uint32_t want = static_cast<uint32_t>(gridDim.x) * static_cast<uint32_t>(kw / kPaceRing + 1);
+        const volatile uint32_t* slot = ring + (kw % kPaceRing);
+        if (*slot >= want) { strikes = 0; return; }
+        const long long t0 = clock64();
+        while (*slot < want) {
+            if (clock64() - t0 > kPaceWait) { ++strikes; return; }
+        }
+        strikes = 0;
+    }
+    // announcements c_from .. per_unit - 1 of unit n without waiting (unit ended early, had no work, or does not exist)
+    __device__ __forceinline__ void top_up(int n, int c_from) {
+        for (int c = c_from; c < per_unit; ++c)
+            atomicAdd(&ring[(static_cast<long long>(n) * per_unit + c) % kPaceRing], 1u);
+    }
+};
+
 // Warp-wide wait: every lane polls (so every lane observes the completed phase itself) and the outcome is
 // made uniform, because the tcgen05.ld / __syncwarp that follow need the whole warp.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
