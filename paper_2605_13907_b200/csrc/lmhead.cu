@@ -97,6 +97,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 for (int t = w.t0; t < w.t1 && ok; ++t) {
                     for (int ks = 0; ks < a.ksteps; ++ks, ++fills) {
                         if (pacer.ring && fills % kPaceFills == 0) pacer.announce(n, fills / kPaceFills);
+                        if (pacer.ring && fills % kPaceFills == kPaceSettle) pacer.settle();
                         if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                         uint8_t* sA = stage_base + st.idx * STG_BYTES;
                         uint8_t* sB = sA + A_BYTES;

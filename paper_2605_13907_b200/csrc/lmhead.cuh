@@ -57,6 +57,7 @@ constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kStages * kMxStageScal
 
 // Pacing of the CTAs of a launch (lmhead_common.cuh): stage fills per announcement, counters in the ring.
 constexpr int kPaceFills = 16;
+constexpr int kPaceSettle = 4;     // stage fills between an announcement and the look at the counter it waits for
 constexpr int kPaceRing = 4096;
 
 struct LmheadArgs {

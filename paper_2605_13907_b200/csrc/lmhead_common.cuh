@@ -38,20 +38,30 @@ struct Pacer {
     uint32_t* ring;      // nullptr: no pacing
     int per_unit;        // announcements per unit (the same for every unit of the launch)
     int strikes = 0;
+    const volatile uint32_t* slot = nullptr;   // counter this CTA still has to see reach `want` (nullptr: nothing pending)
+    uint32_t want = 0, seen = 0;
     __device__ Pacer(uint32_t* r, int c) : ring(r), per_unit(c) {}
+    // Announcement c of unit n.  The counter to wait for is read here and looked at in settle(), a few stage fills
+    // later, so that the read's round trip to L2 is not spent waiting.
     __device__ __forceinline__ void announce(int n, int c) {
         const long long k = static_cast<long long>(n) * per_unit + c;
         atomicAdd(&ring[k % kPaceRing], 1u);
         const long long kw = k - kPaceLag;
         if (kw < 0 || strikes >= 3) return;
-        const uint32_t want = static_cast<uint32_t>(gridDim.x) * static_cast<uint32_t>(kw / kPaceRing + 1);
-        const volatile uint32_t* slot = ring + (kw % kPaceRing);
-        if (*slot >= want) { strikes = 0; return; }
-        const long long t0 = clock64();
-        while (*slot < want) {
-            if (clock64() - t0 > kPaceWait) { ++strikes; return; }
+        want = static_cast<uint32_t>(gridDim.x) * static_cast<uint32_t>(kw / kPaceRing + 1);
+        slot = ring + (kw % kPaceRing);
+        seen = *slot;
+    }
+    __device__ __forceinline__ void settle() {
+        if (slot == nullptr) return;
+        if (seen < want) {
+            const long long t0 = clock64();
+            while (*slot < want) {
+                if (clock64() - t0 > kPaceWait) { ++strikes; slot = nullptr; return; }
+            }
         }
         strikes = 0;
+        slot = nullptr;
     }
     // announcements c_from .. per_unit - 1 of unit n without waiting (unit ended early, had no work, or does not exist)
     __device__ __forceinline__ void top_up(int n, int c_from) {

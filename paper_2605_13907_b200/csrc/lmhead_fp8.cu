@@ -111,6 +111,7 @@ lmhead_fp8_block_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     for (int t = w.t0; t < w.t1 && ok; ++t) {
                         for (int ks = 0; ks < a.ksteps; ++ks, ++fills) {
                             if (pacer.ring && fills % kPaceFills == 0) pacer.announce(n, fills / kPaceFills);
+                            if (pacer.ring && fills % kPaceFills == kPaceSettle) pacer.settle();
                             if (!mbar_wait(&empty[st.idx], st.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                             if (!mbar_wait(&sempty[sc.idx], sc.phase ^ 1u, abort_flag, a.wait_cycles)) { ok = false; break; }
                             uint8_t* sA = stage_base + st.idx * kStageBytes;
